@@ -1,0 +1,179 @@
+/*
+ * gcn_admm.h -- C ABI of the community-based ADMM trainer for graph convolutional networks
+ * (single GPU, sm_100a).
+ *
+ * The calls follow the paper's statement of the problem: Algorithm 1 requires Y, Z_0, nu and
+ * rho and returns Z_{l,m} and W_l; Problem 1 fixes the network (A~ = (D+I)^-1/2 (A+I) (D+I)^-1/2,
+ * layer widths C_0..C_L, Z_l = f_l(A~ Z_{l-1} W_l)); Section 2 fixes the community split.
+ *
+ * General rules
+ *  - Every function returns GCN_ADMM_OK (0) or a negative error code; no exception, abort or
+ *    exit crosses this boundary.  After an error the handle stays valid for
+ *    gcn_admm_last_error() and gcn_admm_destroy().
+ *  - Pointers are plain host pointers unless a parameter says "host or device": those are
+ *    classified with cudaPointerGetAttributes and copied accordingly.
+ *  - All inputs are copied during gcn_admm_create(); the caller may free them afterwards.
+ *    All outputs are caller-allocated and written in the caller's (original) node order; the
+ *    community reordering is internal.
+ *  - Matrices cross the boundary dense and row-major without padding.
+ *  - A handle is not thread-safe; distinct handles are independent.  All device work of a
+ *    handle is enqueued on the stream given at creation; calls return after that work has
+ *    been enqueued, except where an output is a host buffer (then the call synchronises).
+ *  - There is no CPU fallback: every call fails with GCN_ADMM_ERR_CUDA when no usable CUDA
+ *    device is present.
+ */
+#ifndef GCN_ADMM_H
+#define GCN_ADMM_H
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gcn_admm gcn_admm; /* opaque, owned by the library */
+
+enum {
+  GCN_ADMM_OK = 0,
+  GCN_ADMM_ERR_ARG = -1,       /* NULL pointer, non-positive size, unknown selector */
+  GCN_ADMM_ERR_GRAPH = -2,     /* CSR not monotone / column out of range / unsorted or duplicate
+                                  columns / not symmetric / more than 2^31-1 stored entries */
+  GCN_ADMM_ERR_COMMUNITY = -3, /* community id outside 0..M-1, or an empty community */
+  GCN_ADMM_ERR_WIDTHS = -4,    /* a width < 1, fewer than 1 layer, C_L > 128, label >= C_L */
+  GCN_ADMM_ERR_ALLOC = -5,     /* host or device allocation failed */
+  GCN_ADMM_ERR_CUDA = -6,      /* any CUDA runtime failure, including "no device" */
+  GCN_ADMM_ERR_NONFINITE = -7  /* a NaN or infinity reached a step-size decision */
+};
+
+/* Parameters.  nu: penalty of the relaxed hidden-layer constraints (Problem 2).  rho: penalty of
+ * the augmented Lagrangian (Eq. 1).  The remaining fields fix what the paper leaves open:
+ *  tau0, theta0    initial step parameters of the quadratic approximations (Section 3.1, Eq. 8)
+ *  bt_shrink       a search starts from max(previous * bt_shrink, 1e-12)
+ *  bt_growth       and multiplies by bt_growth (> 1) until the condition of Section 3.1 / Eq. 9,
+ *                  in the form f(x - g/t) <= f(x) - ||g||^2/(2t), holds
+ *  bt_max_trials   at most this many trials (1..64); an exhausted block is left unchanged
+ *  fista_iters     iterations of FISTA on the training rows of Eq. 7 (constant step
+ *                  1/(loss_scale/2 + rho), t_1 = 1, warm start, no early exit)
+ *  loss_scale      R = loss_scale * sum over training rows of the softmax cross-entropy
+ *  dual_mode       0: Eq. 3 as printed (Z_L^k, Z_{L-1}^k, W_L^{k+1}); 1: the k+1 iterates
+ *  w_init          L host pointers to row-major C_{l-1} x C_l matrices (required)
+ *  device          CUDA device ordinal;  stream: a cudaStream_t owned by the caller (NULL = the
+ *                  default stream) */
+typedef struct {
+  float nu, rho;
+  float tau0, theta0;
+  float bt_growth, bt_shrink;
+  int bt_max_trials;
+  int fista_iters;
+  float loss_scale;
+  int dual_mode;
+  const float* const* w_init;
+  int device;
+  void* stream;
+} gcn_admm_params;
+
+/* Fills *p with the defaults: nu = rho = 1e-3, tau0 = theta0 = 1, growth 2, shrink 0.5,
+ * 40 trials, 30 FISTA iterations, loss_scale 1, dual_mode 0, device 0, stream NULL, w_init NULL. */
+void gcn_admm_default_params(gcn_admm_params* p);
+
+/* Builds the problem of Algorithm 1 (its REQUIRE line) on the device.
+ *  n                 number of nodes N
+ *  row_ptr, col_idx  CSR pattern of the undirected, unweighted adjacency A (host or device):
+ *                    row_ptr[n+1] ascending from 0, columns strictly ascending inside a row,
+ *                    symmetric.  Diagonal entries are dropped; the identity of A~ is added here.
+ *  X                 Z_0, n x C_0 (host or device)
+ *  y                 class id per node, 0..C_L-1 (only rows with train_mask != 0 are read as labels)
+ *  train_mask        n bytes, non-zero = the node's loss term is part of R
+ *  n_layers, widths  L and C_0..C_L (widths has n_layers+1 entries)
+ *  n_comm, community M and the community id 0..M-1 of every node (Section 2); every community
+ *                    must be non-empty
+ * Work done here (none of it is part of an ADMM iteration): community reordering (nodes sorted by
+ * (community, original id)), A+I in that order with ascending columns, (D+I)^-1/2, the row-segment
+ * table that splits each row by the community of its columns (the blocks A~_{m,r} of Section 2),
+ * P_1 = A~ Z_0, and the initial state: W = w_init, Z from the forward pass of Problem 1, U = 0,
+ * tau_l = tau0, theta_{l,m} = theta0.
+ * On success *out receives the handle. */
+int gcn_admm_create(gcn_admm** out, long long n, const long long* row_ptr, const int* col_idx,
+                    const float* X, const int* y, const unsigned char* train_mask, int n_layers,
+                    const int* widths, const gcn_admm_params* p, int n_comm, const int* community);
+
+/* Runs n_iters passes of Algorithm 1: every W_l (Section 3.1), then every Z_{l,m} (Appendix A,
+ * Eq. 5-10; Eq. 7 for l = L), then U (Eq. 3).  Updates inside a pass are Jacobi: each reads the
+ * previous pass's Z and U and this pass's W.  Device work only; returns after enqueueing. */
+int gcn_admm_step(gcn_admm* h, int n_iters);
+
+/* out[0] = L_rho of Eq. 1, out[1] = R, out[2] = sum over l<L of (nu/2)||Z_l - f_l(A~ Z_{l-1} W_l)||^2,
+ * out[3] = <U, r>, out[4] = (rho/2)||r||^2 with r = Z_L - A~ Z_{L-1} W_L, out[5] = training accuracy of
+ * gcn_admm_predict.  Host pointer; synchronises. */
+int gcn_admm_objective(gcn_admm* h, double out[6]);
+
+/* Copies W_layer (1-based, C_{layer-1} x C_layer, row-major) to the host buffer out. */
+int gcn_admm_weights(gcn_admm* h, int layer, float* out);
+
+/* Forward pass of Problem 1 with the current W (not the auxiliary Z).  logits: n x C_L, labels: n
+ * (row argmax, ties to the lowest class).  Either may be NULL.  Host pointers, original order. */
+int gcn_admm_predict(gcn_admm* h, float* logits, int* labels);
+
+void gcn_admm_destroy(gcn_admm* h);
+
+/* Text of the last error of this handle (or of the last failed create when h is NULL). */
+const char* gcn_admm_last_error(const gcn_admm* h);
+
+/* ---- propagation alone (the product A~ X of Problem 1) ---------------------------------------
+ * out = A~ x for an n x width matrix x in the original node order (host or device, both the same
+ * kind; out may not alias x).  Uses the handle's graph only; the ADMM state is untouched. */
+int gcn_admm_propagate(gcn_admm* h, const float* x, int width, float* out);
+
+/* ---- index tables (Section 2; Appendix A first paragraph) ------------------------------------
+ * Returns a pointer to a host int array owned by the handle (valid until the next call of this
+ * function with the same selector, or destroy) and its length.  New ids = position after sorting
+ * nodes by (community, original id).  comm is used by the per-community selectors only.
+ *  GCN_ADMM_IX_PERM        new id -> original id            [n]
+ *  GCN_ADMM_IX_INV_PERM    original id -> new id            [n]
+ *  GCN_ADMM_IX_COMM_PTR    V_m = new ids comm_ptr[m]..comm_ptr[m+1]-1   [M+1]
+ *  GCN_ADMM_IX_NBR         N_m, ascending                    (per community)
+ *  GCN_ADMM_IX_HALO1       new ids outside V_m adjacent to V_m, ascending (first-order rows)
+ *  GCN_ADMM_IX_HALO2       new ids outside V_m and HALO1 adjacent to HALO1, ascending (second order)
+ *  GCN_ADMM_IX_CSR_ROW_PTR, GCN_ADMM_IX_CSR_COL   pattern of A+I in new ids  [n+1], [nnz]
+ *  GCN_ADMM_IX_SEG_ROW_PTR [n+1], GCN_ADMM_IX_SEG_COMM [S], GCN_ADMM_IX_SEG_BEGIN [S+1]
+ *       row i owns segments seg_row_ptr[i]..seg_row_ptr[i+1]-1; segment s covers positions
+ *       seg_begin[s]..seg_begin[s+1]-1 of csr_col, whose columns all lie in community seg_comm[s]. */
+enum {
+  GCN_ADMM_IX_PERM = 0, GCN_ADMM_IX_INV_PERM, GCN_ADMM_IX_COMM_PTR, GCN_ADMM_IX_NBR,
+  GCN_ADMM_IX_HALO1, GCN_ADMM_IX_HALO2, GCN_ADMM_IX_CSR_ROW_PTR, GCN_ADMM_IX_CSR_COL,
+  GCN_ADMM_IX_SEG_ROW_PTR, GCN_ADMM_IX_SEG_COMM, GCN_ADMM_IX_SEG_BEGIN
+};
+int gcn_admm_index(gcn_admm* h, int which, int comm, const int** data, long long* len);
+
+/* ---- state access (checkpointing and single-block tests) -------------------------------------
+ * Host buffers, dense row-major, original node order.
+ *  GCN_ADMM_ST_W      layer 1..L   float  C_{l-1} x C_l
+ *  GCN_ADMM_ST_Z      layer 1..L   float  n x C_l
+ *  GCN_ADMM_ST_U      layer ignored float n x C_L
+ *  GCN_ADMM_ST_TAU    layer 1..L   double [1]
+ *  GCN_ADMM_ST_THETA  layer 1..L-1 double [M] */
+enum { GCN_ADMM_ST_W = 0, GCN_ADMM_ST_Z, GCN_ADMM_ST_U, GCN_ADMM_ST_TAU, GCN_ADMM_ST_THETA };
+int gcn_admm_get_state(gcn_admm* h, int which, int layer, void* out);
+int gcn_admm_set_state(gcn_admm* h, int which, int layer, const void* in);
+
+/* Runs one block family of Algorithm 1 on the current state and nothing else:
+ *  GCN_ADMM_PHASE_W, layer l    W_l update (Section 3.1)
+ *  GCN_ADMM_PHASE_Z, layer l<L  every Z_{l,m}, m = 1..M (Eq. 5/6, 8-10), with the stored W as W^{k+1}
+ *  GCN_ADMM_PHASE_Z, layer L    Z_L (Eq. 7)
+ *  GCN_ADMM_PHASE_U             U + rho (Z_L - A~ Z_{L-1} W_L) on the stored iterates (Eq. 3) */
+enum { GCN_ADMM_PHASE_W = 0, GCN_ADMM_PHASE_Z = 1, GCN_ADMM_PHASE_U = 2 };
+int gcn_admm_step_block(gcn_admm* h, int phase, int layer);
+
+/* Step-size decisions of the most recent gcn_admm_step / gcn_admm_step_block call, oldest pass first
+ * (at most the last 256 passes are kept).  trial: accepted trial index j (t = start * growth^j),
+ * -1 = skipped (||g||^2 <= 1e-24 ||x||^2), -2 = exhausted, -3 = block not run in that pass.
+ * q = (f(x) - f(x+)) / (||g||^2/(2t)) at the accepted trial (the condition is q >= 1).
+ *  trial_w, q_w   [passes x L]           index pass*L + (l-1)
+ *  trial_z, q_z   [passes x (L-1) x M]   index (pass*(L-1) + (l-1))*M + m
+ * Any pointer may be NULL.  *n_passes receives the number of passes logged; the arrays must hold
+ * max_passes passes and at most that many are written.  Synchronises. */
+int gcn_admm_decisions(gcn_admm* h, int max_passes, int* n_passes, int* trial_w, double* q_w,
+                       int* trial_z, double* q_z);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GCN_ADMM_H */

@@ -212,6 +212,7 @@ class OracleADMM:
         self.L = len(widths) - 1
         self.widths = list(widths)
         self.M = int(n_comm)
+        self.forced_tol = 1e-6    # replay mode: slack on the condition q >= 1 of a forced trial
         self.At = normalized_adjacency(n, row_ptr, col_idx)
         self.y = np.asarray(y, dtype=np.int64)
         self.train = np.asarray(train_mask).astype(bool)
@@ -281,8 +282,14 @@ class OracleADMM:
             t = t * p.bt_growth ** forced
             xn = x - g / t
             q = (f0 - float(fun(xn))) / (gg / (2.0 * t))
-            return xn, t, dict(trial=int(forced), t=t, q=q, margin=abs(q - 1.0), gg=gg,
-                               ok=bool(q >= 1.0 - 1e-6), f0=f0)
+            q_prev = -np.inf          # the trial before the forced one must not have passed
+            if forced > 0:
+                tp = t / p.bt_growth
+                q_prev = (f0 - float(fun(x - g / tp))) / (gg / (2.0 * tp))
+            tol = self.forced_tol
+            return xn, t, dict(trial=int(forced), t=t, q=q, q_reject=q_prev, gg=gg, f0=f0,
+                               margin=min(abs(q - 1.0), abs(q_prev - 1.0)),
+                               ok=bool(q >= 1.0 - tol and q_prev < 1.0 + tol))
         q_reject = np.inf
         for trial in range(p.bt_max_trials):
             xn = x - g / t

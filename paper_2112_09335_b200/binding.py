@@ -1,0 +1,209 @@
+"""ctypes binding of ``libgcn_admm.so``: argument marshalling only.
+
+Every function of ``include/gcn_admm.h`` has a counterpart of the same name on ``GcnAdmm``
+(without the ``gcn_admm_`` prefix).  Nothing is computed here; the library must have been built
+(``python -m paper_2112_09335_b200.build``) or loading fails with an error -- there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libgcn_admm.so")
+
+EXPORTS = [
+    "gcn_admm_default_params", "gcn_admm_create", "gcn_admm_step", "gcn_admm_objective", "gcn_admm_weights",
+    "gcn_admm_predict", "gcn_admm_destroy", "gcn_admm_last_error", "gcn_admm_propagate", "gcn_admm_index",
+    "gcn_admm_get_state", "gcn_admm_set_state", "gcn_admm_step_block", "gcn_admm_decisions",
+]
+
+IX = dict(perm=0, inv_perm=1, comm_ptr=2, nbr=3, halo1=4, halo2=5, csr_row_ptr=6, csr_col=7,
+          seg_row_ptr=8, seg_comm=9, seg_begin=10)
+ST_W, ST_Z, ST_U, ST_TAU, ST_THETA = range(5)
+PHASE_W, PHASE_Z, PHASE_U = range(3)
+
+
+class Params(C.Structure):
+    _fields_ = [("nu", C.c_float), ("rho", C.c_float), ("tau0", C.c_float), ("theta0", C.c_float),
+                ("bt_growth", C.c_float), ("bt_shrink", C.c_float), ("bt_max_trials", C.c_int),
+                ("fista_iters", C.c_int), ("loss_scale", C.c_float), ("dual_mode", C.c_int),
+                ("w_init", C.POINTER(C.POINTER(C.c_float))), ("device", C.c_int), ("stream", C.c_void_p)]
+
+
+class GcnAdmmError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__(f"gcn_admm error {code}: {msg}")
+        self.code = code
+
+
+_lib = None
+
+
+def load():
+    """Loads the shared library (once) and declares the signatures."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(f"{LIB_PATH} is missing: build it with `python -m paper_2112_09335_b200.build`")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64 = C.c_void_p, C.c_int, C.c_longlong
+    lib.gcn_admm_default_params.argtypes = [C.POINTER(Params)]
+    lib.gcn_admm_default_params.restype = None
+    lib.gcn_admm_create.argtypes = [C.POINTER(vp), i64, vp, vp, vp, vp, vp, i32, C.POINTER(i32), C.POINTER(Params),
+                                    i32, vp]
+    lib.gcn_admm_step.argtypes = [vp, i32]
+    lib.gcn_admm_objective.argtypes = [vp, C.POINTER(C.c_double)]
+    lib.gcn_admm_weights.argtypes = [vp, i32, vp]
+    lib.gcn_admm_predict.argtypes = [vp, vp, vp]
+    lib.gcn_admm_destroy.argtypes = [vp]
+    lib.gcn_admm_destroy.restype = None
+    lib.gcn_admm_last_error.argtypes = [vp]
+    lib.gcn_admm_last_error.restype = C.c_char_p
+    lib.gcn_admm_propagate.argtypes = [vp, vp, i32, vp]
+    lib.gcn_admm_index.argtypes = [vp, i32, i32, C.POINTER(C.POINTER(i32)), C.POINTER(i64)]
+    lib.gcn_admm_get_state.argtypes = [vp, i32, i32, vp]
+    lib.gcn_admm_set_state.argtypes = [vp, i32, i32, vp]
+    lib.gcn_admm_step_block.argtypes = [vp, i32, i32]
+    lib.gcn_admm_decisions.argtypes = [vp, i32, C.POINTER(i32), vp, vp, vp, vp]
+    _lib = lib
+    return lib
+
+
+def _ptr(a):
+    """Address of a numpy array, or the raw value of an int (a device pointer)."""
+    if a is None:
+        return None
+    if isinstance(a, int):
+        return C.c_void_p(a)
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def default_params() -> Params:
+    p = Params()
+    load().gcn_admm_default_params(C.byref(p))
+    return p
+
+
+class GcnAdmm:
+    """Owner of one library handle.  Array arguments are numpy arrays (host) or, for ``create``'s
+    graph / feature inputs and ``propagate``, integers holding device addresses."""
+
+    def __init__(self, n, row_ptr, col_idx, X, y, train_mask, widths, n_comm, community, w_init, nu=1e-3, rho=1e-3,
+                 tau0=1.0, theta0=1.0, bt_growth=2.0, bt_shrink=0.5, bt_max_trials=40, fista_iters=30,
+                 loss_scale=1.0, dual_mode=0, device=0, stream=0):
+        lib = load()
+        self._lib = lib
+        self._h = C.c_void_p()
+        self.n, self.widths, self.n_comm = int(n), [int(w) for w in widths], int(n_comm)
+        self.L = len(self.widths) - 1
+        p = default_params()
+        p.nu, p.rho, p.tau0, p.theta0 = nu, rho, tau0, theta0
+        p.bt_growth, p.bt_shrink, p.bt_max_trials = bt_growth, bt_shrink, bt_max_trials
+        p.fista_iters, p.loss_scale, p.dual_mode = fista_iters, loss_scale, dual_mode
+        p.device, p.stream = device, stream or None
+        ws = [np.ascontiguousarray(w, dtype=np.float32) for w in w_init]
+        arr = (C.POINTER(C.c_float) * len(ws))(*[w.ctypes.data_as(C.POINTER(C.c_float)) for w in ws])
+        p.w_init = C.cast(arr, C.POINTER(C.POINTER(C.c_float)))
+        keep = []
+
+        def host(a, dt):
+            if isinstance(a, int):
+                return a
+            b = np.ascontiguousarray(a, dtype=dt)
+            keep.append(b)
+            return b
+        wd = (C.c_int * len(self.widths))(*self.widths)
+        rc = lib.gcn_admm_create(C.byref(self._h), self.n, _ptr(host(row_ptr, np.int64)), _ptr(host(col_idx, np.int32)),
+                                 _ptr(host(X, np.float32)), _ptr(host(y, np.int32)),
+                                 _ptr(host(train_mask, np.uint8)), self.L, wd, C.byref(p), self.n_comm,
+                                 _ptr(host(community, np.int32)))
+        if rc != 0:
+            raise GcnAdmmError(rc, lib.gcn_admm_last_error(None).decode())
+
+    def _check(self, rc):
+        if rc != 0:
+            raise GcnAdmmError(rc, self._lib.gcn_admm_last_error(self._h).decode())
+
+    def destroy(self):
+        if getattr(self, "_h", None) and self._h.value:
+            self._lib.gcn_admm_destroy(self._h)
+            self._h = C.c_void_p()
+
+    __del__ = destroy
+
+    def step(self, n_iters=1):
+        self._check(self._lib.gcn_admm_step(self._h, int(n_iters)))
+
+    def step_block(self, phase, layer=0):
+        self._check(self._lib.gcn_admm_step_block(self._h, int(phase), int(layer)))
+
+    def objective(self):
+        out = (C.c_double * 6)()
+        self._check(self._lib.gcn_admm_objective(self._h, out))
+        return np.array(out[:])
+
+    def weights(self, layer):
+        out = np.empty((self.widths[layer - 1], self.widths[layer]), dtype=np.float32)
+        self._check(self._lib.gcn_admm_weights(self._h, layer, _ptr(out)))
+        return out
+
+    def predict(self):
+        logits = np.empty((self.n, self.widths[-1]), dtype=np.float32)
+        labels = np.empty(self.n, dtype=np.int32)
+        self._check(self._lib.gcn_admm_predict(self._h, _ptr(logits), _ptr(labels)))
+        return logits, labels
+
+    def propagate(self, x, width=None, out=None):
+        """A~ x.  numpy in -> numpy out; device addresses (ints) in -> ``out`` must be given."""
+        if isinstance(x, int):
+            self._check(self._lib.gcn_admm_propagate(self._h, _ptr(x), int(width), _ptr(out)))
+            return out
+        x = np.ascontiguousarray(x, dtype=np.float32)
+        res = np.empty_like(x)
+        self._check(self._lib.gcn_admm_propagate(self._h, _ptr(x), x.shape[1], _ptr(res)))
+        return res
+
+    def index(self, which, comm=0):
+        data = C.POINTER(C.c_int)()
+        length = C.c_longlong()
+        self._check(self._lib.gcn_admm_index(self._h, IX[which], int(comm), C.byref(data), C.byref(length)))
+        if length.value == 0:
+            return np.zeros(0, dtype=np.int32)
+        return np.ctypeslib.as_array(data, shape=(length.value,)).copy()
+
+    def _state_shape(self, which, layer):
+        if which == ST_W:
+            return (self.widths[layer - 1], self.widths[layer]), np.float32
+        if which == ST_Z:
+            return (self.n, self.widths[layer]), np.float32
+        if which == ST_U:
+            return (self.n, self.widths[-1]), np.float32
+        if which == ST_TAU:
+            return (1,), np.float64
+        return (self.n_comm,), np.float64
+
+    def get_state(self, which, layer=0):
+        shape, dt = self._state_shape(which, layer)
+        out = np.empty(shape, dtype=dt)
+        self._check(self._lib.gcn_admm_get_state(self._h, which, layer, _ptr(out)))
+        return out
+
+    def set_state(self, which, layer, value):
+        shape, dt = self._state_shape(which, layer)
+        v = np.ascontiguousarray(value, dtype=dt).reshape(shape)
+        self._check(self._lib.gcn_admm_set_state(self._h, which, layer, _ptr(v)))
+
+    def decisions(self, max_passes=256):
+        L, M = self.L, self.n_comm
+        n = C.c_int()
+        tw = np.empty((max_passes, L), dtype=np.int32)
+        qw = np.empty((max_passes, L), dtype=np.float64)
+        tz = np.empty((max_passes, max(L - 1, 0), M), dtype=np.int32)
+        qz = np.empty((max_passes, max(L - 1, 0), M), dtype=np.float64)
+        self._check(self._lib.gcn_admm_decisions(self._h, max_passes, C.byref(n), _ptr(tw), _ptr(qw), _ptr(tz), _ptr(qz)))
+        k = n.value
+        return dict(trial_w=tw[:k], q_w=qw[:k], trial_z=tz[:k], q_z=qz[:k])

@@ -1,0 +1,893 @@
+// C-ABI library of the community-based ADMM GCN trainer: host orchestration of the kernels in
+// kernels.cuh.  See include/gcn_admm.h for the contract of every entry point.
+#include "../../include/gcn_admm.h"
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "graph_index.hpp"
+#include "kernels.cuh"
+
+using gcn_admm_host::GraphIndex;
+using gk::SearchCtl;
+
+namespace {
+
+constexpr int kLogPasses = 256;
+constexpr int kSmCount = 148;
+
+thread_local std::string g_create_error;
+
+inline int ldpad(int c) { return (c + 3) & ~3; }
+inline long long cdiv(long long a, long long b) { return (a + b - 1) / b; }
+
+struct Fail {
+  int code;
+  std::string msg;
+};
+
+#define CU(expr)                                                                           \
+  do {                                                                                     \
+    cudaError_t e__ = (expr);                                                              \
+    if (e__ != cudaSuccess)                                                                \
+      throw Fail{GCN_ADMM_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e__)};  \
+  } while (0)
+
+template <typename T>
+T* dalloc(size_t count) {
+  void* p = nullptr;
+  cudaError_t e = cudaMalloc(&p, std::max<size_t>(count, 1) * sizeof(T));
+  if (e != cudaSuccess)
+    throw Fail{e == cudaErrorMemoryAllocation ? GCN_ADMM_ERR_ALLOC : GCN_ADMM_ERR_CUDA,
+               std::string("cudaMalloc: ") + cudaGetErrorString(e)};
+  return static_cast<T*>(p);
+}
+
+bool is_device_pointer(const void* p) {
+  cudaPointerAttributes a;
+  if (cudaPointerGetAttributes(&a, p) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  return a.type == cudaMemoryTypeDevice || a.type == cudaMemoryTypeManaged;
+}
+
+}  // namespace
+
+struct gcn_admm {
+  gcn_admm_params p{};
+  cudaStream_t stream = nullptr;
+  int L = 0;
+  long long n = 0;
+  int M = 0;
+  int n_train = 0;
+  std::vector<int> C, ld;   // widths C_0..C_L and their padded leading dimensions
+  int max_ld = 0;
+  GraphIndex gi;
+  std::vector<void*> owned;  // every device allocation, for destroy
+
+  int *d_row_ptr = nullptr, *d_col = nullptr, *d_row_comm = nullptr, *d_perm = nullptr;
+  int *d_seg_row_ptr = nullptr, *d_seg_comm = nullptr, *d_seg_begin = nullptr, *d_y = nullptr;
+  float* d_dinv = nullptr;
+  unsigned char* d_train = nullptr;
+
+  std::vector<float*> W, Wt, Z, P, H;   // 1..L
+  float* U = nullptr;
+  float *B0 = nullptr, *B1 = nullptr, *B2 = nullptr;   // N x max_ld scratch
+  float* grad = nullptr;     // max over l of C_{l-1} x ld_l
+  float* part = nullptr;     // split partial sums of the transposed product
+  size_t part_elems = 0;
+  SearchCtl *ctl_w = nullptr, *ctl_z = nullptr;   // [L+1], [(L+1) * M]
+  double *sums_w = nullptr, *sums_z = nullptr, *acc_w = nullptr, *acc_z = nullptr, *obj = nullptr;
+  int *n_active = nullptr, *status = nullptr;
+  int *log_trial_w = nullptr, *log_trial_z = nullptr;
+  double *log_q_w = nullptr, *log_q_z = nullptr;
+  long long log_count = 0;
+  bool fresh = false;        // P_l, H_l agree with the stored W, Z
+  std::string err;
+  std::vector<int> ix_cache[16];
+
+  template <typename T>
+  T* alloc(size_t count) {
+    T* p_ = dalloc<T>(count);
+    owned.push_back(p_);
+    return p_;
+  }
+  int grid_for(long long work_items, int per_block = 256) const {
+    return (int)std::max<long long>(1, std::min<long long>(cdiv(work_items, per_block), (long long)kSmCount * 8));
+  }
+
+  // ---- launches -----------------------------------------------------------------------
+  void spmm(const float* x, float* out, int ldx) {
+    const int ld4 = ldx / 4;
+    const float4* x4 = reinterpret_cast<const float4*>(x);
+    float4* o4 = reinterpret_cast<float4*>(out);
+    const int nn = (int)n;
+#define SPMM_CASE(G, V)                                                                        \
+  {                                                                                            \
+    const long long threads = n * (G);                                                         \
+    gk::k_spmm<G, V><<<(unsigned)cdiv(threads, 256), 256, 0, stream>>>(d_row_ptr, d_col, d_dinv, x4, o4, nn, ld4); \
+  }
+    if (ld4 <= 1) SPMM_CASE(1, 1)
+    else if (ld4 <= 2) SPMM_CASE(2, 1)
+    else if (ld4 <= 4) SPMM_CASE(4, 1)
+    else if (ld4 <= 8) SPMM_CASE(8, 1)
+    else if (ld4 <= 16) SPMM_CASE(16, 1)
+    else if (ld4 <= 32) SPMM_CASE(32, 1)
+    else SPMM_CASE(32, 2)
+#undef SPMM_CASE
+    CU(cudaGetLastError());
+  }
+
+  void gemm_nn(const float* A, int lda, const float* B, int ldb, float* Cm, int ldc, long long Mr, int N, int K,
+               const int* skip = nullptr) {
+#define NN_CASE(BM, BN, BK, TM, TN)                                                             \
+  {                                                                                             \
+    dim3 grid((unsigned)cdiv(Mr, BM), (unsigned)cdiv(ldc, BN));                                  \
+    gk::k_gemm_nn<BM, BN, BK, TM, TN><<<grid, (BM / TM) * (BN / TN), 0, stream>>>(A, lda, B, ldb, Cm, ldc, (int)Mr, N, K, skip); \
+  }
+    if (N > 64) NN_CASE(128, 128, 16, 8, 8)
+    else if (N > 16) NN_CASE(128, 64, 16, 8, 4)
+    else NN_CASE(256, 16, 16, 4, 4)
+#undef NN_CASE
+    CU(cudaGetLastError());
+  }
+
+  // out[Ka x ldp] = A^T B over `rows` rows, through split partial sums reduced in a fixed order.
+  void gemm_tn(const float* A, int lda, const float* B, int ldb, float* out, int ldp, long long rows, int Ka,
+               int Nb) {
+    int splits = 1;
+    long long rps = rows;
+#define TN_CASE(BM, BN, BK, TM, TN)                                                             \
+  {                                                                                             \
+    const long long tiles = cdiv(Ka, BM) * cdiv(ldp, BN);                                        \
+    splits = (int)std::max<long long>(1, std::min<long long>((4LL * kSmCount) / tiles, cdiv(rows, 64))); \
+    splits = (int)std::min<long long>(splits, (long long)(part_elems / ((size_t)Ka * ldp)));     \
+    rps = cdiv(rows, splits);                                                                    \
+    splits = (int)cdiv(rows, rps);                                                               \
+    dim3 grid((unsigned)cdiv(Ka, BM), (unsigned)cdiv(ldp, BN), (unsigned)splits);                \
+    gk::k_gemm_tn<BM, BN, BK, TM, TN><<<grid, (BM / TM) * (BN / TN), 0, stream>>>(A, lda, B, ldb, part, ldp, rows, rps, Ka, Nb); \
+  }
+    if (Nb > 64) TN_CASE(128, 128, 16, 8, 8)
+    else if (Nb > 16) TN_CASE(128, 64, 16, 8, 4)
+    else if (Nb > 8) TN_CASE(128, 16, 16, 8, 1)
+    else TN_CASE(128, 8, 16, 4, 1)
+#undef TN_CASE
+    CU(cudaGetLastError());
+    const long long elems = (long long)Ka * ldp;
+    gk::k_reduce_splits<<<(unsigned)cdiv(elems, 256), 256, 0, stream>>>(part, out, elems, splits);
+    CU(cudaGetLastError());
+  }
+
+  void resid(int l, float* R) {   // derivative of phi_l with respect to H_l, at the stored H_l
+    const long long n4 = n * ld[l] / 4;
+    if (l < L)
+      gk::k_resid_hidden<<<grid_for(n4), 256, 0, stream>>>((const float4*)H[l], (const float4*)Z[l], (float4*)R, n4, p.nu);
+    else
+      gk::k_resid_out<<<grid_for(n4), 256, 0, stream>>>((const float4*)H[l], (const float4*)Z[l], (const float4*)U,
+                                                        (float4*)R, n4, p.rho);
+    CU(cudaGetLastError());
+  }
+
+  int n_passes() const { return (p.bt_max_trials + gk::kCand - 1) / gk::kCand; }
+
+  int* log_slot_trial_w() { return log_trial_w + (log_count % kLogPasses) * L; }
+  double* log_slot_q_w() { return log_q_w + (log_count % kLogPasses) * L; }
+  int* log_slot_trial_z() { return log_trial_z + (log_count % kLogPasses) * (long long)std::max(L - 1, 0) * M; }
+  double* log_slot_q_z() { return log_q_z + (log_count % kLogPasses) * (long long)std::max(L - 1, 0) * M; }
+
+  void begin_log_pass() {
+    const long long zc = (long long)std::max(L - 1, 0) * M;
+    gk::k_fill_int<<<1, 64, 0, stream>>>(log_slot_trial_w(), L, -3);
+    if (zc > 0) gk::k_fill_int<<<grid_for(zc), 256, 0, stream>>>(log_slot_trial_z(), zc, -3);
+    CU(cudaGetLastError());
+  }
+
+  // ---- W_l block (Section 3.1) --------------------------------------------------------
+  void update_W(int l) {
+    const int Kp = C[l - 1], Cn = C[l], ldc = ld[l];
+    const long long n4 = n * ldc / 4;
+    SearchCtl* ctl = ctl_w + l;
+    resid(l, B0);                                                       // R_l
+    gemm_tn(P[l], ld[l - 1], B0, ldc, grad, ldc, n, Kp, Cn);            // grad = P_l^T R_l
+    gk::k_two_sumsq<<<1, 1024, 0, stream>>>(grad, W[l], (long long)Kp * ldc, sums_w);
+    gk::k_search_begin<<<1, 32, 0, stream>>>(ctl, 1, sums_w, 2, p.bt_shrink, p.bt_growth, acc_w, gk::kCand, nullptr);
+    CU(cudaGetLastError());
+    gemm_nn(P[l], ld[l - 1], grad, ldc, B1, ldc, n, Cn, Kp, &ctl->done);   // D = P_l grad
+    gk::DecideArgs a{};
+    a.growth = p.bt_growth;
+    a.max_trials = p.bt_max_trials;
+    if (l == L) {
+      gk::k_score_w_out<<<grid_for(n4), 256, 0, stream>>>((const float4*)B1, (const float4*)B0, n4, ctl, acc_w);
+      a.mode = 1;
+      a.quad_coef = 0.5 * p.rho;
+      a.last_pass = 1;
+      gk::k_search_decide<<<1, 32, 0, stream>>>(ctl, 1, acc_w, gk::kCand, nullptr, 0, a, nullptr, status);
+    } else {
+      a.mode = 0;
+      a.scale = 0.5 * p.nu;
+      const int passes = n_passes();
+      for (int ps = 0; ps < passes; ++ps) {
+        gk::k_score_w_hidden<<<grid_for(n4), 256, 0, stream>>>((const float4*)H[l], (const float4*)B1,
+                                                               (const float4*)Z[l], n4, ctl, acc_w);
+        a.last_pass = (ps == passes - 1);
+        gk::k_search_decide<<<1, 32, 0, stream>>>(ctl, 1, acc_w, gk::kCand, nullptr, 0, a, nullptr, status);
+      }
+    }
+    CU(cudaGetLastError());
+    gk::k_log_decisions<<<1, 32, 0, stream>>>(ctl, 1, log_slot_trial_w() + (l - 1), log_slot_q_w() + (l - 1));
+    gk::k_apply_w<<<(unsigned)cdiv((long long)Kp * Cn, 256), 256, 0, stream>>>(W[l], Wt[l], grad, Kp, Cn, ldc,
+                                                                               ld[l - 1], ctl);
+    gk::k_axpy_ctl<<<grid_for(n4), 256, 0, stream>>>((float4*)H[l], (const float4*)B1, n4, ctl);   // H_l at W^{k+1}
+    CU(cudaGetLastError());
+  }
+
+  // ---- Z_{l,m}, l < L, every community (Appendix A, Eq. 5/6 and 8-10) ------------------
+  void update_Z_hidden(int l) {
+    const int ldl = ld[l], ldn = ld[l + 1];
+    SearchCtl* ctl = ctl_z + (size_t)l * M;
+    resid(l + 1, B0);                                                    // R'_{l+1}
+    spmm(B0, B1, ldn);                                                   // S = A~ R'
+    gemm_nn(B1, ldn, Wt[l + 1], ldl, B2, ldl, n, C[l], C[l + 1]);        // S W_{l+1}^T
+    CU(cudaMemsetAsync(sums_z, 0, sizeof(double) * 3 * M, stream));
+    CU(cudaMemsetAsync(n_active, 0, sizeof(int), stream));
+    const int rows_per_block = 32;
+    gk::k_zgrad_finish<<<(unsigned)cdiv(n, rows_per_block), 256, 0, stream>>>(
+        (float4*)B2, (const float4*)Z[l], (const float4*)H[l], ldl / 4, n, rows_per_block, d_row_comm, p.nu, sums_z);
+    const bool out = (l + 1 == L);
+    const int per = out ? 2 : gk::kCand;
+    gk::k_search_begin<<<(unsigned)cdiv(M, 128), 128, 0, stream>>>(ctl, M, sums_z, 3, p.bt_shrink, p.bt_growth, acc_z,
+                                                                   per, n_active);
+    CU(cudaGetLastError());
+    gemm_nn(B2, ldl, W[l + 1], ldn, B1, ldn, n, C[l + 1], C[l]);         // T = G W_{l+1}
+    gk::DecideArgs a{};
+    a.growth = p.bt_growth;
+    a.max_trials = p.bt_max_trials;
+    a.own_nu = p.nu;
+    const int ld4 = ldn / 4;
+    const int warps = 8;
+    const unsigned grid = (unsigned)cdiv(n, warps);
+    const size_t smem = (size_t)M * per * sizeof(double);
+    const int use_smem = smem <= 40 * 1024;
+    const size_t dyn = use_smem ? smem : 0;
+#define SCORE_Z(V, OUT)                                                                                   \
+  gk::k_score_z<V, OUT><<<grid, warps * 32, dyn, stream>>>(d_col, d_dinv, d_seg_row_ptr, d_seg_comm, d_seg_begin, \
+      (const float4*)B1, (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0, ld4, (int)n, ctl, M, \
+      acc_z, n_active, use_smem)
+#define SCORE_Z_ANY(OUT)                    \
+  {                                         \
+    if (ld4 <= 32) SCORE_Z(1, OUT);         \
+    else if (ld4 <= 64) SCORE_Z(2, OUT);    \
+    else if (ld4 <= 128) SCORE_Z(4, OUT);   \
+    else SCORE_Z(8, OUT);                   \
+  }
+    if (out) {
+      SCORE_Z_ANY(true)
+      a.mode = 1;
+      a.quad_coef = 0.5 * p.rho;
+      a.last_pass = 1;
+      gk::k_search_decide<<<(unsigned)cdiv(M, 128), 128, 0, stream>>>(ctl, M, acc_z, per, sums_z, 3, a, n_active, status);
+    } else {
+      a.mode = 0;
+      a.scale = 0.5 * p.nu;
+      const int passes = n_passes();
+      for (int ps = 0; ps < passes; ++ps) {
+        SCORE_Z_ANY(false)
+        a.last_pass = (ps == passes - 1);
+        gk::k_search_decide<<<(unsigned)cdiv(M, 128), 128, 0, stream>>>(ctl, M, acc_z, per, sums_z, 3, a, n_active,
+                                                                        status);
+      }
+    }
+#undef SCORE_Z_ANY
+#undef SCORE_Z
+    CU(cudaGetLastError());
+    gk::k_log_decisions<<<(unsigned)cdiv(M, 128), 128, 0, stream>>>(ctl, M, log_slot_trial_z() + (size_t)(l - 1) * M,
+                                                                    log_slot_q_z() + (size_t)(l - 1) * M);
+    gk::k_apply_z<<<grid_for(n * (ldl / 4)), 256, 0, stream>>>((float4*)Z[l], (const float4*)B2, ldl / 4, n, d_row_comm, ctl);
+    CU(cudaGetLastError());
+  }
+
+  // ---- Z_L (Eq. 7) and, in the same sweep, the dual as printed in Eq. 3 -----------------
+  void update_output(bool dual_now, bool update_z) {
+    const int warps = 8;
+    gk::k_output_rows<<<(unsigned)cdiv(n, warps), warps * 32, 0, stream>>>(Z[L], U, H[L], ld[L], C[L], (int)n, d_y, d_train,
+                                                                           p.rho, p.loss_scale, p.fista_iters,
+                                                                           dual_now ? 1 : 0, update_z ? 1 : 0);
+    CU(cudaGetLastError());
+  }
+
+  void dual_from_stored() {   // U + rho (Z_L - H_L) with H_L = A~ Z_{L-1} W_L of the stored iterates
+    const long long n4 = n * ld[L] / 4;
+    gk::k_dual<<<grid_for(n4), 256, 0, stream>>>((float4*)U, (const float4*)Z[L], (const float4*)H[L], n4, p.rho);
+    CU(cudaGetLastError());
+  }
+
+  // P_l = A~ Z_{l-1} (l >= 2; P_1 is constant) and H_l = P_l W_l from the stored W, Z.
+  void refresh() {
+    for (int l = 2; l <= L; ++l) spmm(Z[l - 1], P[l], ld[l - 1]);
+    for (int l = 1; l <= L; ++l) gemm_nn(P[l], ld[l - 1], W[l], ld[l], H[l], ld[l], n, C[l], C[l - 1]);
+    fresh = true;
+  }
+
+  void iterate() {   // Algorithm 1, one pass
+    if (!fresh) refresh();
+    begin_log_pass();
+    for (int l = 1; l <= L; ++l) update_W(l);
+    for (int l = 1; l < L; ++l) update_Z_hidden(l);
+    update_output(p.dual_mode == 0, true);
+    refresh();
+    if (p.dual_mode != 0) dual_from_stored();
+    ++log_count;
+  }
+
+  // logits of Problem 1's forward pass with the stored W, left in B0 (N x ld_L)
+  void forward_logits() {
+    gemm_nn(P[1], ld[0], W[1], ld[1], B0, ld[1], n, C[1], C[0]);
+    for (int l = 1; l < L; ++l) {
+      const long long n4 = n * ld[l] / 4;
+      gk::k_relu_inplace<<<grid_for(n4), 256, 0, stream>>>((float4*)B0, n4);
+      CU(cudaGetLastError());
+      spmm(B0, B1, ld[l]);
+      gemm_nn(B1, ld[l], W[l + 1], ld[l + 1], B0, ld[l + 1], n, C[l + 1], C[l]);
+    }
+  }
+
+  void check_status() {
+    int s = 0;
+    CU(cudaMemcpyAsync(&s, status, sizeof(int), cudaMemcpyDeviceToHost, stream));
+    CU(cudaStreamSynchronize(stream));
+    if (s & 1) {
+      CU(cudaMemsetAsync(status, 0, sizeof(int), stream));
+      throw Fail{GCN_ADMM_ERR_NONFINITE, "a non-finite value reached a step-size decision"};
+    }
+  }
+
+  // rows in the caller's order (dense, width c) <-> internal (community order, padded)
+  void rows_to_host(const float* dev, int c, float* host_out) {
+    float* dense = B2;
+    gk::k_permute_rows<<<grid_for(n * ldpad(c)), 256, 0, stream>>>(dev, dense, d_perm, n, c, ldpad(c), 0);
+    CU(cudaGetLastError());
+    CU(cudaMemcpyAsync(host_out, dense, sizeof(float) * n * c, cudaMemcpyDeviceToHost, stream));
+    CU(cudaStreamSynchronize(stream));
+  }
+  void rows_from_host(const float* host_in, int c, float* dev) {
+    float* dense = B2;
+    CU(cudaMemcpyAsync(dense, host_in, sizeof(float) * n * c, cudaMemcpyHostToDevice, stream));
+    gk::k_permute_rows<<<grid_for(n * ldpad(c)), 256, 0, stream>>>(dense, dev, d_perm, n, c, ldpad(c), 1);
+    CU(cudaGetLastError());
+    CU(cudaStreamSynchronize(stream));
+  }
+  void upload_weight(int l, const float* host_w) {
+    const int r = C[l - 1], c = C[l];
+    std::vector<float> w((size_t)r * ld[l], 0.f), wt((size_t)c * ld[l - 1], 0.f);
+    for (int i = 0; i < r; ++i)
+      for (int j = 0; j < c; ++j) {
+        w[(size_t)i * ld[l] + j] = host_w[(size_t)i * c + j];
+        wt[(size_t)j * ld[l - 1] + i] = host_w[(size_t)i * c + j];
+      }
+    CU(cudaMemcpyAsync(W[l], w.data(), w.size() * sizeof(float), cudaMemcpyHostToDevice, stream));
+    CU(cudaMemcpyAsync(Wt[l], wt.data(), wt.size() * sizeof(float), cudaMemcpyHostToDevice, stream));
+    CU(cudaStreamSynchronize(stream));
+  }
+};
+
+namespace {
+
+template <typename F>
+int guarded(gcn_admm* h, F&& body) {
+  if (h == nullptr) return GCN_ADMM_ERR_ARG;
+  try {
+    cudaError_t e = cudaSetDevice(h->p.device);
+    if (e != cudaSuccess) throw Fail{GCN_ADMM_ERR_CUDA, std::string("cudaSetDevice: ") + cudaGetErrorString(e)};
+    body();
+    return GCN_ADMM_OK;
+  } catch (const Fail& f) {
+    h->err = f.msg;
+    return f.code;
+  } catch (const std::bad_alloc&) {
+    h->err = "host allocation failed";
+    return GCN_ADMM_ERR_ALLOC;
+  } catch (...) {
+    h->err = "unexpected failure";
+    return GCN_ADMM_ERR_CUDA;
+  }
+}
+
+template <typename T>
+std::vector<T> to_host(const T* p, size_t count) {
+  std::vector<T> v(count);
+  if (count == 0) return v;
+  if (is_device_pointer(p)) CU(cudaMemcpy(v.data(), p, count * sizeof(T), cudaMemcpyDeviceToHost));
+  else std::memcpy(v.data(), p, count * sizeof(T));
+  return v;
+}
+
+template <typename T>
+T* upload(gcn_admm* h, const std::vector<T>& v) {
+  T* d = h->alloc<T>(v.size());
+  if (!v.empty()) CU(cudaMemcpy(d, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice));
+  return d;
+}
+
+void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* col_idx, const float* X, const int* y,
+                 const unsigned char* train_mask, int n_layers, const int* widths, int n_comm, const int* community) {
+  const gcn_admm_params& p = h->p;
+  h->L = n_layers;
+  h->n = n;
+  h->M = n_comm;
+  h->C.assign(widths, widths + n_layers + 1);
+  h->ld.resize(n_layers + 1);
+  for (int l = 0; l <= n_layers; ++l) {
+    if (h->C[l] < 1) throw Fail{GCN_ADMM_ERR_WIDTHS, "a layer width is smaller than 1"};
+    h->ld[l] = ldpad(h->C[l]);
+    h->max_ld = std::max(h->max_ld, h->ld[l]);
+  }
+  if (h->C[n_layers] > 32 * gk::kMaxClassesPerLane)
+    throw Fail{GCN_ADMM_ERR_WIDTHS, "more than 128 classes are not supported"};
+  for (int l = 2; l <= n_layers; ++l)
+    if (h->ld[l] / 4 > 256) throw Fail{GCN_ADMM_ERR_WIDTHS, "layer widths above 1024 are supported for C_0 only"};
+
+  // host copies of the graph-side inputs, then the index tables
+  std::vector<long long> rp = to_host(row_ptr, (size_t)n + 1);
+  if (rp[n] < 0 || rp[0] != 0) throw Fail{GCN_ADMM_ERR_GRAPH, "row_ptr must start at 0 and be ascending"};
+  std::vector<int> ci = to_host(col_idx, (size_t)rp[n]);
+  std::vector<int> comm = to_host(community, (size_t)n);
+  std::vector<int> yy = to_host(y, (size_t)n);
+  std::vector<unsigned char> tm = to_host(train_mask, (size_t)n);
+  std::string msg;
+  const int rc = gcn_admm_host::build_graph_index(n, rp.data(), ci.data(), n_comm, comm.data(), h->gi, msg);
+  if (rc == gcn_admm_host::IDX_BAD_GRAPH) throw Fail{GCN_ADMM_ERR_GRAPH, msg};
+  if (rc == gcn_admm_host::IDX_BAD_COMMUNITY) throw Fail{GCN_ADMM_ERR_COMMUNITY, msg};
+  { std::vector<long long>().swap(rp); std::vector<int>().swap(ci); }
+  const GraphIndex& g = h->gi;
+  std::vector<int> y_new(n);
+  std::vector<unsigned char> t_new(n);
+  h->n_train = 0;
+  for (long long i = 0; i < n; ++i) {
+    y_new[i] = yy[g.perm[i]];
+    t_new[i] = tm[g.perm[i]] ? 1 : 0;
+    h->n_train += t_new[i];
+    if (t_new[i] && (y_new[i] < 0 || y_new[i] >= h->C[n_layers]))
+      throw Fail{GCN_ADMM_ERR_WIDTHS, "a training label lies outside 0..C_L-1"};
+    if (y_new[i] < 0 || y_new[i] >= h->C[n_layers]) y_new[i] = 0;
+  }
+  // all host-side validation is done; from here on a CUDA device is required
+  int dev_count = 0;
+  CU(cudaGetDeviceCount(&dev_count));
+  if (p.device < 0 || p.device >= dev_count) throw Fail{GCN_ADMM_ERR_CUDA, "no such CUDA device"};
+  CU(cudaSetDevice(p.device));
+  h->stream = static_cast<cudaStream_t>(p.stream);
+  h->d_row_ptr = upload(h, g.row_ptr);
+  h->d_col = upload(h, g.col);
+  h->d_row_comm = upload(h, g.row_comm);
+  h->d_perm = upload(h, g.perm);
+  h->d_seg_row_ptr = upload(h, g.seg_row_ptr);
+  h->d_seg_comm = upload(h, g.seg_comm);
+  h->d_seg_begin = upload(h, g.seg_begin);
+  h->d_dinv = upload(h, g.dinv);
+  h->d_y = upload(h, y_new);
+  h->d_train = upload(h, t_new);
+
+  const int L = n_layers;
+  const size_t rows = (size_t)n;
+  h->W.assign(L + 1, nullptr); h->Wt.assign(L + 1, nullptr); h->Z.assign(L + 1, nullptr);
+  h->P.assign(L + 1, nullptr); h->H.assign(L + 1, nullptr);
+  size_t grad_elems = 1;
+  h->part_elems = 1;
+  for (int l = 1; l <= L; ++l) {
+    h->W[l] = h->alloc<float>((size_t)h->C[l - 1] * h->ld[l]);
+    h->Wt[l] = h->alloc<float>((size_t)h->C[l] * h->ld[l - 1]);
+    h->Z[l] = h->alloc<float>(rows * h->ld[l]);
+    h->P[l] = h->alloc<float>(rows * h->ld[l - 1]);
+    h->H[l] = h->alloc<float>(rows * h->ld[l]);
+    const size_t ge = (size_t)h->C[l - 1] * h->ld[l];
+    grad_elems = std::max(grad_elems, ge);
+    h->part_elems = std::max(h->part_elems, ge * 4 * kSmCount);
+  }
+  h->part_elems = std::min<size_t>(h->part_elems, (size_t)64 << 20);   // at most 256 MB of partial sums
+  h->part_elems = std::max(h->part_elems, grad_elems);
+  h->U = h->alloc<float>(rows * h->ld[L]);
+  h->B0 = h->alloc<float>(rows * h->max_ld);
+  h->B1 = h->alloc<float>(rows * h->max_ld);
+  h->B2 = h->alloc<float>(rows * h->max_ld);
+  h->grad = h->alloc<float>(grad_elems);
+  h->part = h->alloc<float>(h->part_elems);
+  h->ctl_w = h->alloc<SearchCtl>(L + 1);
+  h->ctl_z = h->alloc<SearchCtl>((size_t)(L + 1) * n_comm);
+  h->sums_w = h->alloc<double>(2);
+  h->sums_z = h->alloc<double>((size_t)3 * n_comm);
+  h->acc_w = h->alloc<double>(gk::kCand);
+  h->acc_z = h->alloc<double>((size_t)gk::kCand * n_comm);
+  h->obj = h->alloc<double>(8);
+  h->n_active = h->alloc<int>(1);
+  h->status = h->alloc<int>(1);
+  h->log_trial_w = h->alloc<int>((size_t)kLogPasses * L);
+  h->log_q_w = h->alloc<double>((size_t)kLogPasses * L);
+  h->log_trial_z = h->alloc<int>((size_t)kLogPasses * std::max(L - 1, 0) * n_comm);
+  h->log_q_z = h->alloc<double>((size_t)kLogPasses * std::max(L - 1, 0) * n_comm);
+  CU(cudaMemset(h->status, 0, sizeof(int)));
+  CU(cudaMemset(h->n_active, 0, sizeof(int)));
+  CU(cudaMemset(h->U, 0, rows * h->ld[L] * sizeof(float)));
+
+  {
+    std::vector<SearchCtl> cw(L + 1), cz((size_t)(L + 1) * n_comm);
+    std::memset(cw.data(), 0, cw.size() * sizeof(SearchCtl));
+    std::memset(cz.data(), 0, cz.size() * sizeof(SearchCtl));
+    for (auto& c : cw) { c.t_prev = p.tau0; c.done = 1; c.trial = -3; }
+    for (auto& c : cz) { c.t_prev = p.theta0; c.done = 1; c.trial = -3; }
+    CU(cudaMemcpy(h->ctl_w, cw.data(), cw.size() * sizeof(SearchCtl), cudaMemcpyHostToDevice));
+    CU(cudaMemcpy(h->ctl_z, cz.data(), cz.size() * sizeof(SearchCtl), cudaMemcpyHostToDevice));
+  }
+
+  // Z_0 in community order, then P_1 = A~ Z_0 (Z_0 never changes, so neither does P_1)
+  {
+    float* dense = nullptr;
+    const bool on_device = is_device_pointer(X);
+    if (!on_device) {
+      dense = dalloc<float>(rows * h->C[0]);
+      cudaError_t e = cudaMemcpy(dense, X, rows * h->C[0] * sizeof(float), cudaMemcpyHostToDevice);
+      if (e != cudaSuccess) { cudaFree(dense); throw Fail{GCN_ADMM_ERR_CUDA, cudaGetErrorString(e)}; }
+    }
+    float* x_pad = nullptr;
+    try {
+      x_pad = dalloc<float>(rows * h->ld[0]);
+      gk::k_permute_rows<<<h->grid_for(n * h->ld[0]), 256, 0, h->stream>>>(on_device ? X : dense, x_pad, h->d_perm, n,
+                                                                           h->C[0], h->ld[0], 1);
+      CU(cudaGetLastError());
+      h->spmm(x_pad, h->P[1], h->ld[0]);
+      CU(cudaStreamSynchronize(h->stream));
+    } catch (...) {
+      if (dense) cudaFree(dense);
+      if (x_pad) cudaFree(x_pad);
+      throw;
+    }
+    if (dense) cudaFree(dense);
+    cudaFree(x_pad);
+  }
+
+  for (int l = 1; l <= L; ++l) h->upload_weight(l, p.w_init[l - 1]);
+  // forward pass of Problem 1 with the same kernels that later recompute H_l, so that the
+  // initial residuals are exactly zero
+  for (int l = 1; l <= L; ++l) {
+    if (l >= 2) h->spmm(h->Z[l - 1], h->P[l], h->ld[l - 1]);
+    h->gemm_nn(h->P[l], h->ld[l - 1], h->W[l], h->ld[l], h->H[l], h->ld[l], n, h->C[l], h->C[l - 1]);
+    const size_t bytes = rows * h->ld[l] * sizeof(float);
+    CU(cudaMemcpyAsync(h->Z[l], h->H[l], bytes, cudaMemcpyDeviceToDevice, h->stream));
+    if (l < L) {
+      const long long n4 = n * h->ld[l] / 4;
+      gk::k_relu_inplace<<<h->grid_for(n4), 256, 0, h->stream>>>((float4*)h->Z[l], n4);
+      CU(cudaGetLastError());
+    }
+  }
+  h->fresh = true;
+  CU(cudaStreamSynchronize(h->stream));
+}
+
+}  // namespace
+
+extern "C" {
+
+void gcn_admm_default_params(gcn_admm_params* p) {
+  if (!p) return;
+  std::memset(p, 0, sizeof(*p));
+  p->nu = 1e-3f; p->rho = 1e-3f;
+  p->tau0 = 1.f; p->theta0 = 1.f;
+  p->bt_growth = 2.f; p->bt_shrink = 0.5f;
+  p->bt_max_trials = 40;
+  p->fista_iters = 30;
+  p->loss_scale = 1.f;
+  p->dual_mode = 0;
+  p->w_init = nullptr;
+  p->device = 0;
+  p->stream = nullptr;
+}
+
+int gcn_admm_create(gcn_admm** out, long long n, const long long* row_ptr, const int* col_idx, const float* X,
+                    const int* y, const unsigned char* train_mask, int n_layers, const int* widths,
+                    const gcn_admm_params* p, int n_comm, const int* community) {
+  if (out) *out = nullptr;
+  if (!out || !row_ptr || !X || !y || !train_mask || !widths || !p || !community || !col_idx) {
+    g_create_error = "NULL argument";
+    return GCN_ADMM_ERR_ARG;
+  }
+  if (n < 1 || n > 2147483647LL / 2 || n_comm < 1) { g_create_error = "n and n_comm must be positive"; return GCN_ADMM_ERR_ARG; }
+  if (n_layers < 1 || n_layers > 64) { g_create_error = "n_layers must be 1..64"; return GCN_ADMM_ERR_WIDTHS; }
+  if (!p->w_init) { g_create_error = "w_init is required"; return GCN_ADMM_ERR_ARG; }
+  for (int l = 0; l < n_layers; ++l)
+    if (!p->w_init[l]) { g_create_error = "w_init holds a NULL pointer"; return GCN_ADMM_ERR_ARG; }
+  if (!(p->nu > 0.f) || !(p->rho > 0.f) || !(p->bt_growth > 1.f) || !(p->bt_shrink > 0.f) || p->bt_max_trials < 1 ||
+      p->bt_max_trials > 64 || p->fista_iters < 0 || !(p->tau0 > 0.f) || !(p->theta0 > 0.f) || !(p->loss_scale > 0.f)) {
+    g_create_error = "a parameter is out of range";
+    return GCN_ADMM_ERR_ARG;
+  }
+  gcn_admm* h = new (std::nothrow) gcn_admm();
+  if (!h) { g_create_error = "host allocation failed"; return GCN_ADMM_ERR_ALLOC; }
+  h->p = *p;
+  int code = GCN_ADMM_OK;
+  try {
+    create_impl(h, n, row_ptr, col_idx, X, y, train_mask, n_layers, widths, n_comm, community);
+  } catch (const Fail& f) {
+    code = f.code; g_create_error = f.msg;
+  } catch (const std::bad_alloc&) {
+    code = GCN_ADMM_ERR_ALLOC; g_create_error = "host allocation failed";
+  } catch (...) {
+    code = GCN_ADMM_ERR_CUDA; g_create_error = "unexpected failure";
+  }
+  if (code != GCN_ADMM_OK) {
+    gcn_admm_destroy(h);
+    return code;
+  }
+  h->p.w_init = nullptr;   // the caller's pointers are not kept
+  *out = h;
+  return GCN_ADMM_OK;
+}
+
+void gcn_admm_destroy(gcn_admm* h) {
+  if (!h) return;
+  if (cudaSetDevice(h->p.device) == cudaSuccess) {
+    cudaStreamSynchronize(h->stream);
+    for (void* q : h->owned) cudaFree(q);
+  }
+  cudaGetLastError();
+  delete h;
+}
+
+const char* gcn_admm_last_error(const gcn_admm* h) { return h ? h->err.c_str() : g_create_error.c_str(); }
+
+int gcn_admm_step(gcn_admm* h, int n_iters) {
+  return guarded(h, [&] {
+    if (n_iters < 0) throw Fail{GCN_ADMM_ERR_ARG, "n_iters must be >= 0"};
+    h->log_count = 0;
+    for (int k = 0; k < n_iters; ++k) h->iterate();
+  });
+}
+
+int gcn_admm_step_block(gcn_admm* h, int phase, int layer) {
+  return guarded(h, [&] {
+    const int L = h->L;
+    if (phase == GCN_ADMM_PHASE_W || phase == GCN_ADMM_PHASE_Z)
+      if (layer < 1 || layer > L) throw Fail{GCN_ADMM_ERR_ARG, "layer out of range"};
+    if (!h->fresh) h->refresh();
+    h->log_count = 0;
+    h->begin_log_pass();
+    if (phase == GCN_ADMM_PHASE_W) {
+      h->update_W(layer);
+    } else if (phase == GCN_ADMM_PHASE_Z) {
+      if (layer < L) h->update_Z_hidden(layer);
+      else h->update_output(false, true);
+      h->fresh = false;
+    } else if (phase == GCN_ADMM_PHASE_U) {
+      h->dual_from_stored();
+    } else {
+      throw Fail{GCN_ADMM_ERR_ARG, "unknown phase"};
+    }
+    ++h->log_count;
+  });
+}
+
+int gcn_admm_objective(gcn_admm* h, double out[6]) {
+  return guarded(h, [&] {
+    if (!out) throw Fail{GCN_ADMM_ERR_ARG, "NULL output"};
+    if (!h->fresh) h->refresh();
+    const int L = h->L;
+    cudaStream_t s = h->stream;
+    CU(cudaMemsetAsync(h->obj, 0, 8 * sizeof(double), s));
+    for (int l = 1; l < L; ++l) {
+      const long long n4 = h->n * h->ld[l] / 4;
+      gk::k_sum_hidden_penalty<<<h->grid_for(n4), 256, 0, s>>>((const float4*)h->Z[l], (const float4*)h->H[l], n4, h->obj + 2);
+    }
+    const long long n4 = h->n * h->ld[L] / 4;
+    gk::k_sum_constraint<<<h->grid_for(n4), 256, 0, s>>>((const float4*)h->Z[L], (const float4*)h->H[L],
+                                                        (const float4*)h->U, n4, h->obj + 3);
+    const int warps = 8;
+    gk::k_row_loss_argmax<<<(unsigned)cdiv(h->n, warps), warps * 32, 0, s>>>(h->Z[L], nullptr, h->ld[L], h->C[L], (int)h->n,
+                                                                             h->d_y, h->d_train, nullptr, h->obj);
+    CU(cudaGetLastError());
+    h->forward_logits();
+    gk::k_row_loss_argmax<<<(unsigned)cdiv(h->n, warps), warps * 32, 0, s>>>(nullptr, h->B0, h->ld[L], h->C[L], (int)h->n,
+                                                                             h->d_y, h->d_train, nullptr, h->obj);
+    CU(cudaGetLastError());
+    double v[8];
+    CU(cudaMemcpyAsync(v, h->obj, 8 * sizeof(double), cudaMemcpyDeviceToHost, s));
+    CU(cudaStreamSynchronize(s));
+    const double R = h->p.loss_scale * v[0];
+    const double pen = 0.5 * h->p.nu * v[2];
+    const double ur = v[3];
+    const double rr = 0.5 * h->p.rho * v[4];
+    out[0] = R + pen + ur + rr;
+    out[1] = R; out[2] = pen; out[3] = ur; out[4] = rr;
+    out[5] = h->n_train > 0 ? v[1] / h->n_train : 0.0;
+    h->check_status();
+  });
+}
+
+int gcn_admm_weights(gcn_admm* h, int layer, float* out) {
+  return gcn_admm_get_state(h, GCN_ADMM_ST_W, layer, out);
+}
+
+int gcn_admm_predict(gcn_admm* h, float* logits, int* labels) {
+  return guarded(h, [&] {
+    const int L = h->L;
+    h->forward_logits();
+    if (labels) {
+      const int warps = 8;
+      int* d_lab = reinterpret_cast<int*>(h->B1);
+      CU(cudaMemsetAsync(h->obj, 0, 8 * sizeof(double), h->stream));
+      gk::k_row_loss_argmax<<<(unsigned)cdiv(h->n, warps), warps * 32, 0, h->stream>>>(
+          nullptr, h->B0, h->ld[L], h->C[L], (int)h->n, h->d_y, h->d_train, d_lab, h->obj);
+      CU(cudaGetLastError());
+      std::vector<int> lab(h->n);
+      CU(cudaMemcpyAsync(lab.data(), d_lab, sizeof(int) * h->n, cudaMemcpyDeviceToHost, h->stream));
+      CU(cudaStreamSynchronize(h->stream));
+      for (long long i = 0; i < h->n; ++i) labels[h->gi.perm[i]] = lab[i];
+    }
+    if (logits) h->rows_to_host(h->B0, h->C[L], logits);
+    CU(cudaStreamSynchronize(h->stream));
+  });
+}
+
+int gcn_admm_propagate(gcn_admm* h, const float* x, int width, float* out) {
+  return guarded(h, [&] {
+    if (!x || !out || width < 1) throw Fail{GCN_ADMM_ERR_ARG, "bad argument"};
+    const int ldw = ldpad(width);
+    const size_t rows = (size_t)h->n;
+    const bool dev_in = is_device_pointer(x), dev_out = is_device_pointer(out);
+    if (dev_in != dev_out) throw Fail{GCN_ADMM_ERR_ARG, "x and out must both be host or both be device pointers"};
+    float *dense = nullptr, *a = nullptr, *b = nullptr;
+    try {
+      dense = dalloc<float>(rows * width);
+      a = dalloc<float>(rows * ldw);
+      b = dalloc<float>(rows * ldw);
+      CU(cudaMemcpyAsync(dense, x, rows * width * sizeof(float), dev_in ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice,
+                         h->stream));
+      gk::k_permute_rows<<<h->grid_for(h->n * ldw), 256, 0, h->stream>>>(dense, a, h->d_perm, h->n, width, ldw, 1);
+      CU(cudaGetLastError());
+      h->spmm(a, b, ldw);
+      gk::k_permute_rows<<<h->grid_for(h->n * ldw), 256, 0, h->stream>>>(b, dense, h->d_perm, h->n, width, ldw, 0);
+      CU(cudaGetLastError());
+      CU(cudaMemcpyAsync(out, dense, rows * width * sizeof(float), dev_out ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost,
+                         h->stream));
+      CU(cudaStreamSynchronize(h->stream));
+    } catch (...) {
+      cudaFree(dense); cudaFree(a); cudaFree(b);
+      throw;
+    }
+    cudaFree(dense); cudaFree(a); cudaFree(b);
+  });
+}
+
+int gcn_admm_index(gcn_admm* h, int which, int comm, const int** data, long long* len) {
+  return guarded(h, [&] {
+    if (!data || !len || which < 0 || which > GCN_ADMM_IX_SEG_BEGIN) throw Fail{GCN_ADMM_ERR_ARG, "bad selector"};
+    const GraphIndex& g = h->gi;
+    const std::vector<int>* v = nullptr;
+    switch (which) {
+      case GCN_ADMM_IX_PERM: v = &g.perm; break;
+      case GCN_ADMM_IX_INV_PERM: v = &g.inv; break;
+      case GCN_ADMM_IX_COMM_PTR: v = &g.comm_ptr; break;
+      case GCN_ADMM_IX_CSR_ROW_PTR: v = &g.row_ptr; break;
+      case GCN_ADMM_IX_CSR_COL: v = &g.col; break;
+      case GCN_ADMM_IX_SEG_ROW_PTR: v = &g.seg_row_ptr; break;
+      case GCN_ADMM_IX_SEG_COMM: v = &g.seg_comm; break;
+      case GCN_ADMM_IX_SEG_BEGIN: v = &g.seg_begin; break;
+      default: {
+        if (comm < 0 || comm >= h->M) throw Fail{GCN_ADMM_ERR_ARG, "community out of range"};
+        std::vector<int>& c = h->ix_cache[which];
+        if (which == GCN_ADMM_IX_NBR) c = gcn_admm_host::nbr_of(g, comm);
+        else if (which == GCN_ADMM_IX_HALO1) c = gcn_admm_host::halo1_of(g, comm);
+        else c = gcn_admm_host::halo2_of(g, comm);
+        v = &c;
+      }
+    }
+    *data = v->data();
+    *len = (long long)v->size();
+  });
+}
+
+int gcn_admm_get_state(gcn_admm* h, int which, int layer, void* out) {
+  return guarded(h, [&] {
+    if (!out) throw Fail{GCN_ADMM_ERR_ARG, "NULL output"};
+    const int L = h->L;
+    auto need_layer = [&](int lo, int hi) {
+      if (layer < lo || layer > hi) throw Fail{GCN_ADMM_ERR_ARG, "layer out of range"};
+    };
+    if (which == GCN_ADMM_ST_W) {
+      need_layer(1, L);
+      const int r = h->C[layer - 1], c = h->C[layer], ldw = h->ld[layer];
+      std::vector<float> w((size_t)r * ldw);
+      CU(cudaMemcpyAsync(w.data(), h->W[layer], w.size() * sizeof(float), cudaMemcpyDeviceToHost, h->stream));
+      CU(cudaStreamSynchronize(h->stream));
+      float* o = static_cast<float*>(out);
+      for (int i = 0; i < r; ++i) std::memcpy(o + (size_t)i * c, w.data() + (size_t)i * ldw, c * sizeof(float));
+    } else if (which == GCN_ADMM_ST_Z) {
+      need_layer(1, L);
+      h->rows_to_host(h->Z[layer], h->C[layer], static_cast<float*>(out));
+    } else if (which == GCN_ADMM_ST_U) {
+      h->rows_to_host(h->U, h->C[L], static_cast<float*>(out));
+    } else if (which == GCN_ADMM_ST_TAU) {
+      need_layer(1, L);
+      SearchCtl c;
+      CU(cudaMemcpyAsync(&c, h->ctl_w + layer, sizeof(c), cudaMemcpyDeviceToHost, h->stream));
+      CU(cudaStreamSynchronize(h->stream));
+      *static_cast<double*>(out) = c.t_prev;
+    } else if (which == GCN_ADMM_ST_THETA) {
+      need_layer(1, L - 1);
+      std::vector<SearchCtl> c(h->M);
+      CU(cudaMemcpyAsync(c.data(), h->ctl_z + (size_t)layer * h->M, c.size() * sizeof(SearchCtl), cudaMemcpyDeviceToHost,
+                         h->stream));
+      CU(cudaStreamSynchronize(h->stream));
+      for (int m = 0; m < h->M; ++m) static_cast<double*>(out)[m] = c[m].t_prev;
+    } else {
+      throw Fail{GCN_ADMM_ERR_ARG, "unknown state selector"};
+    }
+  });
+}
+
+int gcn_admm_set_state(gcn_admm* h, int which, int layer, const void* in) {
+  return guarded(h, [&] {
+    if (!in) throw Fail{GCN_ADMM_ERR_ARG, "NULL input"};
+    const int L = h->L;
+    auto need_layer = [&](int lo, int hi) {
+      if (layer < lo || layer > hi) throw Fail{GCN_ADMM_ERR_ARG, "layer out of range"};
+    };
+    if (which == GCN_ADMM_ST_W) {
+      need_layer(1, L);
+      h->upload_weight(layer, static_cast<const float*>(in));
+      h->fresh = false;
+    } else if (which == GCN_ADMM_ST_Z) {
+      need_layer(1, L);
+      h->rows_from_host(static_cast<const float*>(in), h->C[layer], h->Z[layer]);
+      h->fresh = false;
+    } else if (which == GCN_ADMM_ST_U) {
+      h->rows_from_host(static_cast<const float*>(in), h->C[L], h->U);
+    } else if (which == GCN_ADMM_ST_TAU) {
+      need_layer(1, L);
+      const double t = *static_cast<const double*>(in);
+      if (!(t > 0.0)) throw Fail{GCN_ADMM_ERR_ARG, "tau must be positive"};
+      CU(cudaMemcpyAsync(&h->ctl_w[layer].t_prev, &t, sizeof(double), cudaMemcpyHostToDevice, h->stream));
+      CU(cudaStreamSynchronize(h->stream));
+    } else if (which == GCN_ADMM_ST_THETA) {
+      need_layer(1, L - 1);
+      const double* t = static_cast<const double*>(in);
+      for (int m = 0; m < h->M; ++m) {
+        if (!(t[m] > 0.0)) throw Fail{GCN_ADMM_ERR_ARG, "theta must be positive"};
+        CU(cudaMemcpyAsync(&h->ctl_z[(size_t)layer * h->M + m].t_prev, t + m, sizeof(double), cudaMemcpyHostToDevice,
+                           h->stream));
+      }
+      CU(cudaStreamSynchronize(h->stream));
+    } else {
+      throw Fail{GCN_ADMM_ERR_ARG, "unknown state selector"};
+    }
+  });
+}
+
+int gcn_admm_decisions(gcn_admm* h, int max_passes, int* n_passes, int* trial_w, double* q_w, int* trial_z,
+                       double* q_z) {
+  return guarded(h, [&] {
+    if (!n_passes || max_passes < 0) throw Fail{GCN_ADMM_ERR_ARG, "bad argument"};
+    const int L = h->L;
+    const long long have = std::min<long long>(h->log_count, kLogPasses);
+    const int take = (int)std::min<long long>(have, max_passes);
+    const size_t zper = (size_t)std::max(L - 1, 0) * h->M;
+    CU(cudaStreamSynchronize(h->stream));
+    for (int k = 0; k < take; ++k) {
+      const long long pass = h->log_count - have + k;   // oldest kept pass first
+      const long long slot = pass % kLogPasses;
+      if (trial_w) CU(cudaMemcpy(trial_w + (size_t)k * L, h->log_trial_w + slot * L, L * sizeof(int), cudaMemcpyDeviceToHost));
+      if (q_w) CU(cudaMemcpy(q_w + (size_t)k * L, h->log_q_w + slot * L, L * sizeof(double), cudaMemcpyDeviceToHost));
+      if (zper && trial_z)
+        CU(cudaMemcpy(trial_z + k * zper, h->log_trial_z + slot * zper, zper * sizeof(int), cudaMemcpyDeviceToHost));
+      if (zper && q_z) CU(cudaMemcpy(q_z + k * zper, h->log_q_z + slot * zper, zper * sizeof(double), cudaMemcpyDeviceToHost));
+    }
+    *n_passes = take;
+    h->check_status();
+  });
+}
+
+}  // extern "C"

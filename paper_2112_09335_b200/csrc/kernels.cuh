@@ -1,0 +1,1039 @@
+// Device kernels of the community-based ADMM GCN trainer (sm_100a).
+//
+// Layout: every N x C matrix is row-major fp32 with a leading dimension padded to a multiple
+// of 4 floats, rows in community order, so that a row starts on a 16-byte boundary and can be
+// moved with 128-bit loads.  Padding columns are kept at zero.
+// Scalars that decide a step size (descent sums, squared norms) are accumulated in fp64.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace gk {
+
+constexpr int kCand = 4;        // step-size candidates scored per pass
+constexpr int kMaxClassesPerLane = 4;   // C_L <= 128
+
+// Control block of one quadratic-approximation search (one per W_l, one per Z_{l,m}).
+struct SearchCtl {
+  double t_prev;   // accepted parameter of the previous search (tau_l or theta_{l,m})
+  double t_base;   // first candidate of the current pass
+  double gg;       // ||grad||^2
+  double xx;       // ||x||^2 of the block
+  double q;        // (f(x) - f(x+)) / (gg / 2t) at the accepted trial
+  float inv_step;  // 1/t of the accepted trial, 0 when the block stays
+  int done;        // search finished (accepted, skipped or exhausted)
+  int trial;       // accepted trial index, -1 skipped, -2 exhausted
+  int pass;        // passes already scored
+  float inv_cand[kCand];  // 1/t of the candidates of the current pass
+};
+
+__device__ __forceinline__ float relu(float x) { return x > 0.f ? x : 0.f; }
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Sum of `v` over the block; valid in thread 0.  `sh` holds >= 32 doubles.
+__device__ __forceinline__ double block_sum(double v, double* sh) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  v = warp_sum(v);
+  __syncthreads();
+  if (lane == 0) sh[w] = v;
+  __syncthreads();
+  const int nw = (blockDim.x + 31) >> 5;
+  v = (threadIdx.x < nw) ? sh[threadIdx.x] : 0.0;
+  if (w == 0) v = warp_sum(v);
+  return v;
+}
+
+// ------------------------------------------------------------------------------------------
+// Propagation  out = A~ x,  A~_ij = dinv_i dinv_j on the pattern of A + I (Problem 1).
+// G lanes share one row; each lane owns the float4 columns lane, lane+G, .. of a block of
+// G*V float4 columns; wider rows loop over column blocks.
+// ------------------------------------------------------------------------------------------
+template <int G, int V>
+__global__ void __launch_bounds__(256)
+k_spmm(const int* __restrict__ row_ptr, const int* __restrict__ col, const float* __restrict__ dinv,
+       const float4* __restrict__ x, float4* __restrict__ out, int n, int ld4) {
+  const int lane = threadIdx.x & 31;
+  const int gl = lane & (G - 1);
+  const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << (lane & ~(G - 1)));
+  const long long row = ((long long)blockIdx.x * blockDim.x + threadIdx.x) / G;
+  if (row >= n) return;
+  const int rs = row_ptr[row], re = row_ptr[row + 1];
+  const float di = dinv[row];
+  for (int cb = 0; cb < ld4; cb += G * V) {
+    float4 acc[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int base = rs; base < re; base += G) {
+      const int idx = base + gl;
+      int c = 0;
+      float w = 0.f;
+      if (idx < re) { c = col[idx]; w = dinv[c]; }
+      const int cnt = min(G, re - base);
+      for (int t = 0; t < cnt; t += 4) {
+        int cj[4];
+        float wj[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {   // lanes past the row's end hold (column 0, weight 0)
+          cj[u] = __shfl_sync(gmask, c, (t + u) & (G - 1), G);
+          wj[u] = __shfl_sync(gmask, w, (t + u) & (G - 1), G);
+          if (t + u >= G) wj[u] = 0.f;
+        }
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+          const int f = cb + gl + G * v;
+          if (f < ld4) {
+            float4 xv[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) xv[u] = __ldg(x + (long long)cj[u] * ld4 + f);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              acc[v].x = fmaf(wj[u], xv[u].x, acc[v].x);
+              acc[v].y = fmaf(wj[u], xv[u].y, acc[v].y);
+              acc[v].z = fmaf(wj[u], xv[u].z, acc[v].z);
+              acc[v].w = fmaf(wj[u], xv[u].w, acc[v].w);
+            }
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+      const int f = cb + gl + G * v;
+      if (f < ld4)
+        out[row * ld4 + f] = make_float4(di * acc[v].x, di * acc[v].y, di * acc[v].z, di * acc[v].w);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Dense products.
+//   k_gemm_nn : C[M x N] = A[M x K] B[K x N]          (H = P W, D = P grad, G = S W^T, T = G W)
+//   k_gemm_tn : part[s][Ka x Nb] = sum over the rows of split s of A[r,:]^T B[r,:]   (grad = P^T R)
+// fp32 FFMA register tiles; `skip`, when given, points at a flag that cancels the launch.
+// ------------------------------------------------------------------------------------------
+template <int BM, int BN, int BK, int TM, int TN>
+__global__ void __launch_bounds__((BM / TM) * (BN / TN))
+k_gemm_nn(const float* __restrict__ A, int lda, const float* __restrict__ B, int ldb,
+          float* __restrict__ C, int ldc, int M, int N, int K, const int* __restrict__ skip) {
+  constexpr int NT = (BM / TM) * (BN / TN);
+  constexpr int TX = BN / TN;
+  constexpr int A_F4 = BM * BK / 4, B_F4 = BK * BN / 4;
+  constexpr int A_PER = (A_F4 + NT - 1) / NT, B_PER = (B_F4 + NT - 1) / NT;
+  constexpr int PAD = 4;
+  static_assert(TN == 4 || TN == 8, "TN");
+  static_assert(TM == 4 || TM == 8, "TM");
+  if (skip != nullptr && *skip) return;
+  __shared__ __align__(16) float As[2][BK][BM + PAD];
+  __shared__ __align__(16) float Bs[2][BK][BN];
+  const int tid = threadIdx.x;
+  const int tx = tid % TX, ty = tid / TX;
+  const long long row0 = (long long)blockIdx.x * BM;
+  const int col0 = blockIdx.y * BN;
+
+  float4 ra[A_PER], rb[B_PER];
+  auto load_tiles = [&](int k0) {
+#pragma unroll
+    for (int i = 0; i < A_PER; ++i) {
+      const int f = tid + i * NT;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (f < A_F4) {
+        const int r = f / (BK / 4), kq = (f % (BK / 4)) * 4;
+        const long long gr = row0 + r;
+        const int gk = k0 + kq;
+        if (gr < M && gk < K) {
+          v = *reinterpret_cast<const float4*>(A + gr * lda + gk);   // lda % 4 == 0, gk % 4 == 0
+          if (gk + 1 >= K) v.y = 0.f;
+          if (gk + 2 >= K) v.z = 0.f;
+          if (gk + 3 >= K) v.w = 0.f;
+        }
+      }
+      ra[i] = v;
+    }
+#pragma unroll
+    for (int i = 0; i < B_PER; ++i) {
+      const int f = tid + i * NT;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (f < B_F4) {
+        const int kr = f / (BN / 4), c = (f % (BN / 4)) * 4;
+        const int gk = k0 + kr, gc = col0 + c;
+        if (gk < K && gc < N) {
+          v = *reinterpret_cast<const float4*>(B + (long long)gk * ldb + gc);  // ldb % 4 == 0
+          if (gc + 1 >= N) v.y = 0.f;
+          if (gc + 2 >= N) v.z = 0.f;
+          if (gc + 3 >= N) v.w = 0.f;
+        }
+      }
+      rb[i] = v;
+    }
+  };
+  auto store_tiles = [&](int buf) {
+#pragma unroll
+    for (int i = 0; i < A_PER; ++i) {
+      const int f = tid + i * NT;
+      if (f < A_F4) {
+        const int r = f / (BK / 4), kq = (f % (BK / 4)) * 4;
+        As[buf][kq + 0][r] = ra[i].x;
+        As[buf][kq + 1][r] = ra[i].y;
+        As[buf][kq + 2][r] = ra[i].z;
+        As[buf][kq + 3][r] = ra[i].w;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < B_PER; ++i) {
+      const int f = tid + i * NT;
+      if (f < B_F4) {
+        const int kr = f / (BN / 4), c = (f % (BN / 4)) * 4;
+        *reinterpret_cast<float4*>(&Bs[buf][kr][c]) = rb[i];
+      }
+    }
+  };
+
+  float acc[TM][TN];
+#pragma unroll
+  for (int i = 0; i < TM; ++i)
+#pragma unroll
+    for (int j = 0; j < TN; ++j) acc[i][j] = 0.f;
+
+  load_tiles(0);
+  store_tiles(0);
+  __syncthreads();
+  int buf = 0;
+  for (int k0 = 0; k0 < K; k0 += BK) {
+    const bool more = (k0 + BK) < K;
+    if (more) load_tiles(k0 + BK);
+#pragma unroll
+    for (int k = 0; k < BK; ++k) {
+      float a[TM], b[TN];
+#pragma unroll
+      for (int i = 0; i < TM; i += 4) {
+        const float4 v = *reinterpret_cast<const float4*>(&As[buf][k][ty * TM + i]);
+        a[i] = v.x; a[i + 1] = v.y; a[i + 2] = v.z; a[i + 3] = v.w;
+      }
+      {
+        const float4 v = *reinterpret_cast<const float4*>(&Bs[buf][k][tx * 4]);
+        b[0] = v.x; b[1] = v.y; b[2] = v.z; b[3] = v.w;
+      }
+      if constexpr (TN == 8) {
+        const float4 v = *reinterpret_cast<const float4*>(&Bs[buf][k][BN / 2 + tx * 4]);
+        b[TN - 4] = v.x; b[TN - 3] = v.y; b[TN - 2] = v.z; b[TN - 1] = v.w;
+      }
+#pragma unroll
+      for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    if (more) {
+      store_tiles(buf ^ 1);
+      __syncthreads();
+      buf ^= 1;
+    }
+  }
+  // columns N..ldc-1 (padding) receive the zeros accumulated from the masked B columns
+#pragma unroll
+  for (int i = 0; i < TM; ++i) {
+    const long long gr = row0 + ty * TM + i;
+    if (gr >= M) continue;
+#pragma unroll
+    for (int h = 0; h < TN / 4; ++h) {
+      const int gc = col0 + (h == 0 ? tx * 4 : BN / 2 + tx * 4);
+      if (gc < ldc)
+        *reinterpret_cast<float4*>(C + gr * ldc + gc) =
+            make_float4(acc[i][h * 4], acc[i][h * 4 + 1], acc[i][h * 4 + 2], acc[i][h * 4 + 3]);
+    }
+  }
+}
+
+// part[(split * Ka + ka) * ldp + nb].  A: rows x Ka (lda), B: rows x Nb (ldb).
+// Split s owns rows [s * rows_per_split, min(rows, (s+1) * rows_per_split)).
+template <int BM, int BN, int BK, int TM, int TN>
+__global__ void __launch_bounds__((BM / TM) * (BN / TN))
+k_gemm_tn(const float* __restrict__ A, int lda, const float* __restrict__ B, int ldb,
+          float* __restrict__ part, int ldp, long long rows, long long rows_per_split, int Ka, int Nb) {
+  constexpr int NT = (BM / TM) * (BN / TN);
+  constexpr int TX = BN / TN;
+  constexpr int A_F4 = BK * BM / 4, B_F4 = BK * BN / 4;
+  constexpr int A_PER = (A_F4 + NT - 1) / NT, B_PER = (B_F4 + NT - 1) / NT;
+  static_assert(TM == 4 || TM == 8, "TM");
+  static_assert(BN % 4 == 0, "BN");
+  __shared__ __align__(16) float As[2][BK][BM];
+  __shared__ __align__(16) float Bs[2][BK][BN];
+  const int tid = threadIdx.x;
+  const int tx = tid % TX, ty = tid / TX;
+  const int a0 = blockIdx.x * BM, b0 = blockIdx.y * BN;
+  const long long r_begin = (long long)blockIdx.z * rows_per_split;
+  const long long r_end = min(rows, r_begin + rows_per_split);
+
+  float4 ra[A_PER], rb[B_PER];
+  auto load_tiles = [&](long long r0) {
+#pragma unroll
+    for (int i = 0; i < A_PER; ++i) {
+      const int f = tid + i * NT;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (f < A_F4) {
+        const int rr = f / (BM / 4), c = (f % (BM / 4)) * 4;
+        const long long gr = r0 + rr;
+        const int gc = a0 + c;
+        if (gr < r_end && gc < Ka) {
+          v = *reinterpret_cast<const float4*>(A + gr * lda + gc);
+          if (gc + 1 >= Ka) v.y = 0.f;
+          if (gc + 2 >= Ka) v.z = 0.f;
+          if (gc + 3 >= Ka) v.w = 0.f;
+        }
+      }
+      ra[i] = v;
+    }
+#pragma unroll
+    for (int i = 0; i < B_PER; ++i) {
+      const int f = tid + i * NT;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (f < B_F4) {
+        const int rr = f / (BN / 4), c = (f % (BN / 4)) * 4;
+        const long long gr = r0 + rr;
+        const int gc = b0 + c;
+        if (gr < r_end && gc < Nb) {
+          v = *reinterpret_cast<const float4*>(B + gr * ldb + gc);
+          if (gc + 1 >= Nb) v.y = 0.f;
+          if (gc + 2 >= Nb) v.z = 0.f;
+          if (gc + 3 >= Nb) v.w = 0.f;
+        }
+      }
+      rb[i] = v;
+    }
+  };
+  auto store_tiles = [&](int buf) {
+#pragma unroll
+    for (int i = 0; i < A_PER; ++i) {
+      const int f = tid + i * NT;
+      if (f < A_F4) *reinterpret_cast<float4*>(&As[buf][f / (BM / 4)][(f % (BM / 4)) * 4]) = ra[i];
+    }
+#pragma unroll
+    for (int i = 0; i < B_PER; ++i) {
+      const int f = tid + i * NT;
+      if (f < B_F4) *reinterpret_cast<float4*>(&Bs[buf][f / (BN / 4)][(f % (BN / 4)) * 4]) = rb[i];
+    }
+  };
+
+  float acc[TM][TN];
+#pragma unroll
+  for (int i = 0; i < TM; ++i)
+#pragma unroll
+    for (int j = 0; j < TN; ++j) acc[i][j] = 0.f;
+
+  if (r_begin < r_end) {
+    load_tiles(r_begin);
+    store_tiles(0);
+    __syncthreads();
+    int buf = 0;
+    for (long long r0 = r_begin; r0 < r_end; r0 += BK) {
+      const bool more = (r0 + BK) < r_end;
+      if (more) load_tiles(r0 + BK);
+#pragma unroll
+      for (int k = 0; k < BK; ++k) {
+        float a[TM], b[TN];
+        {
+          const float4 v = *reinterpret_cast<const float4*>(&As[buf][k][ty * 4]);
+          a[0] = v.x; a[1] = v.y; a[2] = v.z; a[3] = v.w;
+        }
+        if constexpr (TM == 8) {
+          const float4 v = *reinterpret_cast<const float4*>(&As[buf][k][BM / 2 + ty * 4]);
+          a[TM - 4] = v.x; a[TM - 3] = v.y; a[TM - 2] = v.z; a[TM - 1] = v.w;
+        }
+        if constexpr (TN >= 4) {
+          const float4 v = *reinterpret_cast<const float4*>(&Bs[buf][k][tx * 4]);
+          b[0] = v.x; b[1] = v.y; b[2] = v.z; b[3] = v.w;
+          if constexpr (TN == 8) {
+            const float4 w = *reinterpret_cast<const float4*>(&Bs[buf][k][BN / 2 + tx * 4]);
+            b[TN - 4] = w.x; b[TN - 3] = w.y; b[TN - 2] = w.z; b[TN - 1] = w.w;
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < TN; ++j) b[j] = Bs[buf][k][tx * TN + j];
+        }
+#pragma unroll
+        for (int i = 0; i < TM; ++i)
+#pragma unroll
+          for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+      }
+      if (more) {
+        store_tiles(buf ^ 1);
+        __syncthreads();
+        buf ^= 1;
+      }
+    }
+  }
+  float* dst = part + (long long)blockIdx.z * Ka * ldp;
+#pragma unroll
+  for (int i = 0; i < TM; ++i) {
+    const int ga = a0 + ((TM == 8 && i >= 4) ? BM / 2 + ty * 4 + (i - 4) : ty * 4 + i);
+    if (ga >= Ka) continue;
+#pragma unroll
+    for (int j = 0; j < TN; ++j) {
+      int gb;
+      if (TN == 8) gb = b0 + (j >= 4 ? BN / 2 + tx * 4 + (j - 4) : tx * 4 + j);
+      else if (TN == 4) gb = b0 + tx * 4 + j;
+      else gb = b0 + tx * TN + j;
+      if (gb < ldp) dst[(long long)ga * ldp + gb] = acc[i][j];
+    }
+  }
+}
+
+// grad[e] = sum over splits of part[s][e], summed in fp64 in split order (fixed order).
+__global__ void k_reduce_splits(const float* __restrict__ part, float* __restrict__ grad, long long elems,
+                                int splits) {
+  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= elems) return;
+  double s = 0.0;
+  for (int k = 0; k < splits; ++k) s += (double)part[(long long)k * elems + e];
+  grad[e] = (float)s;
+}
+
+// out[0] = sum a^2, out[1] = sum b^2 over `elems` floats (one block, fixed order).
+__global__ void k_two_sumsq(const float* __restrict__ a, const float* __restrict__ b, long long elems,
+                            double* __restrict__ out) {
+  __shared__ double sh[32];
+  double sa = 0.0, sb = 0.0;
+  for (long long e = threadIdx.x; e < elems; e += blockDim.x) {
+    const double x = a[e], y = b[e];
+    sa += x * x;
+    sb += y * y;
+  }
+  sa = block_sum(sa, sh);
+  sb = block_sum(sb, sh);
+  if (threadIdx.x == 0) { out[0] = sa; out[1] = sb; }
+}
+
+// ------------------------------------------------------------------------------------------
+// Residuals with respect to the pre-activation H (derivatives of phi, Section 3):
+//   hidden layer  R = nu (f(H) - Z) * f'(H)
+//   last layer    R = -(U + rho (Z - H))
+// ------------------------------------------------------------------------------------------
+__global__ void k_resid_hidden(const float4* __restrict__ H, const float4* __restrict__ Z,
+                               float4* __restrict__ R, long long n4, float nu) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4;
+       i += (long long)gridDim.x * blockDim.x) {
+    const float4 h = H[i], z = Z[i];
+    float4 r;
+    r.x = h.x > 0.f ? nu * (h.x - z.x) : 0.f;
+    r.y = h.y > 0.f ? nu * (h.y - z.y) : 0.f;
+    r.z = h.z > 0.f ? nu * (h.z - z.z) : 0.f;
+    r.w = h.w > 0.f ? nu * (h.w - z.w) : 0.f;
+    R[i] = r;
+  }
+}
+
+__global__ void k_resid_out(const float4* __restrict__ H, const float4* __restrict__ Z,
+                            const float4* __restrict__ U, float4* __restrict__ R, long long n4, float rho) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4;
+       i += (long long)gridDim.x * blockDim.x) {
+    const float4 h = H[i], z = Z[i], u = U[i];
+    float4 r;
+    r.x = -(u.x + rho * (z.x - h.x));
+    r.y = -(u.y + rho * (z.y - h.y));
+    r.z = -(u.z + rho * (z.z - h.z));
+    r.w = -(u.w + rho * (z.w - h.w));
+    R[i] = r;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Step-size search of a W block (Section 3.1).  Along W - grad/t the pre-activation is
+// H - D/t with D = P grad, so every candidate is scored from H, D, Z without another product.
+// ------------------------------------------------------------------------------------------
+// hidden layer: acc[j] += sum ( (z - f(h - d/t_j))^2 - (z - f(h))^2 )   (times nu/2 at decision time)
+__global__ void __launch_bounds__(256)
+k_score_w_hidden(const float4* __restrict__ H, const float4* __restrict__ D, const float4* __restrict__ Z,
+                 long long n4, const SearchCtl* __restrict__ ctl, double* __restrict__ acc) {
+  if (ctl->done) return;
+  __shared__ double sh[32];
+  float inv[kCand];
+#pragma unroll
+  for (int j = 0; j < kCand; ++j) inv[j] = ctl->inv_cand[j];
+  double s[kCand];
+#pragma unroll
+  for (int j = 0; j < kCand; ++j) s[j] = 0.0;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4;
+       i += (long long)gridDim.x * blockDim.x) {
+    const float4 h4 = H[i], d4 = D[i], z4 = Z[i];
+    const float h[4] = {h4.x, h4.y, h4.z, h4.w}, d[4] = {d4.x, d4.y, d4.z, d4.w},
+                z[4] = {z4.x, z4.y, z4.z, z4.w};
+    float part[kCand];
+#pragma unroll
+    for (int j = 0; j < kCand; ++j) part[j] = 0.f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const float f0 = relu(h[c]);
+      const float e0 = z[c] - f0;
+#pragma unroll
+      for (int j = 0; j < kCand; ++j) {
+        const float f1 = relu(fmaf(-d[c], inv[j], h[c]));
+        const float e1 = z[c] - f1;
+        part[j] = fmaf(f0 - f1, e1 + e0, part[j]);   // e1^2 - e0^2 = (e1 - e0)(e1 + e0)
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < kCand; ++j) s[j] += (double)part[j];
+  }
+#pragma unroll
+  for (int j = 0; j < kCand; ++j) {
+    const double v = block_sum(s[j], sh);
+    if (threadIdx.x == 0) atomicAdd(acc + j, v);
+  }
+}
+
+// last layer: phi_L(t) - phi_L = -(1/t) <D, R> + (rho / 2t^2) ||D||^2 ; acc[0] += <D,R>, acc[1] += ||D||^2
+__global__ void __launch_bounds__(256)
+k_score_w_out(const float4* __restrict__ D, const float4* __restrict__ R, long long n4,
+              const SearchCtl* __restrict__ ctl, double* __restrict__ acc) {
+  if (ctl->done) return;
+  __shared__ double sh[32];
+  double s1 = 0.0, s2 = 0.0;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4;
+       i += (long long)gridDim.x * blockDim.x) {
+    const float4 d = D[i], r = R[i];
+    s1 += (double)(d.x * r.x + d.y * r.y + d.z * r.z + d.w * r.w);
+    s2 += (double)(d.x * d.x + d.y * d.y + d.z * d.z + d.w * d.w);
+  }
+  s1 = block_sum(s1, sh);
+  s2 = block_sum(s2, sh);
+  if (threadIdx.x == 0) { atomicAdd(acc, s1); atomicAdd(acc + 1, s2); }
+}
+
+__device__ __forceinline__ void set_candidates(SearchCtl* c, double growth) {
+  double t = c->t_base;
+#pragma unroll
+  for (int j = 0; j < kCand; ++j) { c->inv_cand[j] = (float)(1.0 / t); t *= growth; }
+}
+
+// Starts `count` searches: sums[i*stride + 0] = ||grad||^2, sums[i*stride + 1] = ||x||^2.
+__global__ void k_search_begin(SearchCtl* ctl, int count, const double* __restrict__ sums, int stride,
+                               double shrink, double growth, double* __restrict__ acc, int acc_per,
+                               int* __restrict__ n_active) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  SearchCtl* c = ctl + i;
+  c->gg = sums[i * stride];
+  c->xx = sums[i * stride + 1];
+  c->pass = 0;
+  c->q = 0.0;
+  c->inv_step = 0.f;
+  for (int j = 0; j < acc_per; ++j) acc[i * acc_per + j] = 0.0;
+  if (!(c->gg > 1e-24 * c->xx)) {          // zero up to rounding (also catches NaN): skip
+    c->done = 1;
+    c->trial = (c->gg == c->gg) ? -1 : -2;
+    return;
+  }
+  c->done = 0;
+  c->trial = -2;
+  c->t_base = fmax(c->t_prev * shrink, 1e-12);
+  set_candidates(c, growth);
+  if (n_active) atomicAdd(n_active, 1);
+}
+
+// One decision per search.  mode 0: acc holds kCand sums of a scoring pass, delta_j = scale * acc[j]
+// plus the quadratic own term; mode 1: closed form, delta(t) = -lin/t + quad/t^2, all trials at once.
+//   own term (Z blocks only): -(nu/t) sag + (nu/2t^2) sgg with sag = <Z - f(H), G>, sgg = gg
+struct DecideArgs {
+  double growth;
+  int max_trials;
+  int mode;          // 0 scored candidates, 1 closed form
+  double scale;      // multiplies the scored sums (nu/2)
+  double quad_coef;  // closed form: delta = -acc[0]/t + quad_coef * acc[1] / t^2
+  double own_nu;     // nu when the block has a quadratic own term, else 0
+  int last_pass;     // this is the final pass: mark exhausted searches
+};
+
+__device__ __forceinline__ bool accept(SearchCtl* c, double delta, double t, int trial) {
+  const double need = c->gg / (2.0 * t);
+  if (delta <= -need) {          // f(x+) - f(x) <= -||g||^2 / (2t); false for NaN
+    c->t_prev = t;
+    c->q = -delta / need;
+    c->inv_step = (float)(1.0 / t);
+    c->trial = trial;
+    c->done = 1;
+    return true;
+  }
+  return false;
+}
+
+__global__ void k_search_decide(SearchCtl* ctl, int count, double* __restrict__ acc, int acc_per,
+                                const double* __restrict__ own, int own_stride, DecideArgs a,
+                                int* __restrict__ n_active, int* __restrict__ status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  SearchCtl* c = ctl + i;
+  if (c->done) return;
+  const double sag = (a.own_nu != 0.0) ? own[i * own_stride + 2] : 0.0;
+  if (a.mode == 1) {
+    double t = c->t_base;
+    const double lin = acc[i * acc_per], quad = a.quad_coef * acc[i * acc_per + 1];
+    bool ok = false;
+    for (int trial = 0; trial < a.max_trials && !ok; ++trial) {
+      const double delta = -lin / t + quad / (t * t) - a.own_nu * sag / t + 0.5 * a.own_nu * c->gg / (t * t);
+      ok = accept(c, delta, t, trial);
+      t *= a.growth;
+    }
+    if (!ok) { c->done = 1; c->trial = -2; c->inv_step = 0.f; if (!(lin == lin && quad == quad)) atomicOr(status, 1); }
+    if (n_active) atomicSub(n_active, 1);
+    return;
+  }
+  double t = c->t_base;
+  bool ok = false, finite = true;
+  for (int j = 0; j < kCand && !ok; ++j) {
+    const int trial = c->pass * kCand + j;
+    if (trial >= a.max_trials) break;
+    const double sum = acc[i * acc_per + j];
+    finite = finite && (sum == sum);
+    const double delta = a.scale * sum - a.own_nu * sag / t + 0.5 * a.own_nu * c->gg / (t * t);
+    ok = accept(c, delta, t, trial);
+    t *= a.growth;
+  }
+  if (!finite) atomicOr(status, 1);
+  if (ok) { if (n_active) atomicSub(n_active, 1); return; }
+  c->pass += 1;
+  if (a.last_pass || c->pass * kCand >= a.max_trials) {
+    c->done = 1; c->trial = -2; c->inv_step = 0.f;
+    if (n_active) atomicSub(n_active, 1);
+    return;
+  }
+  c->t_base = t;
+  set_candidates(c, a.growth);
+  for (int j = 0; j < acc_per; ++j) acc[i * acc_per + j] = 0.0;
+}
+
+// Copies the decision of each search into the log of this pass.
+__global__ void k_log_decisions(const SearchCtl* __restrict__ ctl, int count, int* __restrict__ trial,
+                                double* __restrict__ q) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  trial[i] = ctl[i].trial;
+  q[i] = ctl[i].q;
+}
+
+// W <- W - grad / tau (and its transpose copy), C_prev x C matrices with padded leading dimensions.
+__global__ void k_apply_w(float* __restrict__ W, float* __restrict__ Wt, const float* __restrict__ grad,
+                          int rows, int cols, int ldw, int ldwt, const SearchCtl* __restrict__ ctl) {
+  const float s = ctl->inv_step;
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= rows * cols) return;
+  const int r = e / cols, c = e % cols;
+  const float w = fmaf(-grad[r * ldw + c], s, W[r * ldw + c]);
+  W[r * ldw + c] = w;
+  Wt[c * ldwt + r] = w;
+}
+
+// Y <- Y - s X with s = ctl->inv_step (H <- H - D/tau).
+__global__ void k_axpy_ctl(float4* __restrict__ Y, const float4* __restrict__ X, long long n4,
+                           const SearchCtl* __restrict__ ctl) {
+  const float s = ctl->inv_step;
+  if (s == 0.f) return;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4;
+       i += (long long)gridDim.x * blockDim.x) {
+    float4 y = Y[i];
+    const float4 x = X[i];
+    y.x = fmaf(-s, x.x, y.x); y.y = fmaf(-s, x.y, y.y); y.z = fmaf(-s, x.z, y.z); y.w = fmaf(-s, x.w, y.w);
+    Y[i] = y;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Hidden Z blocks (Appendix A).  The gradient of psi_m with respect to Z_{l,m} is the rows V_m of
+//   G = nu (Z_l - f(H_l)) + (A~ R') W_{l+1}^T ,
+// R' the residual of layer l+1 at the new W.  k_zgrad_finish adds the first term to the product
+// and accumulates, per community, sums[m] = { ||G_m||^2, ||Z_{l,m}||^2, <Z_l - f(H_l), G>_m }.
+// One block owns `rows_per_block` consecutive rows.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+k_zgrad_finish(float4* __restrict__ G, const float4* __restrict__ Z, const float4* __restrict__ H, int ld4,
+               long long n, int rows_per_block, const int* __restrict__ row_comm, float nu,
+               double* __restrict__ sums) {
+  __shared__ double sh[32];
+  const long long r0 = (long long)blockIdx.x * rows_per_block;
+  const long long r1 = min(n, r0 + rows_per_block);
+  if (r0 >= r1) return;
+  const bool single = row_comm[r0] == row_comm[r1 - 1];
+  double sgg = 0.0, szz = 0.0, sag = 0.0;
+  int cur = row_comm[r0];
+  const long long e0 = r0 * ld4, e1 = r1 * ld4;
+  for (long long e = e0 + threadIdx.x; e < e1; e += blockDim.x) {
+    const float4 z = Z[e], h = H[e];
+    float4 g = G[e];
+    const float ax = z.x - relu(h.x), ay = z.y - relu(h.y), az = z.z - relu(h.z), aw = z.w - relu(h.w);
+    g.x = fmaf(nu, ax, g.x); g.y = fmaf(nu, ay, g.y); g.z = fmaf(nu, az, g.z); g.w = fmaf(nu, aw, g.w);
+    G[e] = g;
+    if (!single) {
+      const int m = row_comm[e / ld4];
+      if (m != cur) {
+        atomicAdd(sums + cur * 3 + 0, sgg); atomicAdd(sums + cur * 3 + 1, szz); atomicAdd(sums + cur * 3 + 2, sag);
+        sgg = szz = sag = 0.0;
+        cur = m;
+      }
+    }
+    sgg += (double)(g.x * g.x + g.y * g.y + g.z * g.z + g.w * g.w);
+    szz += (double)(z.x * z.x + z.y * z.y + z.z * z.z + z.w * z.w);
+    sag += (double)(ax * g.x + ay * g.y + az * g.z + aw * g.w);
+  }
+  if (single) {
+    sgg = block_sum(sgg, sh); szz = block_sum(szz, sh); sag = block_sum(sag, sh);
+    if (threadIdx.x == 0) {
+      atomicAdd(sums + cur * 3 + 0, sgg); atomicAdd(sums + cur * 3 + 1, szz); atomicAdd(sums + cur * 3 + 2, sag);
+    }
+  } else {
+    atomicAdd(sums + cur * 3 + 0, sgg); atomicAdd(sums + cur * 3 + 1, szz); atomicAdd(sums + cur * 3 + 2, sag);
+  }
+}
+
+// Scoring of the theta candidates of every community in one sweep over the rows.
+// With T = G W_{l+1}, the move of community m changes the pre-activation of row i by
+//   -K_m[i] / theta_m ,  K_m[i] = sum over j in V_m of A~_ij T_j  (row i of A~_{comm(i),m} T_m),
+// which is non-zero on V_m and its first-order neighbour rows only.  A warp owns row i, walks the
+// segments of the row (one per neighbouring community), forms K_m[i] and scores it.
+//   OUT = false (layer l+1 < L, ReLU):  acc[m*kCand + j] += sum_c (z - f(h - k/t_j))^2 - (z - f(h))^2
+//   OUT = true  (layer l+1 = L):        acc[m*2] += <k, R'>, acc[m*2+1] += ||k||^2   (closed form)
+// V = float4 columns per lane (width <= 128 V).
+template <int V, bool OUT>
+__global__ void __launch_bounds__(256)
+k_score_z(const int* __restrict__ col, const float* __restrict__ dinv,
+          const int* __restrict__ seg_row_ptr, const int* __restrict__ seg_comm,
+          const int* __restrict__ seg_begin, const float4* __restrict__ T, const float4* __restrict__ Hn,
+          const float4* __restrict__ Zn, const float4* __restrict__ Rn, int ld4, int n,
+          const SearchCtl* __restrict__ ctl, int n_comm, double* __restrict__ acc,
+          const int* __restrict__ n_active, int use_smem) {
+  if (*n_active <= 0) return;
+  constexpr int PER = OUT ? 2 : kCand;
+  extern __shared__ double s_acc[];
+  double* accp = acc;
+  if (use_smem) {
+    for (int i = threadIdx.x; i < n_comm * PER; i += blockDim.x) s_acc[i] = 0.0;
+    __syncthreads();
+    accp = s_acc;
+  }
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = blockDim.x >> 5;
+  const int row = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+  if (row < n) {
+    float4 a[V], b[V];   // OUT: a = R' ; else a = h, b = z
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+      const int f = lane + 32 * v;
+      a[v] = b[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (f < ld4) {
+        if (OUT) a[v] = Rn[(long long)row * ld4 + f];
+        else { a[v] = Hn[(long long)row * ld4 + f]; b[v] = Zn[(long long)row * ld4 + f]; }
+      }
+    }
+    const float di = dinv[row];
+    const int s0 = seg_row_ptr[row], s1 = seg_row_ptr[row + 1];
+    for (int s = s0; s < s1; ++s) {
+      const int m = seg_comm[s];
+      if (ctl[m].done) continue;
+      const int pb = seg_begin[s], pe = seg_begin[s + 1];
+      float4 k[V];
+#pragma unroll
+      for (int v = 0; v < V; ++v) k[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int base = pb; base < pe; base += 32) {
+        const int idx = base + lane;
+        int c = 0;
+        float w = 0.f;
+        if (idx < pe) { c = col[idx]; w = dinv[c]; }
+        const int cnt = min(32, pe - base);
+        for (int t = 0; t < cnt; t += 4) {
+          int cj[4];
+          float wj[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            cj[u] = __shfl_sync(0xffffffffu, c, (t + u) & 31);
+            wj[u] = __shfl_sync(0xffffffffu, w, (t + u) & 31);
+            if (t + u >= 32) wj[u] = 0.f;
+          }
+#pragma unroll
+          for (int v = 0; v < V; ++v) {
+            const int f = lane + 32 * v;
+            if (f < ld4) {
+              float4 xv[4];
+#pragma unroll
+              for (int u = 0; u < 4; ++u) xv[u] = __ldg(T + (long long)cj[u] * ld4 + f);
+#pragma unroll
+              for (int u = 0; u < 4; ++u) {
+                k[v].x = fmaf(wj[u], xv[u].x, k[v].x); k[v].y = fmaf(wj[u], xv[u].y, k[v].y);
+                k[v].z = fmaf(wj[u], xv[u].z, k[v].z); k[v].w = fmaf(wj[u], xv[u].w, k[v].w);
+              }
+            }
+          }
+        }
+      }
+      if (OUT) {
+        float p1 = 0.f, p2 = 0.f;
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+          const float kx = di * k[v].x, ky = di * k[v].y, kz = di * k[v].z, kw = di * k[v].w;
+          p1 += kx * a[v].x + ky * a[v].y + kz * a[v].z + kw * a[v].w;
+          p2 += kx * kx + ky * ky + kz * kz + kw * kw;
+        }
+        p1 = warp_sum(p1);
+        p2 = warp_sum(p2);
+        if (lane == 0) { atomicAdd(accp + m * 2, (double)p1); atomicAdd(accp + m * 2 + 1, (double)p2); }
+      } else {
+        float inv[kCand], part[kCand];
+#pragma unroll
+        for (int j = 0; j < kCand; ++j) { inv[j] = ctl[m].inv_cand[j]; part[j] = 0.f; }
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+          const float kk[4] = {di * k[v].x, di * k[v].y, di * k[v].z, di * k[v].w};
+          const float hh[4] = {a[v].x, a[v].y, a[v].z, a[v].w};
+          const float zz[4] = {b[v].x, b[v].y, b[v].z, b[v].w};
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const float f0 = relu(hh[c]);
+            const float e0 = zz[c] - f0;
+#pragma unroll
+            for (int j = 0; j < kCand; ++j) {
+              const float f1 = relu(fmaf(-kk[c], inv[j], hh[c]));
+              part[j] = fmaf(f0 - f1, (zz[c] - f1) + e0, part[j]);
+            }
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < kCand; ++j) {
+          const float v = warp_sum(part[j]);
+          if (lane == 0) atomicAdd(accp + m * kCand + j, (double)v);
+        }
+      }
+    }
+  }
+  if (use_smem) {
+    __syncthreads();
+    for (int i = threadIdx.x; i < n_comm * PER; i += blockDim.x)
+      if (s_acc[i] != 0.0) atomicAdd(acc + i, s_acc[i]);
+  }
+}
+
+// Z_l[i,:] <- Z_l[i,:] - G[i,:] / theta_{comm(i)}   (Eq. 10)
+__global__ void k_apply_z(float4* __restrict__ Z, const float4* __restrict__ G, int ld4, long long n,
+                          const int* __restrict__ row_comm, const SearchCtl* __restrict__ ctl) {
+  const long long total = n * ld4;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total;
+       e += (long long)gridDim.x * blockDim.x) {
+    const float s = ctl[row_comm[e / ld4]].inv_step;
+    if (s == 0.f) continue;
+    float4 z = Z[e];
+    const float4 g = G[e];
+    z.x = fmaf(-s, g.x, z.x); z.y = fmaf(-s, g.y, z.y); z.z = fmaf(-s, g.z, z.z); z.w = fmaf(-s, g.w, z.w);
+    Z[e] = z;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Output layer rows (Eq. 7) and the dual (Eq. 3), one warp per row, classes spread over lanes.
+//   q = row of A~ Z_{L-1}^k W_L^{k+1};  training rows: FISTA on
+//   loss_scale * CE(z, y) + <u, z - q> + (rho/2)||z - q||^2 ;  other rows: z = q - u / rho.
+//   dual_now != 0: U <- u + rho (z_old - q) in the same sweep (Eq. 3 as printed).
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+k_output_rows(float* __restrict__ ZL, float* __restrict__ U, const float* __restrict__ HL, int ld, int C,
+              int n, const int* __restrict__ y, const unsigned char* __restrict__ train, float rho,
+              float loss_scale, int iters, int dual_now, int update_z) {
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= n) return;
+  float q[kMaxClassesPerLane], u[kMaxClassesPerLane], z[kMaxClassesPerLane];
+  const long long base = (long long)row * ld;
+#pragma unroll
+  for (int t = 0; t < kMaxClassesPerLane; ++t) {
+    const int c = lane + 32 * t;
+    q[t] = u[t] = z[t] = 0.f;
+    if (c < C) { q[t] = HL[base + c]; u[t] = U[base + c]; z[t] = ZL[base + c]; }
+  }
+  if (dual_now) {
+#pragma unroll
+    for (int t = 0; t < kMaxClassesPerLane; ++t) {
+      const int c = lane + 32 * t;
+      if (c < C) U[base + c] = fmaf(rho, z[t] - q[t], u[t]);
+    }
+  }
+  if (!update_z) return;
+  if (!train[row]) {
+    const float inv_rho = 1.f / rho;
+#pragma unroll
+    for (int t = 0; t < kMaxClassesPerLane; ++t) {
+      const int c = lane + 32 * t;
+      if (c < C) ZL[base + c] = fmaf(-u[t], inv_rho, q[t]);
+    }
+    return;
+  }
+  const int yi = y[row];
+  const float step = 1.f / (0.5f * loss_scale + rho);
+  float xp[kMaxClassesPerLane], v[kMaxClassesPerLane];
+#pragma unroll
+  for (int t = 0; t < kMaxClassesPerLane; ++t) { xp[t] = z[t]; v[t] = z[t]; }
+  double tm = 1.0;
+  for (int it = 0; it < iters; ++it) {
+    float mx = -3.0e38f;
+#pragma unroll
+    for (int t = 0; t < kMaxClassesPerLane; ++t)
+      if (lane + 32 * t < C) mx = fmaxf(mx, v[t]);
+    mx = warp_max(mx);
+    float ex[kMaxClassesPerLane], se = 0.f;
+#pragma unroll
+    for (int t = 0; t < kMaxClassesPerLane; ++t) {
+      ex[t] = (lane + 32 * t < C) ? expf(v[t] - mx) : 0.f;
+      se += ex[t];
+    }
+    se = warp_sum(se);
+    const float inv_se = 1.f / se;
+    const double tn = 0.5 * (1.0 + sqrt(1.0 + 4.0 * tm * tm));
+    const float mom = (float)((tm - 1.0) / tn);
+#pragma unroll
+    for (int t = 0; t < kMaxClassesPerLane; ++t) {
+      const int c = lane + 32 * t;
+      const float p = ex[t] * inv_se - (c == yi ? 1.f : 0.f);
+      const float g = loss_scale * p + u[t] + rho * (v[t] - q[t]);
+      const float x = fmaf(-step, g, v[t]);
+      v[t] = fmaf(mom, x - xp[t], x);
+      xp[t] = x;
+    }
+    tm = tn;
+  }
+#pragma unroll
+  for (int t = 0; t < kMaxClassesPerLane; ++t) {
+    const int c = lane + 32 * t;
+    if (c < C) ZL[base + c] = xp[t];
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Reporting (Eq. 1) and the forward pass of Problem 1.
+// ------------------------------------------------------------------------------------------
+// out[0] += sum (z - f(h))^2
+__global__ void __launch_bounds__(256)
+k_sum_hidden_penalty(const float4* __restrict__ Z, const float4* __restrict__ H, long long n4,
+                     double* __restrict__ out) {
+  __shared__ double sh[32];
+  double s = 0.0;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4;
+       i += (long long)gridDim.x * blockDim.x) {
+    const float4 z = Z[i], h = H[i];
+    const float a = z.x - relu(h.x), b = z.y - relu(h.y), c = z.z - relu(h.z), d = z.w - relu(h.w);
+    s += (double)(a * a + b * b + c * c + d * d);
+  }
+  s = block_sum(s, sh);
+  if (threadIdx.x == 0) atomicAdd(out, s);
+}
+
+// out[0] += <U, Z - H>, out[1] += ||Z - H||^2
+__global__ void __launch_bounds__(256)
+k_sum_constraint(const float4* __restrict__ Z, const float4* __restrict__ H, const float4* __restrict__ U,
+                 long long n4, double* __restrict__ out) {
+  __shared__ double sh[32];
+  double s1 = 0.0, s2 = 0.0;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4;
+       i += (long long)gridDim.x * blockDim.x) {
+    const float4 z = Z[i], h = H[i], u = U[i];
+    const float a = z.x - h.x, b = z.y - h.y, c = z.z - h.z, d = z.w - h.w;
+    s1 += (double)(u.x * a + u.y * b + u.z * c + u.w * d);
+    s2 += (double)(a * a + b * b + c * c + d * d);
+  }
+  s1 = block_sum(s1, sh);
+  s2 = block_sum(s2, sh);
+  if (threadIdx.x == 0) { atomicAdd(out, s1); atomicAdd(out + 1, s2); }
+}
+
+// Per row: cross-entropy of the row of Zrows with its label (training rows only) summed into out[0];
+// argmax of the row of `logits` (lowest index on ties) to labels[row]; out[1] += training rows whose
+// argmax equals the label.  One warp per row.  Either of Zrows / logits may be NULL.
+__global__ void __launch_bounds__(256)
+k_row_loss_argmax(const float* __restrict__ Zrows, const float* __restrict__ logits, int ld, int C, int n,
+                  const int* __restrict__ y, const unsigned char* __restrict__ train,
+                  int* __restrict__ labels, double* __restrict__ out) {
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= n) return;
+  const long long base = (long long)row * ld;
+  const bool tr = train[row] != 0;
+  if (Zrows != nullptr && tr) {
+    float mx = -3.0e38f;
+    for (int c = lane; c < C; c += 32) mx = fmaxf(mx, Zrows[base + c]);
+    mx = warp_max(mx);
+    float se = 0.f;
+    for (int c = lane; c < C; c += 32) se += expf(Zrows[base + c] - mx);
+    se = warp_sum(se);
+    if (lane == 0) atomicAdd(out, (double)(mx + logf(se) - Zrows[base + y[row]]));
+  }
+  if (logits != nullptr) {
+    float best = -3.0e38f;
+    int arg = 0x7fffffff;
+    for (int c = lane; c < C; c += 32) {
+      const float v = logits[base + c];
+      if (v > best) { best = v; arg = c; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oa = __shfl_xor_sync(0xffffffffu, arg, o);
+      if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
+    }
+    if (lane == 0) {
+      if (labels) labels[row] = arg;
+      if (tr && arg == y[row]) atomicAdd(out + 1, 1.0);
+    }
+  }
+}
+
+// Y = relu(Y) in place.
+__global__ void k_relu_inplace(float4* __restrict__ Y, long long n4) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4;
+       i += (long long)gridDim.x * blockDim.x) {
+    float4 y = Y[i];
+    y.x = relu(y.x); y.y = relu(y.y); y.z = relu(y.z); y.w = relu(y.w);
+    Y[i] = y;
+  }
+}
+
+// U <- U + rho (Z - H)
+__global__ void k_dual(float4* __restrict__ U, const float4* __restrict__ Z, const float4* __restrict__ H,
+                       long long n4, float rho) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4;
+       i += (long long)gridDim.x * blockDim.x) {
+    float4 u = U[i];
+    const float4 z = Z[i], h = H[i];
+    u.x = fmaf(rho, z.x - h.x, u.x); u.y = fmaf(rho, z.y - h.y, u.y);
+    u.z = fmaf(rho, z.z - h.z, u.z); u.w = fmaf(rho, z.w - h.w, u.w);
+    U[i] = u;
+  }
+}
+
+__global__ void k_fill_int(int* __restrict__ p, long long count, int value) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count;
+       i += (long long)gridDim.x * blockDim.x)
+    p[i] = value;
+}
+
+// Row gather / scatter between the caller's dense layout (original order, width C) and the
+// internal one (community order, leading dimension ld).  to_internal != 0: dst[new] = src[perm[new]].
+__global__ void k_permute_rows(const float* __restrict__ src, float* __restrict__ dst, const int* __restrict__ perm,
+                               long long n, int C, int ld, int to_internal) {
+  const long long total = n * ld;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total;
+       e += (long long)gridDim.x * blockDim.x) {
+    const long long r = e / ld;
+    const int c = (int)(e % ld);
+    if (to_internal) dst[e] = (c < C) ? src[(long long)perm[r] * C + c] : 0.f;
+    else if (c < C) dst[(long long)perm[r] * C + c] = src[e];
+  }
+}
+
+}  // namespace gk
