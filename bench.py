@@ -1,0 +1,326 @@
+#!/usr/bin/env python
+"""Benchmark of the community-based ADMM GCN trainer: ADMM iterations per second.
+
+One "step" is one full pass of Algorithm 1 (every W_l, every Z_{l,m}, Z_L, U) on the largest
+synthetic workload ("powerlaw-xlarge": 2.45 M nodes, ~62 M edges, 100-256-256-47, 64 communities).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints one JSON line.  With --gpus N > 1 (under torchrun) every rank runs an independent replica
+of the same workload on its own GPU (the method is not sharded across GPUs here) and the value is
+the aggregate over the replicas.  --impl reference times the fp64 CPU oracle on a bounded, scaled
+down sample of the same workload on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "admm_iterations_per_sec"
+UNIT = "iterations/s"
+WORKLOAD_INDEX = 4
+FP32_LANES_PER_SM = 128
+SM_COUNT = 148
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    sm_max_mhz=float(d.get("sm_max_mhz", 1965.0)), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, sm_max_mhz=1965.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index):
+        self.device_index = device_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-lms", "200", "-i", str(self.device_index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                smax.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(smax) if smax else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def config_dict(wl, extra=None):
+    d = dict(workload=wl.name, nodes=int(wl.n), edges=int(wl.n_edges), widths=list(wl.widths), communities=int(wl.n_comm),
+             train_rows=int(wl.train_mask.sum()), nu=wl.nu, rho=wl.rho,
+             l2_policy="working set (tens of GB per iteration) far exceeds the 126 MB L2; no flush needed")
+    if extra:
+        d.update(extra)
+    return d
+
+
+def oracle_rate(index, scale, iters, warm):
+    """Seconds per oracle iteration on a scaled-down sample of workload `index`."""
+    from oracle import gcn_admm_oracle as orc
+    from paper_2112_09335_b200 import inputs
+    wl = inputs.make_workload(index, scale=scale)
+    o = orc.OracleADMM(wl.n, wl.row_ptr, wl.col_idx, wl.X, wl.y, wl.train_mask, wl.widths,
+                       orc.Params(nu=wl.nu, rho=wl.rho), wl.n_comm, wl.community, wl.w_init)
+    for _ in range(warm):
+        o.iterate()
+    t0 = time.perf_counter()
+    for _ in range(iters):
+        o.iterate()
+    dt = (time.perf_counter() - t0) / max(iters, 1)
+    return wl, dt
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([int(p.get("num_threads", 1)) for p in threadpool_info()] + [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    """The fp64 CPU oracle, as it stands, on a bounded sample: the workload's recipe at 1/1000 of
+    its node and edge counts (same widths, same number of communities).  The figure is scaled to
+    the full workload in proportion to the edge count, which flatters the oracle (its cost grows
+    faster than linearly)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2112_09335_b200 import inputs
+    scale = 0.001
+    full = inputs.CONFIGS[WORKLOAD_INDEX]
+    wl, dt = oracle_rate(WORKLOAD_INDEX, scale, args.steps, args.warmup)
+    frac = wl.n_edges / full["edges"]
+    value = (1.0 / dt) * frac
+    cores = blas_threads()
+    sample = (f"oracle iteration on the same recipe at scale {scale} ({wl.n} nodes, {wl.n_edges} edges, "
+              f"{wl.n_comm} communities); rate multiplied by edge ratio {frac:.3e}")
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=dt * 1e3 / frac, higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="f64", data="synthetic",
+                config=config_dict(wl, dict(workload=full["name"], sampled_as=wl.name)),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+def kernel_table(prof, iters, peaks):
+    """Per kernel kind: launches and ms per iteration, achieved GB/s and TFLOP/s on algorithmic work."""
+    rows = []
+    total = sum(v["ms"] for v in prof.values()) or 1.0
+    for name, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"]):
+        ms = v["ms"]
+        rows.append(dict(kernel=name, launches_per_iter=v["launches"] / iters, ms_per_iter=ms / iters,
+                         share=ms / total, gbs=(v["bytes"] / (ms * 1e-3) / 1e9) if ms > 0 else 0.0,
+                         tflops=(v["flops"] / (ms * 1e-3) / 1e12) if ms > 0 else 0.0,
+                         bytes_per_launch=v["bytes"] / max(v["launches"], 1), flops_per_launch=v["flops"] / max(v["launches"], 1)))
+    return rows
+
+
+def run_ours(args):
+    import torch
+    from paper_2112_09335_b200 import binding, build, inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    build.build()
+    peaks = measured_peaks()
+
+    wl = inputs.make_workload(args.config, scale=args.scale)
+    stream = torch.cuda.current_stream()
+
+    def make(host_arrays=None):
+        src = host_arrays or dict(row_ptr=wl.row_ptr, col_idx=wl.col_idx, X=wl.X, y=wl.y, train_mask=wl.train_mask,
+                                  community=wl.community)
+        return binding.GcnAdmm(wl.n, src["row_ptr"], src["col_idx"], src["X"], src["y"], src["train_mask"], wl.widths,
+                               wl.n_comm, src["community"], wl.w_init, nu=wl.nu, rho=wl.rho, device=local,
+                               stream=stream.cuda_stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    g = make()
+    g.step(args.warmup)
+    torch.cuda.synchronize()
+
+    # ---- device-resident timing: K iterations between two events on the library's stream ----
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = g.launches()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record(stream)
+    g.step(args.steps)
+    ev1.record(stream)
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    launches = g.launches() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    if dist is not None:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    obj = g.objective()
+    dec = g.decisions()
+    exhausted = int((dec["trial_w"] == -2).sum() + (dec["trial_z"] == -2).sum())
+
+    # ---- per-kernel times (events around every launch) on further iterations of the same state ----
+    prof_iters = max(2, min(args.steps, 5))
+    g.profile(True)
+    g.step(prof_iters)
+    prof = g.profile_read()
+    g.profile(False)
+    table = kernel_table(prof, prof_iters, peaks)
+    g.destroy()
+    del g
+    torch.cuda.empty_cache()
+
+    # ---- end to end through the C ABI from pinned host buffers: create + K iterations + read-back ----
+    pinned = {}
+    for key, arr in dict(row_ptr=wl.row_ptr, col_idx=wl.col_idx, X=wl.X, y=wl.y, train_mask=wl.train_mask,
+                         community=wl.community).items():
+        t = torch.from_numpy(np.ascontiguousarray(arr)).pin_memory()
+        pinned[key] = t
+    host_np = {k: v.numpy() for k, v in pinned.items()}
+    h2d = sum(v.numel() * v.element_size() for v in pinned.values()) + sum(w.nbytes for w in wl.w_init)
+    barrier()
+    t0 = time.perf_counter()
+    g2 = make(host_np)
+    g2.step(args.steps)
+    ws = [g2.weights(l) for l in range(1, len(wl.widths))]
+    obj2 = g2.objective()
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    d2h = sum(w.nbytes for w in ws) + 48
+    if dist is not None:
+        t = torch.tensor([e2e_s], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    g2.destroy()
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    value = world * args.steps / (ms * 1e-3)
+    dominant = table[0]
+    alu_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12   # fp32 FMA TFLOP/s
+    if dominant["kernel"].startswith("gemm"):
+        roofline = dict(bound="alu", achieved=dominant["tflops"], peak=alu_peak, unit="TFLOP/s",
+                        frac=dominant["tflops"] / alu_peak, traffic=None,
+                        peak_source="148 SMs x 128 fp32 lanes x 2 flop x max SM clock")
+    else:
+        roofline = dict(bound="hbm", achieved=dominant["gbs"], peak=peaks["hbm_gbs"], unit="GB/s",
+                        frac=dominant["gbs"] / peaks["hbm_gbs"], traffic=None, peak_source=peaks["source"])
+    roofline.update(kernel=dominant["kernel"], ms_per_launch=dominant["ms_per_iter"] / max(dominant["launches_per_iter"], 1e-9),
+                    share_of_kernel_time=dominant["share"])
+
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                ms_per_step=ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32",
+                data="synthetic", config=config_dict(wl, dict(parallelism="replicas only" if world > 1 else "single GPU")),
+                clocks=clocks, gpu_launches=int(launches),
+                e2e=dict(value=world * args.steps / e2e_s, unit=UNIT, h2d_bytes_per_step=h2d / args.steps,
+                         d2h_bytes_per_step=d2h / args.steps, seconds=e2e_s,
+                         what="gcn_admm_create from pinned host buffers + K iterations + weights and objective read back"),
+                roofline=roofline,
+                kernels=[dict(kernel=r["kernel"], ms_per_iter=round(r["ms_per_iter"], 4), share=round(r["share"], 4),
+                              launches_per_iter=round(r["launches_per_iter"], 2), gbs=round(r["gbs"], 1),
+                              tflops=round(r["tflops"], 2)) for r in table if r["share"] >= 0.002],
+                objective=dict(L_rho=obj[0], R=obj[1], train_acc=obj[5], exhausted_searches=exhausted,
+                               e2e_L_rho=obj2[0]))
+    if world == 1 and not args.no_cpu_baseline:
+        scale = min(1.0, 2450.0 / inputs.CONFIGS[args.config]["n"])      # about 2.4 k nodes of the same recipe
+        wl_s, dt = oracle_rate(args.config, scale, 3, 1)
+        frac = wl_s.n_edges / max(wl.n_edges, 1)
+        line["cpu_baseline"] = dict(value=(1.0 / dt) * frac, unit=UNIT, cores=blas_threads(), kind="oracle",
+                                    sample=(f"3 oracle iterations (after 1) on the same recipe at {wl_s.n} nodes / "
+                                            f"{wl_s.n_edges} edges / {wl_s.n_comm} communities, {dt:.2f} s each; rate "
+                                            f"multiplied by the edge ratio {frac:.3e} (linear scaling flatters the oracle)"))
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=WORKLOAD_INDEX, help="workload index 0..4 (default: the largest)")
+    ap.add_argument("--scale", type=float, default=1.0, help="shrink the workload (profiling captures only)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -173,6 +173,20 @@ int gcn_admm_step_block(gcn_admm* h, int phase, int layer);
 int gcn_admm_decisions(gcn_admm* h, int max_passes, int* n_passes, int* trial_w, double* q_w,
                        int* trial_z, double* q_z);
 
+/* ---- accounting and timing ---------------------------------------------------------------------
+ * gcn_admm_launches: number of kernels this handle has launched since it was created.
+ * gcn_admm_profile(h, 1) clears the per-kernel table and starts bracketing every launch with CUDA
+ * events on the handle's stream (this costs a little time, so leave it off when timing a whole step);
+ * gcn_admm_profile(h, 0) stops.  gcn_admm_profile_read synchronises and returns one entry per kernel
+ * kind ("spmm@256" = propagation at leading dimension 256, "gemm_nn@256x47" = K x N of the product, ...):
+ * launches, summed device time in ms, and the algorithmic bytes and flops of the work those launches
+ * did (what the operation must move / compute, not what the hardware moved).  names: max_entries x 48
+ * chars.  Any output array may be NULL. */
+int gcn_admm_launches(gcn_admm* h, long long* count);
+int gcn_admm_profile(gcn_admm* h, int enable);
+int gcn_admm_profile_read(gcn_admm* h, int max_entries, int* n_entries, char* names, long long* launches,
+                          double* ms, double* bytes, double* flops);
+
 #ifdef __cplusplus
 }
 #endif

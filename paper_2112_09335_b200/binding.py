@@ -18,6 +18,7 @@ EXPORTS = [
     "gcn_admm_default_params", "gcn_admm_create", "gcn_admm_step", "gcn_admm_objective", "gcn_admm_weights",
     "gcn_admm_predict", "gcn_admm_destroy", "gcn_admm_last_error", "gcn_admm_propagate", "gcn_admm_index",
     "gcn_admm_get_state", "gcn_admm_set_state", "gcn_admm_step_block", "gcn_admm_decisions",
+    "gcn_admm_launches", "gcn_admm_profile", "gcn_admm_profile_read",
 ]
 
 IX = dict(perm=0, inv_perm=1, comm_ptr=2, nbr=3, halo1=4, halo2=5, csr_row_ptr=6, csr_col=7,
@@ -69,6 +70,9 @@ def load():
     lib.gcn_admm_set_state.argtypes = [vp, i32, i32, vp]
     lib.gcn_admm_step_block.argtypes = [vp, i32, i32]
     lib.gcn_admm_decisions.argtypes = [vp, i32, C.POINTER(i32), vp, vp, vp, vp]
+    lib.gcn_admm_launches.argtypes = [vp, C.POINTER(i64)]
+    lib.gcn_admm_profile.argtypes = [vp, i32]
+    lib.gcn_admm_profile_read.argtypes = [vp, i32, C.POINTER(i32), vp, vp, vp, vp, vp]
     _lib = lib
     return lib
 
@@ -196,6 +200,27 @@ class GcnAdmm:
         shape, dt = self._state_shape(which, layer)
         v = np.ascontiguousarray(value, dtype=dt).reshape(shape)
         self._check(self._lib.gcn_admm_set_state(self._h, which, layer, _ptr(v)))
+
+    def launches(self):
+        c = C.c_longlong()
+        self._check(self._lib.gcn_admm_launches(self._h, C.byref(c)))
+        return c.value
+
+    def profile(self, enable):
+        self._check(self._lib.gcn_admm_profile(self._h, 1 if enable else 0))
+
+    def profile_read(self, max_entries=128):
+        n = C.c_int()
+        names = C.create_string_buffer(max_entries * 48)
+        la = np.zeros(max_entries, dtype=np.int64)
+        ms, by, fl = (np.zeros(max_entries) for _ in range(3))
+        self._check(self._lib.gcn_admm_profile_read(self._h, max_entries, C.byref(n), names, _ptr(la), _ptr(ms), _ptr(by),
+                                                    _ptr(fl)))
+        out = {}
+        for k in range(n.value):
+            name = names.raw[k * 48:(k + 1) * 48].split(b"\0")[0].decode()
+            out[name] = dict(launches=int(la[k]), ms=float(ms[k]), bytes=float(by[k]), flops=float(fl[k]))
+        return out
 
     def decisions(self, max_passes=256):
         L, M = self.L, self.n_comm

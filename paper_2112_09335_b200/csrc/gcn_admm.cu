@@ -7,6 +7,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <map>
 #include <new>
 #include <string>
 #include <vector>
@@ -60,8 +61,59 @@ bool is_device_pointer(const void* p) {
 
 }  // namespace
 
+struct ProfStat {
+  long long launches = 0;
+  double ms = 0.0, bytes = 0.0, flops = 0.0;
+};
+struct ProfPending {
+  ProfStat* stat;
+  cudaEvent_t a, b;
+};
+
 struct gcn_admm {
   gcn_admm_params p{};
+  // launch accounting: every kernel launch goes through a Scope (below)
+  long long launches = 0;
+  bool profiling = false;
+  std::map<std::string, ProfStat> prof;
+  std::vector<ProfPending> pending;
+  std::vector<cudaEvent_t> event_pool;
+  cudaEvent_t get_event() {
+    if (!event_pool.empty()) { cudaEvent_t e = event_pool.back(); event_pool.pop_back(); return e; }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+  }
+  // Counts `kernels` launches; when profiling, brackets them with events on the handle's stream and
+  // books the algorithmic bytes / flops of the work under `name`.
+  struct Scope {
+    gcn_admm* h;
+    cudaEvent_t b = nullptr;
+    Scope(gcn_admm* h_, const char* name, int kernels, double bytes, double flops) : h(h_) {
+      h->launches += kernels;
+      if (!h->profiling) return;
+      ProfStat& st = h->prof[name];
+      st.launches += kernels;
+      st.bytes += bytes;
+      st.flops += flops;
+      cudaEvent_t a = h->get_event();
+      b = h->get_event();
+      cudaEventRecord(a, h->stream);
+      h->pending.push_back(ProfPending{&st, a, b});
+    }
+    ~Scope() { if (b) cudaEventRecord(b, h->stream); }
+  };
+  void collect_profile() {
+    cudaStreamSynchronize(stream);
+    for (ProfPending& q : pending) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, q.a, q.b) == cudaSuccess) q.stat->ms += ms;
+      event_pool.push_back(q.a);
+      event_pool.push_back(q.b);
+    }
+    pending.clear();
+  }
+
   cudaStream_t stream = nullptr;
   int L = 0;
   long long n = 0;
@@ -109,6 +161,9 @@ struct gcn_admm {
     const float4* x4 = reinterpret_cast<const float4*>(x);
     float4* o4 = reinterpret_cast<float4*>(out);
     const int nn = (int)n;
+    char name[48];
+    std::snprintf(name, sizeof name, "spmm@%d", ldx);
+    Scope sc(this, name, 1, 4.0 * gi.nnz + 8.0 * n + 8.0 * (double)n * ldx, 2.0 * (double)gi.nnz * ldx);
 #define SPMM_CASE(G, V)                                                                        \
   {                                                                                            \
     const long long threads = n * (G);                                                         \
@@ -127,6 +182,9 @@ struct gcn_admm {
 
   void gemm_nn(const float* A, int lda, const float* B, int ldb, float* Cm, int ldc, long long Mr, int N, int K,
                const int* skip = nullptr) {
+    char name[48];
+    std::snprintf(name, sizeof name, "gemm_nn@%dx%d", K, N);
+    Scope sc(this, name, 1, 4.0 * ((double)Mr * (lda + ldc) + (double)K * ldb), 2.0 * (double)Mr * N * K);
 #define NN_CASE(BM, BN, BK, TM, TN)                                                             \
   {                                                                                             \
     dim3 grid((unsigned)cdiv(Mr, BM), (unsigned)cdiv(ldc, BN));                                  \
@@ -144,6 +202,9 @@ struct gcn_admm {
                int Nb) {
     int splits = 1;
     long long rps = rows;
+    char name[48];
+    std::snprintf(name, sizeof name, "gemm_tn@%dx%d", Ka, Nb);
+    Scope sc(this, name, 2, 4.0 * ((double)rows * (lda + ldb) + (double)Ka * ldp), 2.0 * (double)rows * Ka * Nb);
 #define TN_CASE(BM, BN, BK, TM, TN)                                                             \
   {                                                                                             \
     const long long tiles = cdiv(Ka, BM) * cdiv(ldp, BN);                                        \
@@ -167,6 +228,7 @@ struct gcn_admm {
 
   void resid(int l, float* R) {   // derivative of phi_l with respect to H_l, at the stored H_l
     const long long n4 = n * ld[l] / 4;
+    Scope sc(this, l < L ? "resid_hidden" : "resid_out", 1, 16.0 * n4 * (l < L ? 3 : 4), 0.0);
     if (l < L)
       gk::k_resid_hidden<<<grid_for(n4), 256, 0, stream>>>((const float4*)H[l], (const float4*)Z[l], (float4*)R, n4, p.nu);
     else
@@ -184,6 +246,7 @@ struct gcn_admm {
 
   void begin_log_pass() {
     const long long zc = (long long)std::max(L - 1, 0) * M;
+    Scope sc(this, "small", zc > 0 ? 2 : 1, 0.0, 0.0);
     gk::k_fill_int<<<1, 64, 0, stream>>>(log_slot_trial_w(), L, -3);
     if (zc > 0) gk::k_fill_int<<<grid_for(zc), 256, 0, stream>>>(log_slot_trial_z(), zc, -3);
     CU(cudaGetLastError());
@@ -196,34 +259,49 @@ struct gcn_admm {
     SearchCtl* ctl = ctl_w + l;
     resid(l, B0);                                                       // R_l
     gemm_tn(P[l], ld[l - 1], B0, ldc, grad, ldc, n, Kp, Cn);            // grad = P_l^T R_l
-    gk::k_two_sumsq<<<1, 1024, 0, stream>>>(grad, W[l], (long long)Kp * ldc, sums_w);
-    gk::k_search_begin<<<1, 32, 0, stream>>>(ctl, 1, sums_w, 2, p.bt_shrink, p.bt_growth, acc_w, gk::kCand, nullptr);
-    CU(cudaGetLastError());
+    {
+      Scope sc(this, "small", 2, 0.0, 0.0);
+      gk::k_two_sumsq<<<1, 1024, 0, stream>>>(grad, W[l], (long long)Kp * ldc, sums_w);
+      gk::k_search_begin<<<1, 32, 0, stream>>>(ctl, 1, sums_w, 2, p.bt_shrink, p.bt_growth, acc_w, gk::kCand, nullptr);
+      CU(cudaGetLastError());
+    }
     gemm_nn(P[l], ld[l - 1], grad, ldc, B1, ldc, n, Cn, Kp, &ctl->done);   // D = P_l grad
     gk::DecideArgs a{};
     a.growth = p.bt_growth;
     a.max_trials = p.bt_max_trials;
     if (l == L) {
-      gk::k_score_w_out<<<grid_for(n4), 256, 0, stream>>>((const float4*)B1, (const float4*)B0, n4, ctl, acc_w);
+      {
+        Scope sc(this, "score_w_out", 1, 32.0 * n4, 0.0);
+        gk::k_score_w_out<<<grid_for(n4), 256, 0, stream>>>((const float4*)B1, (const float4*)B0, n4, ctl, acc_w);
+      }
       a.mode = 1;
       a.quad_coef = 0.5 * p.rho;
       a.last_pass = 1;
+      Scope sc(this, "small", 1, 0.0, 0.0);
       gk::k_search_decide<<<1, 32, 0, stream>>>(ctl, 1, acc_w, gk::kCand, nullptr, 0, a, nullptr, status);
     } else {
       a.mode = 0;
       a.scale = 0.5 * p.nu;
       const int passes = n_passes();
       for (int ps = 0; ps < passes; ++ps) {
-        gk::k_score_w_hidden<<<grid_for(n4), 256, 0, stream>>>((const float4*)H[l], (const float4*)B1,
-                                                               (const float4*)Z[l], n4, ctl, acc_w);
+        {   // passes after the first almost always find the search finished and return at once
+          Scope sc(this, ps == 0 ? "score_w_hidden" : "score_w_hidden.retry", 1, ps == 0 ? 48.0 * n4 : 0.0, 0.0);
+          gk::k_score_w_hidden<<<grid_for(n4), 256, 0, stream>>>((const float4*)H[l], (const float4*)B1,
+                                                                 (const float4*)Z[l], n4, ctl, acc_w);
+        }
         a.last_pass = (ps == passes - 1);
+        Scope sc(this, "small", 1, 0.0, 0.0);
         gk::k_search_decide<<<1, 32, 0, stream>>>(ctl, 1, acc_w, gk::kCand, nullptr, 0, a, nullptr, status);
       }
     }
     CU(cudaGetLastError());
-    gk::k_log_decisions<<<1, 32, 0, stream>>>(ctl, 1, log_slot_trial_w() + (l - 1), log_slot_q_w() + (l - 1));
-    gk::k_apply_w<<<(unsigned)cdiv((long long)Kp * Cn, 256), 256, 0, stream>>>(W[l], Wt[l], grad, Kp, Cn, ldc,
+    {
+      Scope sc(this, "small", 2, 0.0, 0.0);
+      gk::k_log_decisions<<<1, 32, 0, stream>>>(ctl, 1, log_slot_trial_w() + (l - 1), log_slot_q_w() + (l - 1));
+      gk::k_apply_w<<<(unsigned)cdiv((long long)Kp * Cn, 256), 256, 0, stream>>>(W[l], Wt[l], grad, Kp, Cn, ldc,
                                                                                ld[l - 1], ctl);
+    }
+    Scope sc(this, "axpy_h", 1, 48.0 * n4, 0.0);
     gk::k_axpy_ctl<<<grid_for(n4), 256, 0, stream>>>((float4*)H[l], (const float4*)B1, n4, ctl);   // H_l at W^{k+1}
     CU(cudaGetLastError());
   }
@@ -238,13 +316,19 @@ struct gcn_admm {
     CU(cudaMemsetAsync(sums_z, 0, sizeof(double) * 3 * M, stream));
     CU(cudaMemsetAsync(n_active, 0, sizeof(int), stream));
     const int rows_per_block = 32;
+    {
+    Scope sc(this, "zgrad_finish", 1, 16.0 * 4.0 * (double)n * (ldl / 4), 0.0);
     gk::k_zgrad_finish<<<(unsigned)cdiv(n, rows_per_block), 256, 0, stream>>>(
         (float4*)B2, (const float4*)Z[l], (const float4*)H[l], ldl / 4, n, rows_per_block, d_row_comm, p.nu, sums_z);
+    }
     const bool out = (l + 1 == L);
     const int per = out ? 2 : gk::kCand;
-    gk::k_search_begin<<<(unsigned)cdiv(M, 128), 128, 0, stream>>>(ctl, M, sums_z, 3, p.bt_shrink, p.bt_growth, acc_z,
-                                                                   per, n_active);
-    CU(cudaGetLastError());
+    {
+      Scope sc(this, "small", 1, 0.0, 0.0);
+      gk::k_search_begin<<<(unsigned)cdiv(M, 128), 128, 0, stream>>>(ctl, M, sums_z, 3, p.bt_shrink, p.bt_growth, acc_z,
+                                                                     per, n_active);
+      CU(cudaGetLastError());
+    }
     gemm_nn(B2, ldl, W[l + 1], ldn, B1, ldn, n, C[l + 1], C[l]);         // T = G W_{l+1}
     gk::DecideArgs a{};
     a.growth = p.bt_growth;
@@ -267,19 +351,33 @@ struct gcn_admm {
     else if (ld4 <= 128) SCORE_Z(4, OUT);   \
     else SCORE_Z(8, OUT);                   \
   }
+    char zname[48];
+    std::snprintf(zname, sizeof zname, out ? "score_z_out@%d" : "score_z_hidden@%d", ldn);
+    const std::string zretry = std::string(zname) + ".retry";
+    const double zbytes = 4.0 * gi.nnz + 8.0 * (double)gi.seg_comm.size() + 8.0 * n +
+                          4.0 * (double)n * ldn * (out ? 2 : 3);
     if (out) {
-      SCORE_Z_ANY(true)
+      {
+        Scope sc(this, zname, 1, zbytes, 2.0 * (double)gi.nnz * ldn);
+        SCORE_Z_ANY(true)
+      }
       a.mode = 1;
       a.quad_coef = 0.5 * p.rho;
       a.last_pass = 1;
+      Scope sc(this, "small", 1, 0.0, 0.0);
       gk::k_search_decide<<<(unsigned)cdiv(M, 128), 128, 0, stream>>>(ctl, M, acc_z, per, sums_z, 3, a, n_active, status);
     } else {
       a.mode = 0;
       a.scale = 0.5 * p.nu;
       const int passes = n_passes();
       for (int ps = 0; ps < passes; ++ps) {
-        SCORE_Z_ANY(false)
+        {   // later passes touch only the segments of communities still searching
+          Scope sc(this, ps == 0 ? zname : zretry.c_str(), 1, ps == 0 ? zbytes : 0.0,
+                   ps == 0 ? 2.0 * (double)gi.nnz * ldn : 0.0);
+          SCORE_Z_ANY(false)
+        }
         a.last_pass = (ps == passes - 1);
+        Scope sc(this, "small", 1, 0.0, 0.0);
         gk::k_search_decide<<<(unsigned)cdiv(M, 128), 128, 0, stream>>>(ctl, M, acc_z, per, sums_z, 3, a, n_active,
                                                                         status);
       }
@@ -287,8 +385,12 @@ struct gcn_admm {
 #undef SCORE_Z_ANY
 #undef SCORE_Z
     CU(cudaGetLastError());
-    gk::k_log_decisions<<<(unsigned)cdiv(M, 128), 128, 0, stream>>>(ctl, M, log_slot_trial_z() + (size_t)(l - 1) * M,
+    {
+      Scope sc(this, "small", 1, 0.0, 0.0);
+      gk::k_log_decisions<<<(unsigned)cdiv(M, 128), 128, 0, stream>>>(ctl, M, log_slot_trial_z() + (size_t)(l - 1) * M,
                                                                     log_slot_q_z() + (size_t)(l - 1) * M);
+    }
+    Scope sc(this, "apply_z", 1, 12.0 * (double)n * ldl, 0.0);
     gk::k_apply_z<<<grid_for(n * (ldl / 4)), 256, 0, stream>>>((float4*)Z[l], (const float4*)B2, ldl / 4, n, d_row_comm, ctl);
     CU(cudaGetLastError());
   }
@@ -296,6 +398,7 @@ struct gcn_admm {
   // ---- Z_L (Eq. 7) and, in the same sweep, the dual as printed in Eq. 3 -----------------
   void update_output(bool dual_now, bool update_z) {
     const int warps = 8;
+    Scope sc(this, "output_rows", 1, 4.0 * (double)n * ld[L] * (3 + (update_z ? 1 : 0) + (dual_now ? 1 : 0)), 0.0);
     gk::k_output_rows<<<(unsigned)cdiv(n, warps), warps * 32, 0, stream>>>(Z[L], U, H[L], ld[L], C[L], (int)n, d_y, d_train,
                                                                            p.rho, p.loss_scale, p.fista_iters,
                                                                            dual_now ? 1 : 0, update_z ? 1 : 0);
@@ -304,6 +407,7 @@ struct gcn_admm {
 
   void dual_from_stored() {   // U + rho (Z_L - H_L) with H_L = A~ Z_{L-1} W_L of the stored iterates
     const long long n4 = n * ld[L] / 4;
+    Scope sc(this, "dual", 1, 64.0 * n4, 0.0);
     gk::k_dual<<<grid_for(n4), 256, 0, stream>>>((float4*)U, (const float4*)Z[L], (const float4*)H[L], n4, p.rho);
     CU(cudaGetLastError());
   }
@@ -331,6 +435,7 @@ struct gcn_admm {
     gemm_nn(P[1], ld[0], W[1], ld[1], B0, ld[1], n, C[1], C[0]);
     for (int l = 1; l < L; ++l) {
       const long long n4 = n * ld[l] / 4;
+      Scope sc(this, "relu", 1, 32.0 * n4, 0.0);
       gk::k_relu_inplace<<<grid_for(n4), 256, 0, stream>>>((float4*)B0, n4);
       CU(cudaGetLastError());
       spmm(B0, B1, ld[l]);
@@ -351,6 +456,7 @@ struct gcn_admm {
   // rows in the caller's order (dense, width c) <-> internal (community order, padded)
   void rows_to_host(const float* dev, int c, float* host_out) {
     float* dense = B2;
+    Scope sc(this, "permute_rows", 1, 8.0 * (double)n * c, 0.0);
     gk::k_permute_rows<<<grid_for(n * ldpad(c)), 256, 0, stream>>>(dev, dense, d_perm, n, c, ldpad(c), 0);
     CU(cudaGetLastError());
     CU(cudaMemcpyAsync(host_out, dense, sizeof(float) * n * c, cudaMemcpyDeviceToHost, stream));
@@ -359,6 +465,7 @@ struct gcn_admm {
   void rows_from_host(const float* host_in, int c, float* dev) {
     float* dense = B2;
     CU(cudaMemcpyAsync(dense, host_in, sizeof(float) * n * c, cudaMemcpyHostToDevice, stream));
+    Scope sc(this, "permute_rows", 1, 8.0 * (double)n * c, 0.0);
     gk::k_permute_rows<<<grid_for(n * ldpad(c)), 256, 0, stream>>>(dense, dev, d_perm, n, c, ldpad(c), 1);
     CU(cudaGetLastError());
     CU(cudaStreamSynchronize(stream));
@@ -537,6 +644,7 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
     float* x_pad = nullptr;
     try {
       x_pad = dalloc<float>(rows * h->ld[0]);
+      gcn_admm::Scope sc(h, "permute_rows", 1, 8.0 * (double)n * h->C[0], 0.0);
       gk::k_permute_rows<<<h->grid_for(n * h->ld[0]), 256, 0, h->stream>>>(on_device ? X : dense, x_pad, h->d_perm, n,
                                                                            h->C[0], h->ld[0], 1);
       CU(cudaGetLastError());
@@ -561,6 +669,7 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
     CU(cudaMemcpyAsync(h->Z[l], h->H[l], bytes, cudaMemcpyDeviceToDevice, h->stream));
     if (l < L) {
       const long long n4 = n * h->ld[l] / 4;
+      gcn_admm::Scope sc(h, "relu", 1, 32.0 * n4, 0.0);
       gk::k_relu_inplace<<<h->grid_for(n4), 256, 0, h->stream>>>((float4*)h->Z[l], n4);
       CU(cudaGetLastError());
     }
@@ -632,6 +741,8 @@ void gcn_admm_destroy(gcn_admm* h) {
   if (!h) return;
   if (cudaSetDevice(h->p.device) == cudaSuccess) {
     cudaStreamSynchronize(h->stream);
+    h->collect_profile();
+    for (cudaEvent_t e : h->event_pool) cudaEventDestroy(e);
     for (void* q : h->owned) cudaFree(q);
   }
   cudaGetLastError();
@@ -680,9 +791,11 @@ int gcn_admm_objective(gcn_admm* h, double out[6]) {
     CU(cudaMemsetAsync(h->obj, 0, 8 * sizeof(double), s));
     for (int l = 1; l < L; ++l) {
       const long long n4 = h->n * h->ld[l] / 4;
+      gcn_admm::Scope sc(h, "objective_sums", 1, 32.0 * n4, 0.0);
       gk::k_sum_hidden_penalty<<<h->grid_for(n4), 256, 0, s>>>((const float4*)h->Z[l], (const float4*)h->H[l], n4, h->obj + 2);
     }
     const long long n4 = h->n * h->ld[L] / 4;
+    gcn_admm::Scope sc_obj(h, "objective_sums", 3, 48.0 * n4, 0.0);
     gk::k_sum_constraint<<<h->grid_for(n4), 256, 0, s>>>((const float4*)h->Z[L], (const float4*)h->H[L],
                                                         (const float4*)h->U, n4, h->obj + 3);
     const int warps = 8;
@@ -719,6 +832,7 @@ int gcn_admm_predict(gcn_admm* h, float* logits, int* labels) {
       const int warps = 8;
       int* d_lab = reinterpret_cast<int*>(h->B1);
       CU(cudaMemsetAsync(h->obj, 0, 8 * sizeof(double), h->stream));
+      gcn_admm::Scope sc(h, "row_argmax", 1, 4.0 * (double)h->n * h->ld[L], 0.0);
       gk::k_row_loss_argmax<<<(unsigned)cdiv(h->n, warps), warps * 32, 0, h->stream>>>(
           nullptr, h->B0, h->ld[L], h->C[L], (int)h->n, h->d_y, h->d_train, d_lab, h->obj);
       CU(cudaGetLastError());
@@ -746,6 +860,7 @@ int gcn_admm_propagate(gcn_admm* h, const float* x, int width, float* out) {
       b = dalloc<float>(rows * ldw);
       CU(cudaMemcpyAsync(dense, x, rows * width * sizeof(float), dev_in ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice,
                          h->stream));
+      gcn_admm::Scope sc(h, "permute_rows", 2, 16.0 * (double)h->n * width, 0.0);
       gk::k_permute_rows<<<h->grid_for(h->n * ldw), 256, 0, h->stream>>>(dense, a, h->d_perm, h->n, width, ldw, 1);
       CU(cudaGetLastError());
       h->spmm(a, b, ldw);
@@ -864,6 +979,40 @@ int gcn_admm_set_state(gcn_admm* h, int which, int layer, const void* in) {
     } else {
       throw Fail{GCN_ADMM_ERR_ARG, "unknown state selector"};
     }
+  });
+}
+
+int gcn_admm_launches(gcn_admm* h, long long* count) {
+  return guarded(h, [&] {
+    if (!count) throw Fail{GCN_ADMM_ERR_ARG, "NULL output"};
+    *count = h->launches;
+  });
+}
+
+int gcn_admm_profile(gcn_admm* h, int enable) {
+  return guarded(h, [&] {
+    h->collect_profile();
+    if (enable) h->prof.clear();
+    h->profiling = enable != 0;
+  });
+}
+
+int gcn_admm_profile_read(gcn_admm* h, int max_entries, int* n_entries, char* names, long long* launches, double* ms,
+                          double* bytes, double* flops) {
+  return guarded(h, [&] {
+    if (!n_entries || max_entries < 0) throw Fail{GCN_ADMM_ERR_ARG, "bad argument"};
+    h->collect_profile();
+    int k = 0;
+    for (const auto& kv : h->prof) {
+      if (k >= max_entries) break;
+      if (names) { std::strncpy(names + (size_t)k * 48, kv.first.c_str(), 47); names[(size_t)k * 48 + 47] = 0; }
+      if (launches) launches[k] = kv.second.launches;
+      if (ms) ms[k] = kv.second.ms;
+      if (bytes) bytes[k] = kv.second.bytes;
+      if (flops) flops[k] = kv.second.flops;
+      ++k;
+    }
+    *n_entries = k;
   });
 }
 

@@ -26,7 +26,7 @@ Recipe, per config index c (seed = BASE_SEED + c, numpy PCG64 streams):
   dropped.  Node ids are then shuffled so that blocks are not contiguous.
 * ADMM communities: the planted blocks when M equals their number, otherwise
   nodes sorted by (block, breadth-first position from the highest-degree node)
-  and cut into M contiguous chunks of ceil(N/M) nodes.
+  and cut into M contiguous, equally sized chunks (node of rank r goes to chunk floor(r M / N)).
 * Initial weights: Glorot-uniform.
 """
 
@@ -147,9 +147,8 @@ def _communities(n, row_ptr, col_idx, block, n_blocks, n_comm):
     rest = np.flatnonzero(pos == n)
     pos[rest] = bfs.shape[0] + np.arange(rest.shape[0])
     order = np.lexsort((pos, block))
-    chunk = -(-n // n_comm)
     community = np.empty(n, dtype=np.int32)
-    community[order] = (np.arange(n) // chunk).astype(np.int32)
+    community[order] = (np.arange(n, dtype=np.int64) * n_comm // n).astype(np.int32)
     return community
 
 
