@@ -125,8 +125,9 @@ struct gcn_admm {
   std::vector<void*> owned;  // every device allocation, for destroy
 
   int *d_row_ptr = nullptr, *d_col = nullptr, *d_row_comm = nullptr, *d_perm = nullptr;
-  int *d_seg_row_ptr = nullptr, *d_seg_comm = nullptr, *d_seg_begin = nullptr, *d_y = nullptr;
+  int* d_y = nullptr;
   float* d_dinv = nullptr;
+  unsigned short* d_col_comm = nullptr;   // community of every stored column
   unsigned char* d_train = nullptr;
 
   std::vector<float*> W, Wt, Z, P, H;   // 1..L
@@ -336,25 +337,31 @@ struct gcn_admm {
     a.own_nu = p.nu;
     const int ld4 = ldn / 4;
     const int warps = 8;
-    const unsigned grid = (unsigned)cdiv(n, warps);
-    const size_t smem = (size_t)M * per * sizeof(double);
-    const int use_smem = smem <= 40 * 1024;
+    const size_t smem = (size_t)warps * M * per * sizeof(double);
+    const int use_smem = smem <= 96 * 1024;
     const size_t dyn = use_smem ? smem : 0;
 #define SCORE_Z(V, OUT)                                                                                   \
-  gk::k_score_z<V, OUT><<<grid, warps * 32, dyn, stream>>>(d_col, d_dinv, d_seg_row_ptr, d_seg_comm, d_seg_begin, \
-      (const float4*)B1, (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0, ld4, (int)n, ctl, M, \
-      acc_z, n_active, use_smem)
+  {                                                                                                       \
+    if (dyn > 48 * 1024)                                                                                  \
+      CU(cudaFuncSetAttribute(gk::k_score_z<V, OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn)); \
+    int occ = 1;                                                                                          \
+    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gk::k_score_z<V, OUT>, warps * 32, dyn));      \
+    const unsigned grid = (unsigned)std::min<long long>(cdiv(n, warps), (long long)kSmCount * std::max(occ, 1)); \
+    gk::k_score_z<V, OUT><<<grid, warps * 32, dyn, stream>>>(d_row_ptr, d_col, d_col_comm, d_dinv,        \
+        (const float4*)B1, (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0, ld4, (int)n, ctl, M, \
+        acc_z, n_active, use_smem);                                                                       \
+  }
 #define SCORE_Z_ANY(OUT)                    \
   {                                         \
-    if (ld4 <= 32) SCORE_Z(1, OUT);         \
-    else if (ld4 <= 64) SCORE_Z(2, OUT);    \
-    else if (ld4 <= 128) SCORE_Z(4, OUT);   \
-    else SCORE_Z(8, OUT);                   \
+    if (ld4 <= 32) SCORE_Z(1, OUT)          \
+    else if (ld4 <= 64) SCORE_Z(2, OUT)     \
+    else if (ld4 <= 128) SCORE_Z(4, OUT)    \
+    else SCORE_Z(8, OUT)                    \
   }
     char zname[48];
     std::snprintf(zname, sizeof zname, out ? "score_z_out@%d" : "score_z_hidden@%d", ldn);
     const std::string zretry = std::string(zname) + ".retry";
-    const double zbytes = 4.0 * gi.nnz + 8.0 * (double)gi.seg_comm.size() + 8.0 * n +
+    const double zbytes = 6.0 * gi.nnz + 8.0 * n +
                           4.0 * (double)n * ldn * (out ? 2 : 3);
     if (out) {
       {
@@ -574,10 +581,12 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
   h->d_col = upload(h, g.col);
   h->d_row_comm = upload(h, g.row_comm);
   h->d_perm = upload(h, g.perm);
-  h->d_seg_row_ptr = upload(h, g.seg_row_ptr);
-  h->d_seg_comm = upload(h, g.seg_comm);
-  h->d_seg_begin = upload(h, g.seg_begin);
   h->d_dinv = upload(h, g.dinv);
+  {
+    std::vector<unsigned short> cc(g.col.size());
+    for (size_t e = 0; e < cc.size(); ++e) cc[e] = (unsigned short)g.row_comm[g.col[e]];
+    h->d_col_comm = upload(h, cc);
+  }
   h->d_y = upload(h, y_new);
   h->d_train = upload(h, t_new);
 
@@ -706,6 +715,7 @@ int gcn_admm_create(gcn_admm** out, long long n, const long long* row_ptr, const
     return GCN_ADMM_ERR_ARG;
   }
   if (n < 1 || n > 2147483647LL / 2 || n_comm < 1) { g_create_error = "n and n_comm must be positive"; return GCN_ADMM_ERR_ARG; }
+  if (n_comm > 65535) { g_create_error = "more than 65535 communities are not supported"; return GCN_ADMM_ERR_COMMUNITY; }
   if (n_layers < 1 || n_layers > 64) { g_create_error = "n_layers must be 1..64"; return GCN_ADMM_ERR_WIDTHS; }
   if (!p->w_init) { g_create_error = "w_init is required"; return GCN_ADMM_ERR_ARG; }
   for (int l = 0; l < n_layers; ++l)

@@ -697,35 +697,59 @@ k_zgrad_finish(float4* __restrict__ G, const float4* __restrict__ Z, const float
   }
 }
 
+// Warp-wide sums of 4 (or 2) per-lane values with 6 (5) shuffles: lane 8*j (16*j) ends up holding
+// the total of value j.
+__device__ __forceinline__ float warp_sum4(float v0, float v1, float v2, float v3, int lane) {
+  const bool up16 = lane & 16, up8 = lane & 8;
+  const float r0 = __shfl_xor_sync(0xffffffffu, up16 ? v0 : v2, 16);
+  const float r1 = __shfl_xor_sync(0xffffffffu, up16 ? v1 : v3, 16);
+  const float a = (up16 ? v2 : v0) + r0, b = (up16 ? v3 : v1) + r1;
+  float c = (up8 ? b : a) + __shfl_xor_sync(0xffffffffu, up8 ? a : b, 8);
+  c += __shfl_xor_sync(0xffffffffu, c, 4);
+  c += __shfl_xor_sync(0xffffffffu, c, 2);
+  c += __shfl_xor_sync(0xffffffffu, c, 1);
+  return c;
+}
+__device__ __forceinline__ float warp_sum2(float v0, float v1, int lane) {
+  const bool up16 = lane & 16;
+  float c = (up16 ? v1 : v0) + __shfl_xor_sync(0xffffffffu, up16 ? v0 : v1, 16);
+  c += __shfl_xor_sync(0xffffffffu, c, 8);
+  c += __shfl_xor_sync(0xffffffffu, c, 4);
+  c += __shfl_xor_sync(0xffffffffu, c, 2);
+  c += __shfl_xor_sync(0xffffffffu, c, 1);
+  return c;
+}
+
 // Scoring of the theta candidates of every community in one sweep over the rows.
 // With T = G W_{l+1}, the move of community m changes the pre-activation of row i by
 //   -K_m[i] / theta_m ,  K_m[i] = sum over j in V_m of A~_ij T_j  (row i of A~_{comm(i),m} T_m),
-// which is non-zero on V_m and its first-order neighbour rows only.  A warp owns row i, walks the
-// segments of the row (one per neighbouring community), forms K_m[i] and scores it.
+// which is non-zero on V_m and its first-order neighbour rows only.  A warp owns row i and walks
+// its stored entries once; col_comm gives the community of every entry, entries of one community
+// are contiguous (ascending columns), and at every change of community the finished K_m[i] is scored:
 //   OUT = false (layer l+1 < L, ReLU):  acc[m*kCand + j] += sum_c (z - f(h - k/t_j))^2 - (z - f(h))^2
 //   OUT = true  (layer l+1 = L):        acc[m*2] += <k, R'>, acc[m*2+1] += ||k||^2   (closed form)
-// V = float4 columns per lane (width <= 128 V).
+// Sums are kept per warp in shared memory (no atomics on the hot path) and added to `acc` once per
+// block; with too many communities for that (use_smem == 0) they go to `acc` directly.
+// V = float4 columns per lane (width <= 128 V).  Persistent grid: rows are dealt to blocks round robin.
 template <int V, bool OUT>
 __global__ void __launch_bounds__(256)
-k_score_z(const int* __restrict__ col, const float* __restrict__ dinv,
-          const int* __restrict__ seg_row_ptr, const int* __restrict__ seg_comm,
-          const int* __restrict__ seg_begin, const float4* __restrict__ T, const float4* __restrict__ Hn,
-          const float4* __restrict__ Zn, const float4* __restrict__ Rn, int ld4, int n,
-          const SearchCtl* __restrict__ ctl, int n_comm, double* __restrict__ acc,
-          const int* __restrict__ n_active, int use_smem) {
+k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
+          const unsigned short* __restrict__ col_comm, const float* __restrict__ dinv,
+          const float4* __restrict__ T, const float4* __restrict__ Hn, const float4* __restrict__ Zn,
+          const float4* __restrict__ Rn, int ld4, int n, const SearchCtl* __restrict__ ctl, int n_comm,
+          double* __restrict__ acc, const int* __restrict__ n_active, int use_smem) {
   if (*n_active <= 0) return;
   constexpr int PER = OUT ? 2 : kCand;
   extern __shared__ double s_acc[];
-  double* accp = acc;
-  if (use_smem) {
-    for (int i = threadIdx.x; i < n_comm * PER; i += blockDim.x) s_acc[i] = 0.0;
-    __syncthreads();
-    accp = s_acc;
-  }
-  const int lane = threadIdx.x & 31;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int warps_per_block = blockDim.x >> 5;
-  const int row = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
-  if (row < n) {
+  double* mine = acc;
+  if (use_smem) {
+    for (int i = threadIdx.x; i < warps_per_block * n_comm * PER; i += blockDim.x) s_acc[i] = 0.0;
+    __syncthreads();
+    mine = s_acc + (size_t)warp * n_comm * PER;
+  }
+  for (int row = blockIdx.x * warps_per_block + warp; row < n; row += gridDim.x * warps_per_block) {
     float4 a[V], b[V];   // OUT: a = R' ; else a = h, b = z
 #pragma unroll
     for (int v = 0; v < V; ++v) {
@@ -737,45 +761,14 @@ k_score_z(const int* __restrict__ col, const float* __restrict__ dinv,
       }
     }
     const float di = dinv[row];
-    const int s0 = seg_row_ptr[row], s1 = seg_row_ptr[row + 1];
-    for (int s = s0; s < s1; ++s) {
-      const int m = seg_comm[s];
-      if (ctl[m].done) continue;
-      const int pb = seg_begin[s], pe = seg_begin[s + 1];
-      float4 k[V];
+    float4 k[V];
 #pragma unroll
-      for (int v = 0; v < V; ++v) k[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int base = pb; base < pe; base += 32) {
-        const int idx = base + lane;
-        int c = 0;
-        float w = 0.f;
-        if (idx < pe) { c = col[idx]; w = dinv[c]; }
-        const int cnt = min(32, pe - base);
-        for (int t = 0; t < cnt; t += 4) {
-          int cj[4];
-          float wj[4];
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            cj[u] = __shfl_sync(0xffffffffu, c, (t + u) & 31);
-            wj[u] = __shfl_sync(0xffffffffu, w, (t + u) & 31);
-            if (t + u >= 32) wj[u] = 0.f;
-          }
-#pragma unroll
-          for (int v = 0; v < V; ++v) {
-            const int f = lane + 32 * v;
-            if (f < ld4) {
-              float4 xv[4];
-#pragma unroll
-              for (int u = 0; u < 4; ++u) xv[u] = __ldg(T + (long long)cj[u] * ld4 + f);
-#pragma unroll
-              for (int u = 0; u < 4; ++u) {
-                k[v].x = fmaf(wj[u], xv[u].x, k[v].x); k[v].y = fmaf(wj[u], xv[u].y, k[v].y);
-                k[v].z = fmaf(wj[u], xv[u].z, k[v].z); k[v].w = fmaf(wj[u], xv[u].w, k[v].w);
-              }
-            }
-          }
-        }
-      }
+    for (int v = 0; v < V; ++v) k[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    int cur = -1;          // community of the segment being accumulated
+    bool cur_on = false;   // its search is still running
+
+    auto finish_segment = [&]() {
+      if (!cur_on) return;
       if (OUT) {
         float p1 = 0.f, p2 = 0.f;
 #pragma unroll
@@ -784,13 +777,15 @@ k_score_z(const int* __restrict__ col, const float* __restrict__ dinv,
           p1 += kx * a[v].x + ky * a[v].y + kz * a[v].z + kw * a[v].w;
           p2 += kx * kx + ky * ky + kz * kz + kw * kw;
         }
-        p1 = warp_sum(p1);
-        p2 = warp_sum(p2);
-        if (lane == 0) { atomicAdd(accp + m * 2, (double)p1); atomicAdd(accp + m * 2 + 1, (double)p2); }
+        const float r = warp_sum2(p1, p2, lane);
+        if ((lane & 15) == 0) {
+          double* dst = mine + cur * 2 + (lane >> 4);
+          if (use_smem) *dst += (double)r; else atomicAdd(dst, (double)r);
+        }
       } else {
         float inv[kCand], part[kCand];
 #pragma unroll
-        for (int j = 0; j < kCand; ++j) { inv[j] = ctl[m].inv_cand[j]; part[j] = 0.f; }
+        for (int j = 0; j < kCand; ++j) { inv[j] = ctl[cur].inv_cand[j]; part[j] = 0.f; }
 #pragma unroll
         for (int v = 0; v < V; ++v) {
           const float kk[4] = {di * k[v].x, di * k[v].y, di * k[v].z, di * k[v].w};
@@ -807,18 +802,74 @@ k_score_z(const int* __restrict__ col, const float* __restrict__ dinv,
             }
           }
         }
+        static_assert(kCand == 4, "warp_sum4 reduces exactly four candidates");
+        const float r = warp_sum4(part[0], part[1], part[2], part[3], lane);
+        if ((lane & 7) == 0) {
+          double* dst = mine + cur * kCand + (lane >> 3);
+          if (use_smem) *dst += (double)r; else atomicAdd(dst, (double)r);
+        }
+      }
+    };
+
+    const int rs = row_ptr[row], re = row_ptr[row + 1];
+    for (int base = rs; base < re; base += 32) {
+      const int idx = base + lane;
+      int c = 0, m = -1;
+      float w = 0.f;
+      if (idx < re) {
+        c = col[idx];
+        m = col_comm[idx];
+        if (ctl[m].done) m |= 0x10000;     // finished search: keep the community, skip the work
+        else w = dinv[c];
+      }
+      const int cnt = min(32, re - base);
+      for (int t = 0; t < cnt; t += 4) {
+        int cj[4], mj[4];
+        float wj[4];
 #pragma unroll
-        for (int j = 0; j < kCand; ++j) {
-          const float v = warp_sum(part[j]);
-          if (lane == 0) atomicAdd(accp + m * kCand + j, (double)v);
+        for (int u = 0; u < 4; ++u) {
+          cj[u] = __shfl_sync(0xffffffffu, c, (t + u) & 31);
+          mj[u] = __shfl_sync(0xffffffffu, m, (t + u) & 31);
+          wj[u] = __shfl_sync(0xffffffffu, w, (t + u) & 31);
+          if (t + u >= cnt) mj[u] = -1;
+        }
+        float4 xv[4][V];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+          for (int v = 0; v < V; ++v) {
+            const int f = lane + 32 * v;
+            xv[u][v] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (mj[u] >= 0 && mj[u] < 0x10000 && f < ld4) xv[u][v] = __ldg(T + (long long)cj[u] * ld4 + f);
+          }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (mj[u] < 0) continue;                       // past the end of the row (warp-uniform)
+          const int mm = mj[u] & 0xffff;
+          if (mm != cur) {
+            finish_segment();
+            cur = mm;
+            cur_on = mj[u] < 0x10000;
+#pragma unroll
+            for (int v = 0; v < V; ++v) k[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+#pragma unroll
+          for (int v = 0; v < V; ++v) {
+            k[v].x = fmaf(wj[u], xv[u][v].x, k[v].x); k[v].y = fmaf(wj[u], xv[u][v].y, k[v].y);
+            k[v].z = fmaf(wj[u], xv[u][v].z, k[v].z); k[v].w = fmaf(wj[u], xv[u][v].w, k[v].w);
+          }
         }
       }
     }
+    finish_segment();
   }
   if (use_smem) {
     __syncthreads();
-    for (int i = threadIdx.x; i < n_comm * PER; i += blockDim.x)
-      if (s_acc[i] != 0.0) atomicAdd(acc + i, s_acc[i]);
+    for (int i = threadIdx.x; i < n_comm * PER; i += blockDim.x) {
+      double t = 0.0;
+      for (int wq = 0; wq < warps_per_block; ++wq) t += s_acc[(size_t)wq * n_comm * PER + i];
+      if (t != 0.0) atomicAdd(acc + i, t);
+    }
   }
 }
 
