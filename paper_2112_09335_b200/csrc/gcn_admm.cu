@@ -6,6 +6,7 @@
 
 #include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <new>
@@ -165,18 +166,19 @@ struct gcn_admm {
     char name[48];
     std::snprintf(name, sizeof name, "spmm@%d", ldx);
     Scope sc(this, name, 1, 4.0 * gi.nnz + 8.0 * n + 8.0 * (double)n * ldx, 2.0 * (double)gi.nnz * ldx);
-#define SPMM_CASE(G, V)                                                                        \
+    // 64-thread blocks: rows differ widely in length, small blocks keep the SMs evenly loaded
+#define SPMM_CASE(G, V, UN)                                                                    \
   {                                                                                            \
     const long long threads = n * (G);                                                         \
-    gk::k_spmm<G, V><<<(unsigned)cdiv(threads, 256), 256, 0, stream>>>(d_row_ptr, d_col, d_dinv, x4, o4, nn, ld4); \
+    gk::k_spmm<G, V, UN><<<(unsigned)cdiv(threads, 64), 64, 0, stream>>>(d_row_ptr, d_col, d_dinv, x4, o4, nn, ld4); \
   }
-    if (ld4 <= 1) SPMM_CASE(1, 1)
-    else if (ld4 <= 2) SPMM_CASE(2, 1)
-    else if (ld4 <= 4) SPMM_CASE(4, 1)
-    else if (ld4 <= 8) SPMM_CASE(8, 1)
-    else if (ld4 <= 16) SPMM_CASE(16, 1)
-    else if (ld4 <= 32) SPMM_CASE(32, 1)
-    else SPMM_CASE(32, 2)
+    if (ld4 <= 1) SPMM_CASE(1, 1, 4)
+    else if (ld4 <= 2) SPMM_CASE(2, 1, 4)
+    else if (ld4 <= 4) SPMM_CASE(4, 1, 8)
+    else if (ld4 <= 8) SPMM_CASE(8, 1, 8)
+    else if (ld4 <= 16) SPMM_CASE(16, 1, 8)
+    else if (ld4 <= 32) SPMM_CASE(32, 1, 4)
+    else SPMM_CASE(32, 2, 4)
 #undef SPMM_CASE
     CU(cudaGetLastError());
   }

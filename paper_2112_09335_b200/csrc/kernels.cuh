@@ -63,7 +63,7 @@ __device__ __forceinline__ double block_sum(double v, double* sh) {
 // G lanes share one row; each lane owns the float4 columns lane, lane+G, .. of a block of
 // G*V float4 columns; wider rows loop over column blocks.
 // ------------------------------------------------------------------------------------------
-template <int G, int V>
+template <int G, int V, int UN>
 __global__ void __launch_bounds__(256)
 k_spmm(const int* __restrict__ row_ptr, const int* __restrict__ col, const float* __restrict__ dinv,
        const float4* __restrict__ x, float4* __restrict__ out, int n, int ld4) {
@@ -84,11 +84,11 @@ k_spmm(const int* __restrict__ row_ptr, const int* __restrict__ col, const float
       float w = 0.f;
       if (idx < re) { c = col[idx]; w = dinv[c]; }
       const int cnt = min(G, re - base);
-      for (int t = 0; t < cnt; t += 4) {
-        int cj[4];
-        float wj[4];
+      for (int t = 0; t < cnt; t += UN) {
+        int cj[UN];
+        float wj[UN];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {   // lanes past the row's end hold (column 0, weight 0)
+        for (int u = 0; u < UN; ++u) {   // lanes past the row's end hold (column 0, weight 0)
           cj[u] = __shfl_sync(gmask, c, (t + u) & (G - 1), G);
           wj[u] = __shfl_sync(gmask, w, (t + u) & (G - 1), G);
           if (t + u >= G) wj[u] = 0.f;
@@ -97,11 +97,11 @@ k_spmm(const int* __restrict__ row_ptr, const int* __restrict__ col, const float
         for (int v = 0; v < V; ++v) {
           const int f = cb + gl + G * v;
           if (f < ld4) {
-            float4 xv[4];
+            float4 xv[UN];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) xv[u] = __ldg(x + (long long)cj[u] * ld4 + f);
+            for (int u = 0; u < UN; ++u) xv[u] = __ldg(x + (long long)cj[u] * ld4 + f);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < UN; ++u) {
               acc[v].x = fmaf(wj[u], xv[u].x, acc[v].x);
               acc[v].y = fmaf(wj[u], xv[u].y, acc[v].y);
               acc[v].z = fmaf(wj[u], xv[u].z, acc[v].z);
@@ -127,7 +127,7 @@ k_spmm(const int* __restrict__ row_ptr, const int* __restrict__ col, const float
 // fp32 FFMA register tiles; `skip`, when given, points at a flag that cancels the launch.
 // ------------------------------------------------------------------------------------------
 template <int BM, int BN, int BK, int TM, int TN>
-__global__ void __launch_bounds__((BM / TM) * (BN / TN))
+__global__ void __launch_bounds__((BM / TM) * (BN / TN), 2)
 k_gemm_nn(const float* __restrict__ A, int lda, const float* __restrict__ B, int ldb,
           float* __restrict__ C, int ldc, int M, int N, int K, const int* __restrict__ skip) {
   constexpr int NT = (BM / TM) * (BN / TN);
@@ -261,7 +261,7 @@ k_gemm_nn(const float* __restrict__ A, int lda, const float* __restrict__ B, int
 // part[(split * Ka + ka) * ldp + nb].  A: rows x Ka (lda), B: rows x Nb (ldb).
 // Split s owns rows [s * rows_per_split, min(rows, (s+1) * rows_per_split)).
 template <int BM, int BN, int BK, int TM, int TN>
-__global__ void __launch_bounds__((BM / TM) * (BN / TN))
+__global__ void __launch_bounds__((BM / TM) * (BN / TN), 2)
 k_gemm_tn(const float* __restrict__ A, int lda, const float* __restrict__ B, int ldb,
           float* __restrict__ part, int ldp, long long rows, long long rows_per_split, int Ka, int Nb) {
   constexpr int NT = (BM / TM) * (BN / TN);
