@@ -29,6 +29,13 @@ struct SearchCtl {
 
 __device__ __forceinline__ float relu(float x) { return x > 0.f ? x : 0.f; }
 
+// relu(h) - relu(h - s) without forming h - s when both sides are active, so that a step s far
+// below the rounding unit of h still registers exactly.
+__device__ __forceinline__ float relu_drop(float h, float s) {
+  const bool on0 = h > 0.f, on1 = h > s;
+  return on0 ? (on1 ? s : h) : (on1 ? s - h : 0.f);
+}
+
 __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -476,13 +483,11 @@ k_score_w_hidden(const float4* __restrict__ H, const float4* __restrict__ D, con
     for (int j = 0; j < kCand; ++j) part[j] = 0.f;
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
-      const float f0 = relu(h[c]);
-      const float e0 = z[c] - f0;
+      const float e0 = z[c] - relu(h[c]);
 #pragma unroll
       for (int j = 0; j < kCand; ++j) {
-        const float f1 = relu(fmaf(-d[c], inv[j], h[c]));
-        const float e1 = z[c] - f1;
-        part[j] = fmaf(f0 - f1, e1 + e0, part[j]);   // e1^2 - e0^2 = (e1 - e0)(e1 + e0)
+        const float df = relu_drop(h[c], d[c] * inv[j]);
+        part[j] = fmaf(df, fmaf(2.f, e0, df), part[j]);   // e1^2 - e0^2 = (e1 - e0)(e1 + e0), e1 - e0 = df
       }
     }
 #pragma unroll
@@ -793,12 +798,11 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
           const float zz[4] = {b[v].x, b[v].y, b[v].z, b[v].w};
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
-            const float f0 = relu(hh[c]);
-            const float e0 = zz[c] - f0;
+            const float e0 = zz[c] - relu(hh[c]);
 #pragma unroll
             for (int j = 0; j < kCand; ++j) {
-              const float f1 = relu(fmaf(-kk[c], inv[j], hh[c]));
-              part[j] = fmaf(f0 - f1, (zz[c] - f1) + e0, part[j]);
+              const float df = relu_drop(hh[c], kk[c] * inv[j]);
+              part[j] = fmaf(df, fmaf(2.f, e0, df), part[j]);
             }
           }
         }
