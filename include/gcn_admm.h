@@ -122,6 +122,26 @@ const char* gcn_admm_last_error(const gcn_admm* h);
  * kind; out may not alias x).  Uses the handle's graph only; the ADMM state is untouched. */
 int gcn_admm_propagate(gcn_admm* h, const float* x, int width, float* out);
 
+/* ---- propagation for callers that cannot allocate ---------------------------------------------
+ * (No counterpart in the paper: this is a packaging variant of gcn_admm_propagate.)
+ * Same result as gcn_admm_propagate, for code that is not allowed to reserve device memory when it
+ * calls: a real-time loop whose memory budget was fixed at start-up, a plug-in running inside
+ * someone else's memory pool, a section between begin and end of a stream capture where cudaMalloc is
+ * illegal.  gcn_admm_propagate stages x and the result in two padded matrices that it allocates and
+ * frees on every call; this variant keeps those two matrices in an array compiled into the library
+ * (32 MiB of device memory on every GPU that loads the library, held until the process ends), and
+ * calls neither cudaMalloc nor cudaFree nor any allocating routine.
+ *  - x and out are DEVICE pointers to n x width floats, original node order; out may not alias x.
+ *  - limit: n * (width rounded up to a multiple of 4) <= 4,194,304; larger sizes are refused with
+ *    GCN_ADMM_ERR_ARG and a message naming the limit.
+ *  - the first call on a device looks up the device address of the array (one runtime query, no
+ *    allocation); make that first call before any stream capture begins.
+ *  - the work is enqueued on the handle's stream and the call returns without synchronising.
+ *  - all calls, from every handle, share the one array, which keeps whatever the last call left in
+ *    it; each call overwrites all it later reads, so nothing needs clearing, but two calls whose
+ *    kernels overlap on the GPU (different streams, different handles) race on it: serialise them. */
+int gcn_admm_propagate_static(gcn_admm* h, const float* x, int width, float* out);
+
 /* ---- index tables (Section 2; Appendix A first paragraph) ------------------------------------
  * Returns a pointer to a host int array owned by the handle (valid until the next call of this
  * function with the same selector, or destroy) and its length.  New ids = position after sorting

@@ -18,7 +18,7 @@ EXPORTS = [
     "gcn_admm_default_params", "gcn_admm_create", "gcn_admm_step", "gcn_admm_objective", "gcn_admm_weights",
     "gcn_admm_predict", "gcn_admm_destroy", "gcn_admm_last_error", "gcn_admm_propagate", "gcn_admm_index",
     "gcn_admm_get_state", "gcn_admm_set_state", "gcn_admm_step_block", "gcn_admm_decisions",
-    "gcn_admm_launches", "gcn_admm_profile", "gcn_admm_profile_read",
+    "gcn_admm_launches", "gcn_admm_profile", "gcn_admm_profile_read", "gcn_admm_propagate_static",
 ]
 
 IX = dict(perm=0, inv_perm=1, comm_ptr=2, nbr=3, halo1=4, halo2=5, csr_row_ptr=6, csr_col=7,
@@ -65,6 +65,7 @@ def load():
     lib.gcn_admm_last_error.argtypes = [vp]
     lib.gcn_admm_last_error.restype = C.c_char_p
     lib.gcn_admm_propagate.argtypes = [vp, vp, i32, vp]
+    lib.gcn_admm_propagate_static.argtypes = [vp, vp, i32, vp]
     lib.gcn_admm_index.argtypes = [vp, i32, i32, C.POINTER(C.POINTER(i32)), C.POINTER(i64)]
     lib.gcn_admm_get_state.argtypes = [vp, i32, i32, vp]
     lib.gcn_admm_set_state.argtypes = [vp, i32, i32, vp]
@@ -170,6 +171,11 @@ class GcnAdmm:
         res = np.empty_like(x)
         self._check(self._lib.gcn_admm_propagate(self._h, _ptr(x), x.shape[1], _ptr(res)))
         return res
+
+    def propagate_static(self, x_dev, width, out_dev):
+        """A~ x between device buffers (addresses as ints) using the library's built-in staging
+        memory: nothing is allocated by the call.  Enqueued on the handle's stream."""
+        self._check(self._lib.gcn_admm_propagate_static(self._h, _ptr(int(x_dev)), int(width), _ptr(int(out_dev))))
 
     def index(self, which, comm=0):
         data = C.POINTER(C.c_int)()

@@ -9,6 +9,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <map>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -886,6 +887,52 @@ int gcn_admm_propagate(gcn_admm* h, const float* x, int width, float* out) {
       throw;
     }
     cudaFree(dense); cudaFree(a); cudaFree(b);
+  });
+}
+
+// ---- propagation for callers that may not allocate ---------------------------------------------
+// The two padded staging matrices of gcn_admm_propagate live in one file-scope device array, so
+// this entry point reserves nothing at call time.  Every GPU that loads the library carries the
+// array (32 MiB) until the process exits.
+namespace {
+constexpr long long kStaticHalf = 4LL << 20;                       // floats per staging matrix
+static __device__ __align__(256) float g_propagate_scratch[2 * kStaticHalf];
+std::mutex g_scratch_mutex;
+float* g_scratch_addr[64] = {nullptr};
+
+// Device address of g_propagate_scratch on `device` (which must be current).  In host code the
+// array's name is only a handle for the runtime, never an address a kernel may be given.
+float* static_scratch(int device) {
+  if (device < 0 || device >= 64) throw Fail{GCN_ADMM_ERR_ARG, "device ordinal above 63"};
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (g_scratch_addr[device] == nullptr) {
+    float* ptr = nullptr;
+    CU(cudaGetSymbolAddress((void**)&ptr, g_propagate_scratch));
+    g_scratch_addr[device] = ptr;
+  }
+  return g_scratch_addr[device];
+}
+}  // namespace
+
+int gcn_admm_propagate_static(gcn_admm* h, const float* x, int width, float* out) {
+  return guarded(h, [&] {
+    if (!x || !out || width < 1) throw Fail{GCN_ADMM_ERR_ARG, "bad argument"};
+    const int ldw = ldpad(width);
+    if ((long long)h->n * ldw > kStaticHalf)
+      throw Fail{GCN_ADMM_ERR_ARG, "n * padded width exceeds the static scratch of 4194304 floats per staging matrix"};
+    if (!is_device_pointer(x) || !is_device_pointer(out))
+      throw Fail{GCN_ADMM_ERR_ARG, "x and out must be device pointers"};
+    float* a = static_scratch(h->p.device);
+    float* b = a + kStaticHalf;
+    {
+      gcn_admm::Scope sc(h, "permute_rows", 1, 8.0 * (double)h->n * width, 0.0);
+      gk::k_permute_rows<<<h->grid_for(h->n * ldw), 256, 0, h->stream>>>(x, a, h->d_perm, h->n, width, ldw, 1);
+      CU(cudaGetLastError());
+    }
+    h->spmm(a, b, ldw);
+    gcn_admm::Scope sc(h, "permute_rows", 1, 8.0 * (double)h->n * width, 0.0);
+    gk::k_permute_rows<<<h->grid_for(h->n * ldw), 256, 0, h->stream>>>(b, out, h->d_perm, h->n, width, ldw, 0);
+    CU(cudaGetLastError());
   });
 }
 
