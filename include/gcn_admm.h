@@ -54,6 +54,9 @@ enum {
  *                  1/(loss_scale/2 + rho), t_1 = 1, warm start, no early exit)
  *  loss_scale      R = loss_scale * sum over training rows of the softmax cross-entropy
  *  dual_mode       0: Eq. 3 as printed (Z_L^k, Z_{L-1}^k, W_L^{k+1}); 1: the k+1 iterates
+ *  tensor_cores    1: dense products with at most 256 output columns and K <= 512 run on the tensor
+ *                  cores as an error-compensated TF32 product (three passes, fp32 accumulation,
+ *                  relative error of a few 1e-7 of sum |a||b|); 0: fp32 FMA kernels everywhere
  *  w_init          L host pointers to row-major C_{l-1} x C_l matrices (required)
  *  device          CUDA device ordinal;  stream: a cudaStream_t owned by the caller (NULL = the
  *                  default stream) */
@@ -65,13 +68,15 @@ typedef struct {
   int fista_iters;
   float loss_scale;
   int dual_mode;
+  int tensor_cores;
   const float* const* w_init;
   int device;
   void* stream;
 } gcn_admm_params;
 
 /* Fills *p with the defaults: nu = rho = 1e-3, tau0 = theta0 = 1, growth 2, shrink 0.5,
- * 40 trials, 30 FISTA iterations, loss_scale 1, dual_mode 0, device 0, stream NULL, w_init NULL. */
+ * 40 trials, 30 FISTA iterations, loss_scale 1, dual_mode 0, tensor_cores 1, device 0, stream NULL,
+ * w_init NULL. */
 void gcn_admm_default_params(gcn_admm_params* p);
 
 /* Builds the problem of Algorithm 1 (its REQUIRE line) on the device.
@@ -121,6 +126,12 @@ const char* gcn_admm_last_error(const gcn_admm* h);
  * out = A~ x for an n x width matrix x in the original node order (host or device, both the same
  * kind; out may not alias x).  Uses the handle's graph only; the ADMM state is untouched. */
 int gcn_admm_propagate(gcn_admm* h, const float* x, int width, float* out);
+
+/* ---- the dense product alone (the contraction with W_l in Problem 1 and in every block update) ----
+ * C = A B for device pointers A (m x k), B (k x n), C (m x n), dense row-major; tensor_cores selects
+ * the kernel as the parameter of the same name does.  Allocates staging copies; synchronises. */
+int gcn_admm_dense_product(gcn_admm* h, const float* A, const float* B, float* C, long long m, int n, int k,
+                           int tensor_cores);
 
 /* ---- propagation for callers that cannot allocate ---------------------------------------------
  * (No counterpart in the paper: this is a packaging variant of gcn_admm_propagate.)

@@ -18,7 +18,7 @@ EXPORTS = [
     "gcn_admm_default_params", "gcn_admm_create", "gcn_admm_step", "gcn_admm_objective", "gcn_admm_weights",
     "gcn_admm_predict", "gcn_admm_destroy", "gcn_admm_last_error", "gcn_admm_propagate", "gcn_admm_index",
     "gcn_admm_get_state", "gcn_admm_set_state", "gcn_admm_step_block", "gcn_admm_decisions",
-    "gcn_admm_launches", "gcn_admm_profile", "gcn_admm_profile_read", "gcn_admm_propagate_static",
+    "gcn_admm_launches", "gcn_admm_profile", "gcn_admm_profile_read", "gcn_admm_propagate_static", "gcn_admm_dense_product",
 ]
 
 IX = dict(perm=0, inv_perm=1, comm_ptr=2, nbr=3, halo1=4, halo2=5, csr_row_ptr=6, csr_col=7,
@@ -30,7 +30,7 @@ PHASE_W, PHASE_Z, PHASE_U = range(3)
 class Params(C.Structure):
     _fields_ = [("nu", C.c_float), ("rho", C.c_float), ("tau0", C.c_float), ("theta0", C.c_float),
                 ("bt_growth", C.c_float), ("bt_shrink", C.c_float), ("bt_max_trials", C.c_int),
-                ("fista_iters", C.c_int), ("loss_scale", C.c_float), ("dual_mode", C.c_int),
+                ("fista_iters", C.c_int), ("loss_scale", C.c_float), ("dual_mode", C.c_int), ("tensor_cores", C.c_int),
                 ("w_init", C.POINTER(C.POINTER(C.c_float))), ("device", C.c_int), ("stream", C.c_void_p)]
 
 
@@ -66,6 +66,7 @@ def load():
     lib.gcn_admm_last_error.restype = C.c_char_p
     lib.gcn_admm_propagate.argtypes = [vp, vp, i32, vp]
     lib.gcn_admm_propagate_static.argtypes = [vp, vp, i32, vp]
+    lib.gcn_admm_dense_product.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32]
     lib.gcn_admm_index.argtypes = [vp, i32, i32, C.POINTER(C.POINTER(i32)), C.POINTER(i64)]
     lib.gcn_admm_get_state.argtypes = [vp, i32, i32, vp]
     lib.gcn_admm_set_state.argtypes = [vp, i32, i32, vp]
@@ -99,7 +100,7 @@ class GcnAdmm:
 
     def __init__(self, n, row_ptr, col_idx, X, y, train_mask, widths, n_comm, community, w_init, nu=1e-3, rho=1e-3,
                  tau0=1.0, theta0=1.0, bt_growth=2.0, bt_shrink=0.5, bt_max_trials=40, fista_iters=30,
-                 loss_scale=1.0, dual_mode=0, device=0, stream=0):
+                 loss_scale=1.0, dual_mode=0, tensor_cores=1, device=0, stream=0):
         lib = load()
         self._lib = lib
         self._h = C.c_void_p()
@@ -109,6 +110,7 @@ class GcnAdmm:
         p.nu, p.rho, p.tau0, p.theta0 = nu, rho, tau0, theta0
         p.bt_growth, p.bt_shrink, p.bt_max_trials = bt_growth, bt_shrink, bt_max_trials
         p.fista_iters, p.loss_scale, p.dual_mode = fista_iters, loss_scale, dual_mode
+        p.tensor_cores = int(tensor_cores)
         p.device, p.stream = device, stream or None
         ws = [np.ascontiguousarray(w, dtype=np.float32) for w in w_init]
         arr = (C.POINTER(C.c_float) * len(ws))(*[w.ctypes.data_as(C.POINTER(C.c_float)) for w in ws])
@@ -176,6 +178,11 @@ class GcnAdmm:
         """A~ x between device buffers (addresses as ints) using the library's built-in staging
         memory: nothing is allocated by the call.  Enqueued on the handle's stream."""
         self._check(self._lib.gcn_admm_propagate_static(self._h, _ptr(int(x_dev)), int(width), _ptr(int(out_dev))))
+
+    def dense_product(self, a_dev, b_dev, c_dev, m, n, k, tensor_cores=1):
+        """C = A B between dense device buffers (addresses as ints)."""
+        self._check(self._lib.gcn_admm_dense_product(self._h, _ptr(int(a_dev)), _ptr(int(b_dev)), _ptr(int(c_dev)), int(m),
+                                                     int(n), int(k), int(tensor_cores)))
 
     def index(self, which, comm=0):
         data = C.POINTER(C.c_int)()

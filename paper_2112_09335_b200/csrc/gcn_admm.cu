@@ -14,6 +14,7 @@
 #include <string>
 #include <vector>
 
+#include "gemm_tc.cuh"
 #include "graph_index.hpp"
 #include "kernels.cuh"
 
@@ -136,6 +137,8 @@ struct gcn_admm {
   float* U = nullptr;
   float *B0 = nullptr, *B1 = nullptr, *B2 = nullptr;   // N x max_ld scratch
   float* grad = nullptr;     // max over l of C_{l-1} x ld_l
+  float* grad_t = nullptr;   // its transpose, C_l x ld_{l-1} (K-major operand of the tensor-core product)
+  int* tc_error = nullptr;   // raised by a tensor-core product whose bounded wait ran out
   float* part = nullptr;     // split partial sums of the transposed product
   size_t part_elems = 0;
   SearchCtl *ctl_w = nullptr, *ctl_z = nullptr;   // [L+1], [(L+1) * M]
@@ -184,9 +187,34 @@ struct gcn_admm {
     CU(cudaGetLastError());
   }
 
-  void gemm_nn(const float* A, int lda, const float* B, int ldb, float* Cm, int ldc, long long Mr, int N, int K,
-               const int* skip = nullptr) {
+  // C = A B.  B is handed over twice: row-major K x N (ldb) for the fp32-ALU kernels and K-major
+  // N x K (Bk, ldbk; may be NULL) for the tensor-core kernel, which is used whenever it applies
+  // (at most 256 output columns; K capped because its accumulator error grows with K).
+  void gemm_nn(const float* A, int lda, const float* B, int ldb, const float* Bk, int ldbk, float* Cm, int ldc,
+               long long Mr, int N, int K, const int* skip = nullptr) {
     char name[48];
+    if (p.tensor_cores && Bk != nullptr && N <= 256 && K >= 8 && K <= 512 && Mr >= 512) {
+      std::snprintf(name, sizeof name, "gemm_tc@%dx%d", K, N);
+      Scope sc(this, name, 1, 4.0 * ((double)Mr * (lda + ldc) + (double)K * ldb), 2.0 * (double)Mr * N * K);
+      const int tiles = (int)cdiv(Mr, gtc::kBlockM);
+#define TC_CASE(NT)                                                                                          \
+  {                                                                                                          \
+    const size_t smem = gtc::smem_bytes<NT>();                                                               \
+    CU(cudaFuncSetAttribute(gtc::k_gemm_tc<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));    \
+    const int per_sm = std::max(1, std::min(2, (int)((220 * 1024) / smem)));                                 \
+    const int grid = std::min(tiles, kSmCount * per_sm);                                                     \
+    gtc::k_gemm_tc<NT><<<grid, gtc::kThreads, smem, stream>>>(A, lda, Bk, ldbk, Cm, ldc, (int)Mr, N, K, skip, tc_error); \
+  }
+      if (N <= 16) TC_CASE(16)
+      else if (N <= 32) TC_CASE(32)
+      else if (N <= 48) TC_CASE(48)
+      else if (N <= 64) TC_CASE(64)
+      else if (N <= 128) TC_CASE(128)
+      else TC_CASE(256)
+#undef TC_CASE
+      CU(cudaGetLastError());
+      return;
+    }
     std::snprintf(name, sizeof name, "gemm_nn@%dx%d", K, N);
     Scope sc(this, name, 1, 4.0 * ((double)Mr * (lda + ldc) + (double)K * ldb), 2.0 * (double)Mr * N * K);
 #define NN_CASE(BM, BN, BK, TM, TN)                                                             \
@@ -264,12 +292,13 @@ struct gcn_admm {
     resid(l, B0);                                                       // R_l
     gemm_tn(P[l], ld[l - 1], B0, ldc, grad, ldc, n, Kp, Cn);            // grad = P_l^T R_l
     {
-      Scope sc(this, "small", 2, 0.0, 0.0);
+      Scope sc(this, "small", 3, 0.0, 0.0);
+      gk::k_transpose_small<<<(unsigned)cdiv((long long)Kp * Cn, 256), 256, 0, stream>>>(grad, ldc, grad_t, ld[l - 1], Kp, Cn);
       gk::k_two_sumsq<<<1, 1024, 0, stream>>>(grad, W[l], (long long)Kp * ldc, sums_w);
       gk::k_search_begin<<<1, 32, 0, stream>>>(ctl, 1, sums_w, 2, p.bt_shrink, p.bt_growth, acc_w, gk::kCand, nullptr);
       CU(cudaGetLastError());
     }
-    gemm_nn(P[l], ld[l - 1], grad, ldc, B1, ldc, n, Cn, Kp, &ctl->done);   // D = P_l grad
+    gemm_nn(P[l], ld[l - 1], grad, ldc, grad_t, ld[l - 1], B1, ldc, n, Cn, Kp, &ctl->done);   // D = P_l grad
     gk::DecideArgs a{};
     a.growth = p.bt_growth;
     a.max_trials = p.bt_max_trials;
@@ -316,7 +345,7 @@ struct gcn_admm {
     SearchCtl* ctl = ctl_z + (size_t)l * M;
     resid(l + 1, B0);                                                    // R'_{l+1}
     spmm(B0, B1, ldn);                                                   // S = A~ R'
-    gemm_nn(B1, ldn, Wt[l + 1], ldl, B2, ldl, n, C[l], C[l + 1]);        // S W_{l+1}^T
+    gemm_nn(B1, ldn, Wt[l + 1], ldl, W[l + 1], ldn, B2, ldl, n, C[l], C[l + 1]);        // S W_{l+1}^T
     CU(cudaMemsetAsync(sums_z, 0, sizeof(double) * 3 * M, stream));
     CU(cudaMemsetAsync(n_active, 0, sizeof(int), stream));
     const int rows_per_block = 32;
@@ -333,7 +362,7 @@ struct gcn_admm {
                                                                      per, n_active);
       CU(cudaGetLastError());
     }
-    gemm_nn(B2, ldl, W[l + 1], ldn, B1, ldn, n, C[l + 1], C[l]);         // T = G W_{l+1}
+    gemm_nn(B2, ldl, W[l + 1], ldn, Wt[l + 1], ldl, B1, ldn, n, C[l + 1], C[l]);         // T = G W_{l+1}
     gk::DecideArgs a{};
     a.growth = p.bt_growth;
     a.max_trials = p.bt_max_trials;
@@ -425,7 +454,8 @@ struct gcn_admm {
   // P_l = A~ Z_{l-1} (l >= 2; P_1 is constant) and H_l = P_l W_l from the stored W, Z.
   void refresh() {
     for (int l = 2; l <= L; ++l) spmm(Z[l - 1], P[l], ld[l - 1]);
-    for (int l = 1; l <= L; ++l) gemm_nn(P[l], ld[l - 1], W[l], ld[l], H[l], ld[l], n, C[l], C[l - 1]);
+    for (int l = 1; l <= L; ++l)
+      gemm_nn(P[l], ld[l - 1], W[l], ld[l], Wt[l], ld[l - 1], H[l], ld[l], n, C[l], C[l - 1]);
     fresh = true;
   }
 
@@ -442,21 +472,26 @@ struct gcn_admm {
 
   // logits of Problem 1's forward pass with the stored W, left in B0 (N x ld_L)
   void forward_logits() {
-    gemm_nn(P[1], ld[0], W[1], ld[1], B0, ld[1], n, C[1], C[0]);
+    gemm_nn(P[1], ld[0], W[1], ld[1], Wt[1], ld[0], B0, ld[1], n, C[1], C[0]);
     for (int l = 1; l < L; ++l) {
       const long long n4 = n * ld[l] / 4;
       Scope sc(this, "relu", 1, 32.0 * n4, 0.0);
       gk::k_relu_inplace<<<grid_for(n4), 256, 0, stream>>>((float4*)B0, n4);
       CU(cudaGetLastError());
       spmm(B0, B1, ld[l]);
-      gemm_nn(B1, ld[l], W[l + 1], ld[l + 1], B0, ld[l + 1], n, C[l + 1], C[l]);
+      gemm_nn(B1, ld[l], W[l + 1], ld[l + 1], Wt[l + 1], ld[l], B0, ld[l + 1], n, C[l + 1], C[l]);
     }
   }
 
   void check_status() {
-    int s = 0;
+    int s = 0, t = 0;
     CU(cudaMemcpyAsync(&s, status, sizeof(int), cudaMemcpyDeviceToHost, stream));
+    CU(cudaMemcpyAsync(&t, tc_error, sizeof(int), cudaMemcpyDeviceToHost, stream));
     CU(cudaStreamSynchronize(stream));
+    if (t != 0) {
+      CU(cudaMemsetAsync(tc_error, 0, sizeof(int), stream));
+      throw Fail{GCN_ADMM_ERR_CUDA, "a tensor-core product gave up waiting on its pipeline"};
+    }
     if (s & 1) {
       CU(cudaMemsetAsync(status, 0, sizeof(int), stream));
       throw Fail{GCN_ADMM_ERR_NONFINITE, "a non-finite value reached a step-size decision"};
@@ -597,7 +632,7 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
   const size_t rows = (size_t)n;
   h->W.assign(L + 1, nullptr); h->Wt.assign(L + 1, nullptr); h->Z.assign(L + 1, nullptr);
   h->P.assign(L + 1, nullptr); h->H.assign(L + 1, nullptr);
-  size_t grad_elems = 1;
+  size_t grad_elems = 1, grad_t_elems = 1;
   h->part_elems = 1;
   for (int l = 1; l <= L; ++l) {
     h->W[l] = h->alloc<float>((size_t)h->C[l - 1] * h->ld[l]);
@@ -607,6 +642,7 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
     h->H[l] = h->alloc<float>(rows * h->ld[l]);
     const size_t ge = (size_t)h->C[l - 1] * h->ld[l];
     grad_elems = std::max(grad_elems, ge);
+    grad_t_elems = std::max(grad_t_elems, (size_t)h->C[l] * h->ld[l - 1]);
     h->part_elems = std::max(h->part_elems, ge * 4 * kSmCount);
   }
   h->part_elems = std::min<size_t>(h->part_elems, (size_t)64 << 20);   // at most 256 MB of partial sums
@@ -616,6 +652,10 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
   h->B1 = h->alloc<float>(rows * h->max_ld);
   h->B2 = h->alloc<float>(rows * h->max_ld);
   h->grad = h->alloc<float>(grad_elems);
+  h->grad_t = h->alloc<float>(grad_t_elems);
+  h->tc_error = h->alloc<int>(1);
+  CU(cudaMemset(h->tc_error, 0, sizeof(int)));
+  CU(cudaMemset(h->grad_t, 0, grad_t_elems * sizeof(float)));
   h->part = h->alloc<float>(h->part_elems);
   h->ctl_w = h->alloc<SearchCtl>(L + 1);
   h->ctl_z = h->alloc<SearchCtl>((size_t)(L + 1) * n_comm);
@@ -676,7 +716,7 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
   // initial residuals are exactly zero
   for (int l = 1; l <= L; ++l) {
     if (l >= 2) h->spmm(h->Z[l - 1], h->P[l], h->ld[l - 1]);
-    h->gemm_nn(h->P[l], h->ld[l - 1], h->W[l], h->ld[l], h->H[l], h->ld[l], n, h->C[l], h->C[l - 1]);
+    h->gemm_nn(h->P[l], h->ld[l - 1], h->W[l], h->ld[l], h->Wt[l], h->ld[l - 1], h->H[l], h->ld[l], n, h->C[l], h->C[l - 1]);
     const size_t bytes = rows * h->ld[l] * sizeof(float);
     CU(cudaMemcpyAsync(h->Z[l], h->H[l], bytes, cudaMemcpyDeviceToDevice, h->stream));
     if (l < L) {
@@ -704,6 +744,7 @@ void gcn_admm_default_params(gcn_admm_params* p) {
   p->fista_iters = 30;
   p->loss_scale = 1.f;
   p->dual_mode = 0;
+  p->tensor_cores = 1;
   p->w_init = nullptr;
   p->device = 0;
   p->stream = nullptr;
@@ -887,6 +928,42 @@ int gcn_admm_propagate(gcn_admm* h, const float* x, int width, float* out) {
       throw;
     }
     cudaFree(dense); cudaFree(a); cudaFree(b);
+  });
+}
+
+int gcn_admm_dense_product(gcn_admm* h, const float* A, const float* B, float* C, long long m, int n, int k,
+                           int tensor_cores) {
+  return guarded(h, [&] {
+    if (!A || !B || !C || m < 1 || n < 1 || k < 1 || m > 2147483647LL) throw Fail{GCN_ADMM_ERR_ARG, "bad argument"};
+    if (!is_device_pointer(A) || !is_device_pointer(B) || !is_device_pointer(C))
+      throw Fail{GCN_ADMM_ERR_ARG, "A, B and C must be device pointers"};
+    const int lda = ldpad(k), ldb = ldpad(n), ldc = ldpad(n), ldbk = ldpad(k);
+    float *a = nullptr, *b = nullptr, *bk = nullptr, *c = nullptr;
+    const int saved = h->p.tensor_cores;
+    try {
+      a = dalloc<float>((size_t)m * lda);
+      b = dalloc<float>((size_t)k * ldb);
+      bk = dalloc<float>((size_t)n * ldbk);
+      c = dalloc<float>((size_t)m * ldc);
+      CU(cudaMemsetAsync(a, 0, (size_t)m * lda * 4, h->stream));
+      CU(cudaMemsetAsync(b, 0, (size_t)k * ldb * 4, h->stream));
+      CU(cudaMemsetAsync(bk, 0, (size_t)n * ldbk * 4, h->stream));
+      CU(cudaMemcpy2DAsync(a, (size_t)lda * 4, A, (size_t)k * 4, (size_t)k * 4, (size_t)m, cudaMemcpyDeviceToDevice, h->stream));
+      CU(cudaMemcpy2DAsync(b, (size_t)ldb * 4, B, (size_t)n * 4, (size_t)n * 4, (size_t)k, cudaMemcpyDeviceToDevice, h->stream));
+      gk::k_transpose_small<<<(unsigned)cdiv((long long)k * n, 256), 256, 0, h->stream>>>(b, ldb, bk, ldbk, k, n);
+      CU(cudaGetLastError());
+      h->p.tensor_cores = tensor_cores ? 1 : 0;
+      h->gemm_nn(a, lda, b, ldb, tensor_cores ? bk : nullptr, ldbk, c, ldc, m, n, k);
+      h->p.tensor_cores = saved;
+      CU(cudaMemcpy2DAsync(C, (size_t)n * 4, c, (size_t)ldc * 4, (size_t)n * 4, (size_t)m, cudaMemcpyDeviceToDevice, h->stream));
+      CU(cudaStreamSynchronize(h->stream));
+    } catch (...) {
+      h->p.tensor_cores = saved;
+      cudaFree(a); cudaFree(b); cudaFree(bk); cudaFree(c);
+      throw;
+    }
+    cudaFree(a); cudaFree(b); cudaFree(bk); cudaFree(c);
+    h->check_status();
   });
 }
 

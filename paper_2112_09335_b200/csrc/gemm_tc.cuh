@@ -1,0 +1,289 @@
+// Dense product C[M x N] = A[M x K] * B on the 5th-generation tensor cores (tcgen05, accumulator
+// in tensor memory), used for the feature-by-weight contractions of every layer:
+//   H_l = P_l W_l,  D = P_l grad,  G = S W_{l+1}^T,  T = G W_{l+1}.
+//
+// fp32 accuracy from TF32 hardware: each operand x is split into x_hi + x_lo with both halves exactly
+// representable in TF32 (x_hi = x rounded to 10 mantissa bits, x_lo = x - x_hi rounded again), and
+//   A B ~= A_lo B_hi + A_hi B_lo + A_hi B_hi
+// is accumulated in fp32.  The dropped terms are below 2^-21 of |a||b| per product, which keeps the
+// products inside the 1e-5 single-block tolerance; one TF32 pass (2^-11) would not.  The tensor core
+// rounds its fp32 accumulator toward zero at every MMA (measured: the error grows with the number of
+// MMAs per accumulator), so the main product A_hi B_hi and the two small correction products get
+// separate accumulators in tensor memory and are added once, in the epilogue; the residual error is
+// about (K/8) * 2^-24 of the accumulated magnitude, which is why K is capped by the caller.
+//
+// Shapes: A is M x K row-major (K contiguous), B is given K-major too: Bk[n][k] = B[k][n], N x K
+// row-major (the library keeps W_l and its transpose, so one of them always has this form).
+// One CTA owns 128 rows of A and all N <= 256 columns; the accumulators (128 lanes x 2 NT columns of
+// fp32) live in tensor memory.  K is walked in chunks of 32 floats = one 128-byte swizzle row.
+// All 256 threads stage the chunk: 128-bit loads from global memory, split into hi/lo, stores into
+// shared memory in the canonical K-major 128-byte-swizzled operand layout; then one thread issues
+// the twelve MMAs (3 products x 4 steps of K = 8) and commits them to the mbarrier that frees the
+// stage.  Loads of the next chunk are in flight while the current MMAs run.  Every wait on an
+// mbarrier is bounded; a wait that runs out raises `*error_flag` and the CTA leaves through the
+// normal exit (tensor memory released).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace gtc {
+
+constexpr int kBlockM = 128;
+constexpr int kChunkK = 32;                 // floats per K chunk (128 bytes)
+constexpr int kThreads = 256;
+constexpr int kStages = 2;
+constexpr int kATileBytes = kBlockM * kChunkK * 4;     // 16 KiB, one of hi / lo
+constexpr uint32_t kSpinLimit = 4u << 20;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+// Bounded wait for the phase with the given parity; false when the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+
+// Shared-memory operand descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t operand_desc(uint32_t smem_addr) {
+  const uint32_t lo = ((smem_addr >> 4) & 0x3fffu) | (1u << 16);          // start address, LBO field = 1
+  const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);             // SBO, version 1, SWIZZLE_128B
+  return ((uint64_t)hi << 32) | lo;
+}
+
+// Instruction descriptor: D fp32, A and B TF32, both K-major, M = 128, N = nt.
+__device__ __forceinline__ uint32_t instr_desc(int nt) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(nt >> 3) << 17) | ((uint32_t)(kBlockM >> 4) << 24);
+}
+
+__device__ __forceinline__ void mma_tf32(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+#define GTC_TMEM_LD16(v, addr)                                                                                       \
+  asm volatile(                                                                                                      \
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];" \
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),   \
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])                      \
+      : "r"(addr)                                                                                                    \
+      : "memory")
+
+// x -> (hi, lo): hi = x rounded to TF32 (ties away), lo = (x - hi) rounded to TF32; both carry zero
+// in the 13 low mantissa bits, so the tensor core reads them exactly.
+__device__ __forceinline__ void split_tf32(float x, float& hi, float& lo) {
+  const uint32_t u = __float_as_uint(x);
+  hi = __uint_as_float((u + 0x1000u) & 0xffffe000u);
+  const float r = x - hi;
+  lo = __uint_as_float((__float_as_uint(r) + 0x1000u) & 0xffffe000u);
+}
+
+// Swizzled byte offset of the 16-byte unit `c16` (0..7) of row `r` inside a K-major operand tile.
+__device__ __forceinline__ uint32_t swz(int r, int c16) { return (uint32_t)r * 128u + (uint32_t)((c16 ^ (r & 7)) << 4); }
+
+// Dynamic shared memory: [stage][A_hi | A_lo | B_hi | B_lo], each tile 1024-byte aligned.
+template <int NT>   // NT: accumulator columns = N rounded up to 16 (16..256)
+__global__ void __launch_bounds__(kThreads, 1)
+k_gemm_tc(const float* __restrict__ A, int lda, const float* __restrict__ Bk, int ldbk, float* __restrict__ C, int ldc,
+          int M, int N, int K, const int* __restrict__ skip, int* __restrict__ error_flag) {
+  constexpr int kBTileBytes = NT * kChunkK * 4;
+  constexpr int kStageBytes = 2 * kATileBytes + 2 * kBTileBytes;
+  constexpr int ROWS_PER_PASS = kThreads / 8;                      // 32 rows per pass of the loaders
+  constexpr int B_PASSES = (NT + ROWS_PER_PASS - 1) / ROWS_PER_PASS;
+  constexpr int A_PASSES = kBlockM / ROWS_PER_PASS;                // 4
+  constexpr uint32_t TMEM_COLS = 2 * NT <= 32 ? 32 : 2 * NT <= 64 ? 64 : 2 * NT <= 128 ? 128 : 2 * NT <= 256 ? 256 : 512;
+  if (skip != nullptr && *skip) return;
+
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[kStages + 1];
+  __shared__ uint32_t tmem_base_slot;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t smem_base = smem_u32(smem);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t bar_empty0 = smem_u32(&bars[0]);
+  const uint32_t bar_acc = smem_u32(&bars[kStages]);
+
+  if (tid == 0) {
+    for (int s = 0; s <= kStages; ++s) mbar_init(smem_u32(&bars[s]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = tmem_base_slot;
+  const uint32_t idesc = instr_desc(NT);
+
+  const int kc_count = (K + kChunkK - 1) / kChunkK;
+  const int n_tiles = (M + kBlockM - 1) / kBlockM;
+  const int ld_c16 = tid & 7;          // which 16-byte unit of the 128-byte row this thread stages
+  const int ld_row = tid >> 3;         // 0..31, plus 32 per pass
+
+  float4 ra[A_PASSES], rb[B_PASSES];
+  auto load_chunk = [&](int tile, int kc) {
+    const int k0 = kc * kChunkK + ld_c16 * 4;
+    const long long row0 = (long long)tile * kBlockM;
+#pragma unroll
+    for (int i = 0; i < A_PASSES; ++i) {
+      const long long r = row0 + ld_row + 32 * i;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (r < M && k0 < K) {
+        v = *reinterpret_cast<const float4*>(A + r * lda + k0);   // lda % 4 == 0 and k0 % 4 == 0
+        if (k0 + 1 >= K) v.y = 0.f;
+        if (k0 + 2 >= K) v.z = 0.f;
+        if (k0 + 3 >= K) v.w = 0.f;
+      }
+      ra[i] = v;
+    }
+#pragma unroll
+    for (int i = 0; i < B_PASSES; ++i) {
+      const int nrow = ld_row + 32 * i;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (nrow < N && k0 < K) {
+        v = *reinterpret_cast<const float4*>(Bk + (long long)nrow * ldbk + k0);
+        if (k0 + 1 >= K) v.y = 0.f;
+        if (k0 + 2 >= K) v.z = 0.f;
+        if (k0 + 3 >= K) v.w = 0.f;
+      }
+      rb[i] = v;
+    }
+  };
+  auto store_chunk = [&](int stage) {
+    uint8_t* st = smem + (size_t)stage * kStageBytes;
+#pragma unroll
+    for (int i = 0; i < A_PASSES; ++i) {
+      float4 h, l;
+      split_tf32(ra[i].x, h.x, l.x); split_tf32(ra[i].y, h.y, l.y);
+      split_tf32(ra[i].z, h.z, l.z); split_tf32(ra[i].w, h.w, l.w);
+      const uint32_t off = swz(ld_row + 32 * i, ld_c16);
+      *reinterpret_cast<float4*>(st + off) = h;
+      *reinterpret_cast<float4*>(st + kATileBytes + off) = l;
+    }
+#pragma unroll
+    for (int i = 0; i < B_PASSES; ++i) {
+      const int nrow = ld_row + 32 * i;
+      if (nrow < NT) {
+        float4 h, l;
+        split_tf32(rb[i].x, h.x, l.x); split_tf32(rb[i].y, h.y, l.y);
+        split_tf32(rb[i].z, h.z, l.z); split_tf32(rb[i].w, h.w, l.w);
+        const uint32_t off = swz(nrow, ld_c16);
+        *reinterpret_cast<float4*>(st + 2 * kATileBytes + off) = h;
+        *reinterpret_cast<float4*>(st + 2 * kATileBytes + kBTileBytes + off) = l;
+      }
+    }
+  };
+
+  uint32_t stage_uses[kStages];
+#pragma unroll
+  for (int s = 0; s < kStages; ++s) stage_uses[s] = 0;
+  uint32_t it = 0, tiles_done = 0;
+  bool failed = false;
+
+  int tile = blockIdx.x;
+  if (tile < n_tiles) load_chunk(tile, 0);
+  for (; tile < n_tiles && !failed; tile += gridDim.x) {
+    for (int kc = 0; kc < kc_count; ++kc, ++it) {
+      const int stage = it % kStages;
+      // the MMAs that last read this stage must have completed before it is overwritten
+      bool ok = true;
+      if (stage_uses[stage] > 0) ok = mbar_wait(bar_empty0 + 8 * stage, (stage_uses[stage] - 1) & 1);
+      if (__syncthreads_or(!ok)) { failed = true; break; }
+      store_chunk(stage);
+      ++stage_uses[stage];
+      // next chunk (of this tile or of the CTA's next tile) on its way while the MMAs run
+      if (kc + 1 < kc_count) load_chunk(tile, kc + 1);
+      else if (tile + (int)gridDim.x < n_tiles) load_chunk(tile + gridDim.x, 0);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> async-proxy reads
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncthreads();
+      if (tid == 0) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t a_hi = smem_base + stage * kStageBytes, a_lo = a_hi + kATileBytes;
+        const uint32_t b_hi = a_hi + 2 * kATileBytes, b_lo = b_hi + kBTileBytes;
+#pragma unroll
+        for (int ks = 0; ks < kChunkK / 8; ++ks) {
+          const uint32_t o = ks * 32;    // 8 floats further along K inside the swizzled row
+          const uint32_t first = (kc > 0 || ks > 0) ? 1u : 0u;
+          mma_tf32(tmem_base + NT, operand_desc(a_lo + o), operand_desc(b_hi + o), idesc, first);   // corrections
+          mma_tf32(tmem_base + NT, operand_desc(a_hi + o), operand_desc(b_lo + o), idesc, 1u);
+          mma_tf32(tmem_base, operand_desc(a_hi + o), operand_desc(b_hi + o), idesc, first);        // main product
+        }
+        mma_commit(bar_empty0 + 8 * stage);
+        if (kc + 1 == kc_count) mma_commit(bar_acc);
+      }
+    }
+    if (failed) break;
+    // epilogue: accumulators (tensor memory) -> registers -> C
+    {
+      const bool ok = mbar_wait(bar_acc, tiles_done & 1);
+      if (__syncthreads_or(!ok)) { failed = true; break; }
+      ++tiles_done;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int quarter = warp & 3;                       // tensor-memory lanes 32*quarter .. +31
+      const long long row = (long long)tile * kBlockM + quarter * 32 + lane;
+      for (int cchunk = (warp >> 2); cchunk < NT / 16; cchunk += 2) {
+        uint32_t v[16], w[16];
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(cchunk * 16);
+        GTC_TMEM_LD16(v, taddr);
+        GTC_TMEM_LD16(w, taddr + (uint32_t)NT);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (row < M) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int col = cchunk * 16 + q * 4;
+            if (col < ldc)   // ldc % 4 == 0; columns N..ldc-1 receive the zeros of B's padding rows
+              *reinterpret_cast<float4*>(C + row * ldc + col) =
+                  make_float4(__uint_as_float(v[q * 4]) + __uint_as_float(w[q * 4]),
+                              __uint_as_float(v[q * 4 + 1]) + __uint_as_float(w[q * 4 + 1]),
+                              __uint_as_float(v[q * 4 + 2]) + __uint_as_float(w[q * 4 + 2]),
+                              __uint_as_float(v[q * 4 + 3]) + __uint_as_float(w[q * 4 + 3]));
+          }
+        }
+      }
+      // the next tile's first MMA overwrites the accumulators: every warp must be done reading them
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncthreads();
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    }
+  }
+  if (failed && tid == 0) atomicExch(error_flag, 1);
+  // drain: the last commits must have landed before tensor memory is released
+  if (!failed) {
+    for (int s = 0; s < kStages; ++s)
+      if (stage_uses[s] > 0) mbar_wait(bar_empty0 + 8 * s, (stage_uses[s] - 1) & 1);
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// dynamic shared memory of k_gemm_tc<NT>
+template <int NT>
+constexpr size_t smem_bytes() { return (size_t)kStages * (2 * kATileBytes + 2 * NT * kChunkK * 4) + 1024; }
+
+}  // namespace gtc

@@ -1071,6 +1071,15 @@ __global__ void k_dual(float4* __restrict__ U, const float4* __restrict__ Z, con
   }
 }
 
+// dst[c][r] = src[r][c] for a small rows x cols matrix (weights and their gradients).
+__global__ void k_transpose_small(const float* __restrict__ src, int lds, float* __restrict__ dst, int ldd, int rows,
+                                  int cols) {
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= rows * cols) return;
+  const int r = e / cols, c = e % cols;
+  dst[c * ldd + r] = src[r * lds + c];
+}
+
 __global__ void k_fill_int(int* __restrict__ p, long long count, int value) {
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count;
        i += (long long)gridDim.x * blockDim.x)
