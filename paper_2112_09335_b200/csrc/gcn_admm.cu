@@ -197,6 +197,27 @@ struct gcn_admm {
       std::snprintf(name, sizeof name, "gemm_tc@%dx%d", K, N);
       Scope sc(this, name, 1, 4.0 * ((double)Mr * (lda + ldc) + (double)K * ldb), 2.0 * (double)Mr * N * K);
       const int tiles = (int)cdiv(Mr, gtc::kBlockM);
+      const size_t smem_cap = 227 * 1024;
+      // preferred form: the split weight operand stays in shared memory (column groups of NT columns)
+#define TC_RES(NT)                                                                                             \
+  if (!launched && gtc::resident_smem_bytes<NT>(K) <= smem_cap) {                                              \
+    const size_t smem = gtc::resident_smem_bytes<NT>(K);                                                       \
+    const int groups = (int)cdiv(N, NT);                                                                       \
+    CU(cudaFuncSetAttribute(gtc::k_gemm_tc_resident<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+    dim3 grid((unsigned)std::max(1, std::min(tiles, kSmCount / groups)), (unsigned)groups);                    \
+    gtc::k_gemm_tc_resident<NT><<<grid, gtc::kThreads, smem, stream>>>(A, lda, Bk, ldbk, Cm, ldc, (int)Mr, N, K, skip, tc_error); \
+    launched = true;                                                                                           \
+  }
+      bool launched = false;
+      const int want = N <= 16 ? 16 : N <= 32 ? 32 : N <= 48 ? 48 : N <= 64 ? 64 : N <= 128 ? 128 : 256;
+      if (want >= 256) TC_RES(256)
+      if (want >= 128) TC_RES(128)
+      if (want >= 64) TC_RES(64)
+      if (want == 48) TC_RES(48)
+      if (want >= 32) TC_RES(32)
+      TC_RES(16)
+#undef TC_RES
+      if (launched) { CU(cudaGetLastError()); return; }
 #define TC_CASE(NT)                                                                                          \
   {                                                                                                          \
     const size_t smem = gtc::smem_bytes<NT>();                                                               \

@@ -282,6 +282,212 @@ k_gemm_tc(const float* __restrict__ A, int lda, const float* __restrict__ Bk, in
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Second form, used whenever the split weight operand fits in shared memory next to the pipeline:
+// B stays resident.  The grid is (row workers) x (column groups of NT columns); a CTA splits its
+// NT x K slice of B into hi/lo once, keeps it for all of its row tiles, and streams only A:
+// three stages, each filled two chunks ahead with 16-byte cp.async copies (zero-filled past the
+// matrix edge), split in place by the thread that copied them (raw -> hi in the same slot, lo in
+// the neighbouring one), then consumed by the twelve MMAs of the chunk.
+// ------------------------------------------------------------------------------------------------
+constexpr int kAStages = 3;
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+
+template <int NT>
+__global__ void __launch_bounds__(kThreads, 1)
+k_gemm_tc_resident(const float* __restrict__ A, int lda, const float* __restrict__ Bk, int ldbk, float* __restrict__ C,
+                   int ldc, int M, int N, int K, const int* __restrict__ skip, int* __restrict__ error_flag) {
+  constexpr int kBTileBytes = NT * kChunkK * 4;          // one of hi / lo, one chunk
+  constexpr int kAStageBytes = 2 * kATileBytes;
+  constexpr int ROWS_PER_PASS = kThreads / 8;
+  constexpr int B_PASSES = (NT + ROWS_PER_PASS - 1) / ROWS_PER_PASS;
+  constexpr int A_PASSES = kBlockM / ROWS_PER_PASS;
+  constexpr uint32_t TMEM_COLS = 2 * NT <= 32 ? 32 : 2 * NT <= 64 ? 64 : 2 * NT <= 128 ? 128 : 2 * NT <= 256 ? 256 : 512;
+  if (skip != nullptr && *skip) return;
+
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[kAStages + 1];
+  __shared__ uint32_t tmem_base_slot;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int kc_count = (K + kChunkK - 1) / kChunkK;
+  uint8_t* a_stages = smem;                                        // kAStages x [A_hi | A_lo]
+  uint8_t* b_res = smem + (size_t)kAStages * kAStageBytes;         // kc_count x [B_hi | B_lo]
+  const uint32_t a_base = smem_u32(a_stages), b_base = smem_u32(b_res);
+  const uint32_t bar_empty0 = smem_u32(&bars[0]);
+  const uint32_t bar_acc = smem_u32(&bars[kAStages]);
+
+  if (tid == 0) {
+    for (int s = 0; s <= kAStages; ++s) mbar_init(smem_u32(&bars[s]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+
+  const int ld_c16 = tid & 7, ld_row = tid >> 3;
+  const int n0 = blockIdx.y * NT;                 // first output column of this CTA
+  const int n_loc = min(NT, N - n0);
+  // resident B: rows n0 .. n0+n_loc-1 of Bk, all K, split into hi / lo
+  for (int kc = 0; kc < kc_count; ++kc) {
+    const int k0 = kc * kChunkK + ld_c16 * 4;
+#pragma unroll
+    for (int i = 0; i < B_PASSES; ++i) {
+      const int nrow = ld_row + 32 * i;
+      if (nrow < NT) {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (nrow < n_loc && k0 < K) {
+          v = *reinterpret_cast<const float4*>(Bk + (long long)(n0 + nrow) * ldbk + k0);
+          if (k0 + 1 >= K) v.y = 0.f;
+          if (k0 + 2 >= K) v.z = 0.f;
+          if (k0 + 3 >= K) v.w = 0.f;
+        }
+        float4 h, l;
+        split_tf32(v.x, h.x, l.x); split_tf32(v.y, h.y, l.y); split_tf32(v.z, h.z, l.z); split_tf32(v.w, h.w, l.w);
+        uint8_t* dst = b_res + (size_t)kc * 2 * kBTileBytes + swz(nrow, ld_c16);
+        *reinterpret_cast<float4*>(dst) = h;
+        *reinterpret_cast<float4*>(dst + kBTileBytes) = l;
+      }
+    }
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = tmem_base_slot;
+  const uint32_t idesc = instr_desc(NT);
+
+  const int n_tiles = (M + kBlockM - 1) / kBlockM;
+  const int my_tiles = (n_tiles > (int)blockIdx.x) ? (n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  const int total = my_tiles * kc_count;
+
+  // copies of chunk j = (tile, kc) into the hi slot of stage j % kAStages, raw fp32
+  auto issue_load = [&](int j) {
+    if (j < total) {
+      const int tile = blockIdx.x + (j / kc_count) * gridDim.x, kc = j % kc_count;
+      const int k0 = kc * kChunkK + ld_c16 * 4;
+      const int kbytes = max(0, min(16, 4 * (K - k0)));
+      const uint32_t st = a_base + (j % kAStages) * kAStageBytes;
+#pragma unroll
+      for (int i = 0; i < A_PASSES; ++i) {
+        const int rr = ld_row + 32 * i;
+        const long long r = (long long)tile * kBlockM + rr;
+        const bool in = r < M && kbytes > 0;
+        cp_async16(st + swz(rr, ld_c16), in ? (const void*)(A + r * lda + k0) : (const void*)A, in ? kbytes : 0);
+      }
+    }
+    cp_async_commit();
+  };
+
+  uint32_t stage_uses[kAStages];
+#pragma unroll
+  for (int s = 0; s < kAStages; ++s) stage_uses[s] = 0;
+  uint32_t tiles_done = 0;
+  bool failed = false, bad = false;   // bad: this thread saw a wait run out; failed: the whole CTA agreed to stop
+  issue_load(0);
+  issue_load(1);
+  for (int j = 0; j < total; ++j) {
+    const int stage = j % kAStages;
+    const int kc = j % kc_count;
+    const int tile = blockIdx.x + (j / kc_count) * gridDim.x;
+    cp_async_wait_all_but_one();                   // this thread's copies of chunk j have landed
+    {
+      uint8_t* st = a_stages + (size_t)stage * kAStageBytes;
+#pragma unroll
+      for (int i = 0; i < A_PASSES; ++i) {
+        const uint32_t off = swz(ld_row + 32 * i, ld_c16);
+        const float4 v = *reinterpret_cast<const float4*>(st + off);
+        float4 h, l;
+        split_tf32(v.x, h.x, l.x); split_tf32(v.y, h.y, l.y); split_tf32(v.z, h.z, l.z); split_tf32(v.w, h.w, l.w);
+        *reinterpret_cast<float4*>(st + off) = h;
+        *reinterpret_cast<float4*>(st + kATileBytes + off) = l;
+      }
+    }
+    ++stage_uses[stage];
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    if (__syncthreads_or(bad)) { failed = true; break; }
+    if (tid == 0) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t a_hi = a_base + stage * kAStageBytes, a_lo = a_hi + kATileBytes;
+      const uint32_t b_hi = b_base + kc * 2 * kBTileBytes, b_lo = b_hi + kBTileBytes;
+#pragma unroll
+      for (int ks = 0; ks < kChunkK / 8; ++ks) {
+        const uint32_t o = ks * 32;
+        const uint32_t first = (kc > 0 || ks > 0) ? 1u : 0u;
+        mma_tf32(tmem_base + NT, operand_desc(a_lo + o), operand_desc(b_hi + o), idesc, first);   // corrections
+        mma_tf32(tmem_base + NT, operand_desc(a_hi + o), operand_desc(b_lo + o), idesc, 1u);
+        mma_tf32(tmem_base, operand_desc(a_hi + o), operand_desc(b_hi + o), idesc, first);        // main product
+      }
+      mma_commit(bar_empty0 + 8 * stage);
+      if (kc + 1 == kc_count) mma_commit(bar_acc);
+    }
+    // refill the stage that chunk j-1 used (its MMAs were issued one iteration ago) with chunk j+2
+    {
+      const int prev = (j + 2) % kAStages;
+      if (j + 2 < total && stage_uses[prev] > 0 && !mbar_wait(bar_empty0 + 8 * prev, (stage_uses[prev] - 1) & 1))
+        bad = true;
+      issue_load(bad ? total : j + 2);
+    }
+    if (kc + 1 == kc_count) {
+      // epilogue: accumulators (tensor memory) -> registers -> C
+      const bool ok = mbar_wait(bar_acc, tiles_done & 1);
+      if (__syncthreads_or(!ok || bad)) { failed = true; break; }
+      ++tiles_done;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int quarter = warp & 3;
+      const long long row = (long long)tile * kBlockM + quarter * 32 + lane;
+      for (int cchunk = (warp >> 2); cchunk < NT / 16; cchunk += 2) {
+        uint32_t v[16], w[16];
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(cchunk * 16);
+        GTC_TMEM_LD16(v, taddr);
+        GTC_TMEM_LD16(w, taddr + (uint32_t)NT);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (row < M) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int col = n0 + cchunk * 16 + q * 4;
+            if (col < ldc && cchunk * 16 + q * 4 < NT)
+              *reinterpret_cast<float4*>(C + row * ldc + col) =
+                  make_float4(__uint_as_float(v[q * 4]) + __uint_as_float(w[q * 4]),
+                              __uint_as_float(v[q * 4 + 1]) + __uint_as_float(w[q * 4 + 1]),
+                              __uint_as_float(v[q * 4 + 2]) + __uint_as_float(w[q * 4 + 2]),
+                              __uint_as_float(v[q * 4 + 3]) + __uint_as_float(w[q * 4 + 3]));
+          }
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncthreads();
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    }
+  }
+  asm volatile("cp.async.wait_all;" ::: "memory");
+  if (failed && tid == 0) atomicExch(error_flag, 1);
+  if (!failed) {
+    for (int s = 0; s < kAStages; ++s)
+      if (stage_uses[s] > 0) mbar_wait(bar_empty0 + 8 * s, (stage_uses[s] - 1) & 1);
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// dynamic shared memory of k_gemm_tc_resident<NT> for a given K
+template <int NT>
+inline size_t resident_smem_bytes(int K) {
+  const int kc = (K + kChunkK - 1) / kChunkK;
+  return (size_t)kAStages * 2 * kATileBytes + (size_t)kc * 2 * NT * kChunkK * 4 + 1024;
+}
+
 // dynamic shared memory of k_gemm_tc<NT>
 template <int NT>
 constexpr size_t smem_bytes() { return (size_t)kStages * (2 * kATileBytes + 2 * NT * kChunkK * 4) + 1024; }
