@@ -198,9 +198,10 @@ struct gcn_admm {
       Scope sc(this, name, 1, 4.0 * ((double)Mr * (lda + ldc) + (double)K * ldb), 2.0 * (double)Mr * N * K);
       const int tiles = (int)cdiv(Mr, gtc::kBlockM);
       const size_t smem_cap = 227 * 1024;
-      // preferred form: the split weight operand stays in shared memory (column groups of NT columns)
+      // preferred form when one or two column groups suffice: the split weight operand stays in shared
+      // memory; with more groups the re-reads of A cost more than re-staging B (measured), so B is streamed
 #define TC_RES(NT)                                                                                             \
-  if (!launched && gtc::resident_smem_bytes<NT>(K) <= smem_cap) {                                              \
+  if (!launched && (N + (NT) - 1) / (NT) <= 2 && gtc::resident_smem_bytes<NT>(K) <= smem_cap) {                \
     const size_t smem = gtc::resident_smem_bytes<NT>(K);                                                       \
     const int groups = (int)cdiv(N, NT);                                                                       \
     CU(cudaFuncSetAttribute(gtc::k_gemm_tc_resident<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
