@@ -56,7 +56,8 @@ enum {
  *  dual_mode       0: Eq. 3 as printed (Z_L^k, Z_{L-1}^k, W_L^{k+1}); 1: the k+1 iterates
  *  tensor_cores    1: dense products with at most 256 output columns and K <= 512 run on the tensor
  *                  cores as an error-compensated TF32 product (three passes, fp32 accumulation,
- *                  relative error of a few 1e-7 of sum |a||b|); 0: fp32 FMA kernels everywhere
+ *                  relative error of a few 1e-7 of sum |a||b|); 2: the same product with its earlier, unsplit
+ *                  scheduling (kept for comparison); 0: fp32 FMA kernels everywhere
  *  w_init          L host pointers to row-major C_{l-1} x C_l matrices (required)
  *  device          CUDA device ordinal;  stream: a cudaStream_t owned by the caller (NULL = the
  *                  default stream) */

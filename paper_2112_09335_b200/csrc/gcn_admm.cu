@@ -197,6 +197,24 @@ struct gcn_admm {
       std::snprintf(name, sizeof name, "gemm_tc@%dx%d", K, N);
       Scope sc(this, name, 1, 4.0 * ((double)Mr * (lda + ldc) + (double)K * ldb), 2.0 * (double)Mr * N * K);
       const int tiles = (int)cdiv(Mr, gtc::kBlockM);
+      if (p.tensor_cores == 1) {   // role-split kernel: producers / MMA issue / epilogue overlap
+#define TC_WS(NT)                                                                                              \
+  {                                                                                                            \
+    const size_t smem = gtc::WsCfg<NT>::kSmem;                                                                 \
+    const int groups = (int)cdiv(N, NT);                                                                       \
+    CU(cudaFuncSetAttribute(gtc::k_gemm_tc_ws<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));   \
+    dim3 grid((unsigned)std::max(1, std::min(tiles, kSmCount / groups)), (unsigned)groups);                    \
+    gtc::k_gemm_tc_ws<NT><<<grid, gtc::kWsThreads, smem, stream>>>(A, lda, Bk, ldbk, Cm, ldc, (int)Mr, N, K, skip, tc_error); \
+  }
+        if (N <= 16) TC_WS(16)
+        else if (N <= 32) TC_WS(32)
+        else if (N <= 48) TC_WS(48)
+        else if (N <= 64) TC_WS(64)
+        else TC_WS(128)
+#undef TC_WS
+        CU(cudaGetLastError());
+        return;
+      }
       const size_t smem_cap = 227 * 1024;
       // preferred form when one or two column groups suffice: the split weight operand stays in shared
       // memory; with more groups the re-reads of A cost more than re-staging B (measured), so B is streamed
@@ -974,7 +992,7 @@ int gcn_admm_dense_product(gcn_admm* h, const float* A, const float* B, float* C
       CU(cudaMemcpy2DAsync(b, (size_t)ldb * 4, B, (size_t)n * 4, (size_t)n * 4, (size_t)k, cudaMemcpyDeviceToDevice, h->stream));
       gk::k_transpose_small<<<(unsigned)cdiv((long long)k * n, 256), 256, 0, h->stream>>>(b, ldb, bk, ldbk, k, n);
       CU(cudaGetLastError());
-      h->p.tensor_cores = tensor_cores ? 1 : 0;
+      h->p.tensor_cores = tensor_cores;
       h->gemm_nn(a, lda, b, ldb, tensor_cores ? bk : nullptr, ldbk, c, ldc, m, n, k);
       h->p.tensor_cores = saved;
       CU(cudaMemcpy2DAsync(C, (size_t)n * 4, c, (size_t)ldc * 4, (size_t)n * 4, (size_t)m, cudaMemcpyDeviceToDevice, h->stream));

@@ -488,6 +488,230 @@ inline size_t resident_smem_bytes(int K) {
   return (size_t)kAStages * 2 * kATileBytes + (size_t)kc * 2 * NT * kChunkK * 4 + 1024;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Third form: the same product with the work split by role, so that staging, MMA issue and the
+// epilogue overlap instead of taking turns.
+//   warps 0-7   producers: 128-bit loads of the A and B chunks (two chunks ahead, in registers),
+//               hi/lo split, swizzled stores, fence, arrive on full[stage]
+//   warps 8-11  epilogue: wait for a finished accumulator set, tensor memory -> registers -> C,
+//               arrive on acc_empty[set]  (warp w reads lanes 32 (w mod 4) .. +31)
+//   warp 12     MMA: waits full[stage] (and, at the first chunk of a tile, acc_empty[set]), issues
+//               the twelve MMAs, commits to empty[stage] and, at the last chunk, to acc_full[set]
+// Two accumulator sets (main + correction each) alternate between consecutive tiles, so NT <= 128
+// (4 NT <= 512 columns of tensor memory); wider outputs use two column groups.
+// A wait that runs out raises a shared abort flag that every other wait polls; all roles then meet
+// at the closing barrier and tensor memory is released.
+// ------------------------------------------------------------------------------------------------
+constexpr int kWsThreads = 13 * 32;
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if ((i & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+template <int NT>
+struct WsCfg {
+  static constexpr int kStagesWs = NT > 64 ? 3 : 4;
+  static constexpr int kBTile = NT * kChunkK * 4;                       // one of hi / lo
+  static constexpr int kStage = 2 * kATileBytes + 2 * kBTile;
+  static constexpr uint32_t kTmemCols = 4 * NT <= 64 ? 64 : 4 * NT <= 128 ? 128 : 4 * NT <= 256 ? 256 : 512;
+  static constexpr size_t kSmem = (size_t)kStagesWs * kStage + 1024;
+};
+
+template <int NT>
+__global__ void __launch_bounds__(kWsThreads, 1)
+k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk, int ldbk, float* __restrict__ C, int ldc,
+             int M, int N, int K, const int* __restrict__ skip, int* __restrict__ error_flag) {
+  using Cfg = WsCfg<NT>;
+  constexpr int S = Cfg::kStagesWs;
+  constexpr int B_PASSES = (NT + 31) / 32;
+  constexpr int A_PASSES = kBlockM / 32;
+  static_assert(NT <= 128 && NT % 16 == 0, "NT");
+  if (skip != nullptr && *skip) return;
+
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2 * S + 4];      // full[S], empty[S], acc_full[2], acc_empty[2]
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t smem_base = smem_u32(smem);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[S]);
+  const uint32_t bar_acc_full = smem_u32(&bars[2 * S]), bar_acc_empty = smem_u32(&bars[2 * S + 2]);
+
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 256); mbar_init(bar_empty + 8 * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, 128); }
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 12) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                 "r"(Cfg::kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = tmem_base_slot;
+  volatile int* abortp = &abort_flag;
+
+  const int kc_count = (K + kChunkK - 1) / kChunkK;
+  const int n_tiles = (M + kBlockM - 1) / kBlockM;
+  const int my_tiles = (n_tiles > (int)blockIdx.x) ? (n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  const int total = my_tiles * kc_count;
+  const int n0 = blockIdx.y * NT;
+  const int n_loc = min(NT, N - n0);
+
+  if (warp < 8) {
+    // ---------------- producers ----------------
+    const int ld_c16 = tid & 7, ld_row = tid >> 3;
+    float4 ra[2][A_PASSES], rb[2][B_PASSES];
+    auto load_chunk = [&](int j, float4* pa, float4* pb) {
+      if (j >= total) return;
+      const int tile = blockIdx.x + (j / kc_count) * gridDim.x, kc = j % kc_count;
+      const int k0 = kc * kChunkK + ld_c16 * 4;
+      const long long row0 = (long long)tile * kBlockM;
+#pragma unroll
+      for (int i = 0; i < A_PASSES; ++i) {
+        const long long r = row0 + ld_row + 32 * i;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (r < M && k0 < K) {
+          v = *reinterpret_cast<const float4*>(A + r * lda + k0);
+          if (k0 + 1 >= K) v.y = 0.f;
+          if (k0 + 2 >= K) v.z = 0.f;
+          if (k0 + 3 >= K) v.w = 0.f;
+        }
+        pa[i] = v;
+      }
+#pragma unroll
+      for (int i = 0; i < B_PASSES; ++i) {
+        const int nrow = ld_row + 32 * i;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (nrow < n_loc && k0 < K) {
+          v = *reinterpret_cast<const float4*>(Bk + (long long)(n0 + nrow) * ldbk + k0);
+          if (k0 + 1 >= K) v.y = 0.f;
+          if (k0 + 2 >= K) v.z = 0.f;
+          if (k0 + 3 >= K) v.w = 0.f;
+        }
+        pb[i] = v;
+      }
+    };
+    auto store_chunk = [&](int stage, const float4* pa, const float4* pb) {
+      uint8_t* st = smem + (size_t)stage * Cfg::kStage;
+#pragma unroll
+      for (int i = 0; i < A_PASSES; ++i) {
+        float4 h, l;
+        split_tf32(pa[i].x, h.x, l.x); split_tf32(pa[i].y, h.y, l.y);
+        split_tf32(pa[i].z, h.z, l.z); split_tf32(pa[i].w, h.w, l.w);
+        const uint32_t off = swz(ld_row + 32 * i, ld_c16);
+        *reinterpret_cast<float4*>(st + off) = h;
+        *reinterpret_cast<float4*>(st + kATileBytes + off) = l;
+      }
+#pragma unroll
+      for (int i = 0; i < B_PASSES; ++i) {
+        const int nrow = ld_row + 32 * i;
+        if (nrow < NT) {
+          float4 h, l;
+          split_tf32(pb[i].x, h.x, l.x); split_tf32(pb[i].y, h.y, l.y);
+          split_tf32(pb[i].z, h.z, l.z); split_tf32(pb[i].w, h.w, l.w);
+          const uint32_t off = swz(nrow, ld_c16);
+          *reinterpret_cast<float4*>(st + 2 * kATileBytes + off) = h;
+          *reinterpret_cast<float4*>(st + 2 * kATileBytes + Cfg::kBTile + off) = l;
+        }
+      }
+    };
+    load_chunk(0, ra[0], rb[0]);
+    load_chunk(1, ra[1], rb[1]);
+    for (int j = 0; j < total; ++j) {
+      const int stage = j % S;
+      if (j >= S && !mbar_wait_abortable(bar_empty + 8 * stage, ((j / S) - 1) & 1, abortp)) break;
+      if (j & 1) { store_chunk(stage, ra[1], rb[1]); load_chunk(j + 2, ra[1], rb[1]); }
+      else       { store_chunk(stage, ra[0], rb[0]); load_chunk(j + 2, ra[0], rb[0]); }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_arrive(bar_full + 8 * stage);
+    }
+  } else if (warp == 12) {
+    // ---------------- MMA issue ----------------
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc(NT);
+      for (int j = 0; j < total; ++j) {
+        const int stage = j % S, kc = j % kc_count, tile_i = j / kc_count, set = tile_i & 1;
+        if (kc == 0 && tile_i >= 2 && !mbar_wait_abortable(bar_acc_empty + 8 * set, ((tile_i >> 1) - 1) & 1, abortp)) break;
+        if (!mbar_wait_abortable(bar_full + 8 * stage, (j / S) & 1, abortp)) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t a_hi = smem_base + stage * Cfg::kStage, a_lo = a_hi + kATileBytes;
+        const uint32_t b_hi = a_hi + 2 * kATileBytes, b_lo = b_hi + Cfg::kBTile;
+        const uint32_t acc = tmem_base + (uint32_t)(set * 2 * NT);
+#pragma unroll
+        for (int ks = 0; ks < kChunkK / 8; ++ks) {
+          const uint32_t o = ks * 32;
+          const uint32_t first = (kc > 0 || ks > 0) ? 1u : 0u;
+          mma_tf32(acc + NT, operand_desc(a_lo + o), operand_desc(b_hi + o), idesc, first);   // corrections
+          mma_tf32(acc + NT, operand_desc(a_hi + o), operand_desc(b_lo + o), idesc, 1u);
+          mma_tf32(acc, operand_desc(a_hi + o), operand_desc(b_hi + o), idesc, first);        // main product
+        }
+        mma_commit(bar_empty + 8 * stage);
+        if (kc + 1 == kc_count) mma_commit(bar_acc_full + 8 * set);
+      }
+    }
+  } else {
+    // ---------------- epilogue ----------------
+    const int quarter = warp & 3;
+    for (int tile_i = 0; tile_i < my_tiles; ++tile_i) {
+      const int set = tile_i & 1;
+      if (!mbar_wait_abortable(bar_acc_full + 8 * set, (tile_i >> 1) & 1, abortp)) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const long long row = (long long)(blockIdx.x + tile_i * gridDim.x) * kBlockM + quarter * 32 + lane;
+#pragma unroll 1
+      for (int cchunk = 0; cchunk < NT / 16; ++cchunk) {
+        uint32_t v[16], w[16];
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(set * 2 * NT + cchunk * 16);
+        GTC_TMEM_LD16(v, taddr);
+        GTC_TMEM_LD16(w, taddr + (uint32_t)NT);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (row < M) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int col = n0 + cchunk * 16 + q * 4;
+            if (col < ldc)
+              *reinterpret_cast<float4*>(C + row * ldc + col) =
+                  make_float4(__uint_as_float(v[q * 4]) + __uint_as_float(w[q * 4]),
+                              __uint_as_float(v[q * 4 + 1]) + __uint_as_float(w[q * 4 + 1]),
+                              __uint_as_float(v[q * 4 + 2]) + __uint_as_float(w[q * 4 + 2]),
+                              __uint_as_float(v[q * 4 + 3]) + __uint_as_float(w[q * 4 + 3]));
+          }
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      mbar_arrive(bar_acc_empty + 8 * set);
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (tid == 0 && abort_flag) atomicExch(error_flag, 1);
+  if (warp == 12) {
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(Cfg::kTmemCols) : "memory");
+  }
+}
+
 // dynamic shared memory of k_gemm_tc<NT>
 template <int NT>
 constexpr size_t smem_bytes() { return (size_t)kStages * (2 * kATileBytes + 2 * NT * kChunkK * 4) + 1024; }

@@ -20,7 +20,7 @@ def handle():
     g.destroy()
 
 
-@pytest.mark.parametrize("tensor_cores", [1, 0])
+@pytest.mark.parametrize("tensor_cores", [1, 2, 0])
 @pytest.mark.parametrize("m,n,k", SHAPES)
 def test_dense_product_against_fp64(handle, m, n, k, tensor_cores):
     import torch
