@@ -2,8 +2,8 @@
 // in tensor memory), used for the feature-by-weight contractions of every layer:
 //   H_l = P_l W_l,  D = P_l grad,  G = S W_{l+1}^T,  T = G W_{l+1}.
 //
-// fp32 accuracy from TF32 hardware: each operand x is split into x_hi + x_lo with both halves exactly
-// representable in TF32 (x_hi = x rounded to 10 mantissa bits, x_lo = x - x_hi rounded again), and
+// fp32 accuracy from TF32 hardware: each operand x is split into x_hi + x_lo with both halves held
+// at TF32 resolution (x_hi = x rounded to 10 mantissa bits, x_lo = x - x_hi, at most 2^-11 of x), and
 //   A B ~= A_lo B_hi + A_hi B_lo + A_hi B_hi
 // is accumulated in fp32.  The dropped terms are below 2^-21 of |a||b| per product, which keeps the
 // products inside the 1e-5 single-block tolerance; one TF32 pass (2^-11) would not.  The tensor core
@@ -11,6 +11,10 @@
 // MMAs per accumulator), so the main product A_hi B_hi and the two small correction products get
 // separate accumulators in tensor memory and are added once, in the epilogue; the residual error is
 // about (K/8) * 2^-24 of the accumulated magnitude, which is why K is capped by the caller.
+//
+// Operand padding: leading dimensions are multiples of 4 floats and the columns K .. ld-1 of A and of
+// Bk hold zeros (the library's layout invariant), so a 128-bit load that straddles K needs no masking --
+// which matters: touching a loaded value right after the load would stall the prefetch.
 //
 // Shapes: A is M x K row-major (K contiguous), B is given K-major too: Bk[n][k] = B[k][n], N x K
 // row-major (the library keeps W_l and its transpose, so one of them always has this form).
@@ -88,13 +92,12 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
       : "r"(addr)                                                                                                    \
       : "memory")
 
-// x -> (hi, lo): hi = x rounded to TF32 (ties away), lo = (x - hi) rounded to TF32; both carry zero
-// in the 13 low mantissa bits, so the tensor core reads them exactly.
+// x -> (hi, lo): hi = x rounded to TF32 (ties away; zero in the 13 low mantissa bits, so the tensor
+// core reads it exactly), lo = x - hi exactly (|lo| <= 2^-11 |x|).  lo is handed over as it is: whatever
+// the hardware does with its low 13 bits moves it by at most 2^-10 |lo| <= 2^-21 |x|.
 __device__ __forceinline__ void split_tf32(float x, float& hi, float& lo) {
-  const uint32_t u = __float_as_uint(x);
-  hi = __uint_as_float((u + 0x1000u) & 0xffffe000u);
-  const float r = x - hi;
-  lo = __uint_as_float((__float_as_uint(r) + 0x1000u) & 0xffffe000u);
+  hi = __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xffffe000u);
+  lo = x - hi;
 }
 
 // Swizzled byte offset of the 16-byte unit `c16` (0..7) of row `r` inside a K-major operand tile.
@@ -152,9 +155,6 @@ k_gemm_tc(const float* __restrict__ A, int lda, const float* __restrict__ Bk, in
       float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
       if (r < M && k0 < K) {
         v = *reinterpret_cast<const float4*>(A + r * lda + k0);   // lda % 4 == 0 and k0 % 4 == 0
-        if (k0 + 1 >= K) v.y = 0.f;
-        if (k0 + 2 >= K) v.z = 0.f;
-        if (k0 + 3 >= K) v.w = 0.f;
       }
       ra[i] = v;
     }
@@ -164,9 +164,6 @@ k_gemm_tc(const float* __restrict__ A, int lda, const float* __restrict__ Bk, in
       float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
       if (nrow < N && k0 < K) {
         v = *reinterpret_cast<const float4*>(Bk + (long long)nrow * ldbk + k0);
-        if (k0 + 1 >= K) v.y = 0.f;
-        if (k0 + 2 >= K) v.z = 0.f;
-        if (k0 + 3 >= K) v.w = 0.f;
       }
       rb[i] = v;
     }
@@ -345,9 +342,6 @@ k_gemm_tc_resident(const float* __restrict__ A, int lda, const float* __restrict
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (nrow < n_loc && k0 < K) {
           v = *reinterpret_cast<const float4*>(Bk + (long long)(n0 + nrow) * ldbk + k0);
-          if (k0 + 1 >= K) v.y = 0.f;
-          if (k0 + 2 >= K) v.z = 0.f;
-          if (k0 + 3 >= K) v.w = 0.f;
         }
         float4 h, l;
         split_tf32(v.x, h.x, l.x); split_tf32(v.y, h.y, l.y); split_tf32(v.z, h.z, l.z); split_tf32(v.w, h.w, l.w);
@@ -594,9 +588,6 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (r < M && k0 < K) {
           v = *reinterpret_cast<const float4*>(A + r * lda + k0);
-          if (k0 + 1 >= K) v.y = 0.f;
-          if (k0 + 2 >= K) v.z = 0.f;
-          if (k0 + 3 >= K) v.w = 0.f;
         }
         pa[i] = v;
       }
@@ -606,9 +597,6 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (nrow < n_loc && k0 < K) {
           v = *reinterpret_cast<const float4*>(Bk + (long long)(n0 + nrow) * ldbk + k0);
-          if (k0 + 1 >= K) v.y = 0.f;
-          if (k0 + 2 >= K) v.z = 0.f;
-          if (k0 + 3 >= K) v.w = 0.f;
         }
         pb[i] = v;
       }
