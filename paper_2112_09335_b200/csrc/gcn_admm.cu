@@ -143,7 +143,7 @@ struct gcn_admm {
   size_t part_elems = 0;
   SearchCtl *ctl_w = nullptr, *ctl_z = nullptr;   // [L+1], [(L+1) * M]
   double *sums_w = nullptr, *sums_z = nullptr, *acc_w = nullptr, *acc_z = nullptr, *obj = nullptr;
-  int *n_active = nullptr, *status = nullptr;
+  int *n_active = nullptr, *status = nullptr, *row_counter = nullptr;
   int *log_trial_w = nullptr, *log_trial_z = nullptr;
   double *log_q_w = nullptr, *log_q_z = nullptr;
   long long log_count = 0;
@@ -416,12 +416,13 @@ struct gcn_admm {
   {                                                                                                       \
     if (dyn > 48 * 1024)                                                                                  \
       CU(cudaFuncSetAttribute(gk::k_score_z<V, OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn)); \
+    CU(cudaMemsetAsync(row_counter, 0, sizeof(int), stream));                                             \
     int occ = 1;                                                                                          \
     CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gk::k_score_z<V, OUT>, warps * 32, dyn));      \
     const unsigned grid = (unsigned)std::min<long long>(cdiv(n, warps), (long long)kSmCount * std::max(occ, 1)); \
     gk::k_score_z<V, OUT><<<grid, warps * 32, dyn, stream>>>(d_row_ptr, d_col, d_col_comm, d_dinv,        \
         (const float4*)B1, (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0, ld4, (int)n, ctl, M, \
-        acc_z, n_active, use_smem);                                                                       \
+        acc_z, n_active, use_smem, row_counter);                                                          \
   }
 #define SCORE_Z_ANY(OUT)                    \
   {                                         \
@@ -706,6 +707,7 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
   h->obj = h->alloc<double>(8);
   h->n_active = h->alloc<int>(1);
   h->status = h->alloc<int>(1);
+  h->row_counter = h->alloc<int>(1);
   h->log_trial_w = h->alloc<int>((size_t)kLogPasses * L);
   h->log_q_w = h->alloc<double>((size_t)kLogPasses * L);
   h->log_trial_z = h->alloc<int>((size_t)kLogPasses * std::max(L - 1, 0) * n_comm);

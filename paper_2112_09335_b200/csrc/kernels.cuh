@@ -735,14 +735,14 @@ __device__ __forceinline__ float warp_sum2(float v0, float v1, int lane) {
 //   OUT = true  (layer l+1 = L):        acc[m*2] += <k, R'>, acc[m*2+1] += ||k||^2   (closed form)
 // Sums are kept per warp in shared memory (no atomics on the hot path) and added to `acc` once per
 // block; with too many communities for that (use_smem == 0) they go to `acc` directly.
-// V = float4 columns per lane (width <= 128 V).  Persistent grid: rows are dealt to blocks round robin.
+// V = float4 columns per lane (width <= 128 V).  Persistent grid; `row_counter` must be zero at launch.
 template <int V, bool OUT>
 __global__ void __launch_bounds__(256)
 k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
           const unsigned short* __restrict__ col_comm, const float* __restrict__ dinv,
           const float4* __restrict__ T, const float4* __restrict__ Hn, const float4* __restrict__ Zn,
           const float4* __restrict__ Rn, int ld4, int n, const SearchCtl* __restrict__ ctl, int n_comm,
-          double* __restrict__ acc, const int* __restrict__ n_active, int use_smem) {
+          double* __restrict__ acc, const int* __restrict__ n_active, int use_smem, int* __restrict__ row_counter) {
   if (*n_active <= 0) return;
   constexpr int PER = OUT ? 2 : kCand;
   extern __shared__ double s_acc[];
@@ -754,7 +754,15 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
     __syncthreads();
     mine = s_acc + (size_t)warp * n_comm * PER;
   }
-  for (int row = blockIdx.x * warps_per_block + warp; row < n; row += gridDim.x * warps_per_block) {
+  // rows are handed out four at a time from a global counter: row lengths follow a power law, a
+  // static deal leaves most warps waiting at the closing barrier for the unlucky ones
+  for (;;) {
+    int row_base = 0;
+    if (lane == 0) row_base = atomicAdd(row_counter, 4);
+    row_base = __shfl_sync(0xffffffffu, row_base, 0);
+    if (row_base >= n) break;
+    const int row_end = min(n, row_base + 4);
+  for (int row = row_base; row < row_end; ++row) {
     float4 a[V], b[V];   // OUT: a = R' ; else a = h, b = z
 #pragma unroll
     for (int v = 0; v < V; ++v) {
@@ -866,6 +874,7 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
       }
     }
     finish_segment();
+  }
   }
   if (use_smem) {
     __syncthreads();
