@@ -134,6 +134,12 @@ int gcn_admm_propagate(gcn_admm* h, const float* x, int width, float* out);
 int gcn_admm_dense_product(gcn_admm* h, const float* A, const float* B, float* C, long long m, int n, int k,
                            int tensor_cores);
 
+/* C = A^T B for device pointers A (rows x ka), B (rows x nb), C (ka x nb): the reduction over the node
+ * dimension that forms the weight gradient P^T R (Section 3.1).  ka x (nb rounded up to 4) must fit
+ * the handle's partial-sum scratch (it does for every layer shape of the handle).  Synchronises. */
+int gcn_admm_dense_product_tn(gcn_admm* h, const float* A, const float* B, float* C, long long rows, int ka, int nb,
+                              int tensor_cores);
+
 /* ---- propagation for callers that cannot allocate ---------------------------------------------
  * (No counterpart in the paper: this is a packaging variant of gcn_admm_propagate.)
  * Same result as gcn_admm_propagate, for code that is not allowed to reserve device memory when it

@@ -18,7 +18,7 @@ EXPORTS = [
     "gcn_admm_default_params", "gcn_admm_create", "gcn_admm_step", "gcn_admm_objective", "gcn_admm_weights",
     "gcn_admm_predict", "gcn_admm_destroy", "gcn_admm_last_error", "gcn_admm_propagate", "gcn_admm_index",
     "gcn_admm_get_state", "gcn_admm_set_state", "gcn_admm_step_block", "gcn_admm_decisions",
-    "gcn_admm_launches", "gcn_admm_profile", "gcn_admm_profile_read", "gcn_admm_propagate_static", "gcn_admm_dense_product",
+    "gcn_admm_launches", "gcn_admm_profile", "gcn_admm_profile_read", "gcn_admm_propagate_static", "gcn_admm_dense_product", "gcn_admm_dense_product_tn",
 ]
 
 IX = dict(perm=0, inv_perm=1, comm_ptr=2, nbr=3, halo1=4, halo2=5, csr_row_ptr=6, csr_col=7,
@@ -67,6 +67,7 @@ def load():
     lib.gcn_admm_propagate.argtypes = [vp, vp, i32, vp]
     lib.gcn_admm_propagate_static.argtypes = [vp, vp, i32, vp]
     lib.gcn_admm_dense_product.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32]
+    lib.gcn_admm_dense_product_tn.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32]
     lib.gcn_admm_index.argtypes = [vp, i32, i32, C.POINTER(C.POINTER(i32)), C.POINTER(i64)]
     lib.gcn_admm_get_state.argtypes = [vp, i32, i32, vp]
     lib.gcn_admm_set_state.argtypes = [vp, i32, i32, vp]
@@ -183,6 +184,11 @@ class GcnAdmm:
         """C = A B between dense device buffers (addresses as ints)."""
         self._check(self._lib.gcn_admm_dense_product(self._h, _ptr(int(a_dev)), _ptr(int(b_dev)), _ptr(int(c_dev)), int(m),
                                                      int(n), int(k), int(tensor_cores)))
+
+    def dense_product_tn(self, a_dev, b_dev, c_dev, rows, ka, nb, tensor_cores=1):
+        """C = A^T B between dense device buffers (addresses as ints): A rows x ka, B rows x nb."""
+        self._check(self._lib.gcn_admm_dense_product_tn(self._h, _ptr(int(a_dev)), _ptr(int(b_dev)), _ptr(int(c_dev)),
+                                                        int(rows), int(ka), int(nb), int(tensor_cores)))
 
     def index(self, which, comm=0):
         data = C.POINTER(C.c_int)()

@@ -275,6 +275,34 @@ struct gcn_admm {
     int splits = 1;
     long long rps = rows;
     char name[48];
+    if (p.tensor_cores == 1 && Nb <= 256 && rows >= 4096) {
+      std::snprintf(name, sizeof name, "gemm_tn_tc@%dx%d", Ka, Nb);
+      Scope sc(this, name, 2, 4.0 * ((double)rows * (lda + ldb) + (double)Ka * ldp), 2.0 * (double)rows * Ka * Nb);
+      const int groups = (int)cdiv(Ka, gtc::kBlockM);
+      splits = (int)std::max<long long>(1, std::min<long long>(kSmCount / groups, cdiv(rows, 256)));
+      splits = (int)std::min<long long>(splits, (long long)(part_elems / ((size_t)Ka * ldp)));
+      rps = cdiv(rows, splits);
+      splits = (int)cdiv(rows, rps);
+#define TN_TC(NT)                                                                                              \
+  {                                                                                                            \
+    const size_t smem = gtc::TnCfg<NT>::kSmem;                                                                 \
+    CU(cudaFuncSetAttribute(gtc::k_gemm_tn_tc<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));   \
+    dim3 grid((unsigned)splits, (unsigned)groups);                                                             \
+    gtc::k_gemm_tn_tc<NT><<<grid, gtc::kTnThreads, smem, stream>>>(A, lda, B, ldb, part, ldp, rows, rps, Ka, Nb, tc_error); \
+  }
+      if (Nb <= 16) TN_TC(16)
+      else if (Nb <= 32) TN_TC(32)
+      else if (Nb <= 48) TN_TC(48)
+      else if (Nb <= 64) TN_TC(64)
+      else if (Nb <= 128) TN_TC(128)
+      else TN_TC(256)
+#undef TN_TC
+      CU(cudaGetLastError());
+      const long long elems_tc = (long long)Ka * ldp;
+      gk::k_reduce_splits<<<(unsigned)cdiv(elems_tc, 256), 256, 0, stream>>>(part, out, elems_tc, splits);
+      CU(cudaGetLastError());
+      return;
+    }
     std::snprintf(name, sizeof name, "gemm_tn@%dx%d", Ka, Nb);
     Scope sc(this, name, 2, 4.0 * ((double)rows * (lda + ldb) + (double)Ka * ldp), 2.0 * (double)rows * Ka * Nb);
 #define TN_CASE(BM, BN, BK, TM, TN)                                                             \
@@ -1005,6 +1033,39 @@ int gcn_admm_dense_product(gcn_admm* h, const float* A, const float* B, float* C
       throw;
     }
     cudaFree(a); cudaFree(b); cudaFree(bk); cudaFree(c);
+    h->check_status();
+  });
+}
+
+int gcn_admm_dense_product_tn(gcn_admm* h, const float* A, const float* B, float* C, long long rows, int ka, int nb,
+                              int tensor_cores) {
+  return guarded(h, [&] {
+    if (!A || !B || !C || rows < 1 || ka < 1 || nb < 1) throw Fail{GCN_ADMM_ERR_ARG, "bad argument"};
+    if (!is_device_pointer(A) || !is_device_pointer(B) || !is_device_pointer(C))
+      throw Fail{GCN_ADMM_ERR_ARG, "A, B and C must be device pointers"};
+    const int lda = ldpad(ka), ldb = ldpad(nb), ldp = ldpad(nb);
+    if ((size_t)ka * ldp > h->part_elems) throw Fail{GCN_ADMM_ERR_ARG, "ka x nb exceeds the handle's partial-sum scratch"};
+    float *a = nullptr, *b = nullptr, *c = nullptr;
+    const int saved = h->p.tensor_cores;
+    try {
+      a = dalloc<float>((size_t)rows * lda);
+      b = dalloc<float>((size_t)rows * ldb);
+      c = dalloc<float>((size_t)ka * ldp);
+      CU(cudaMemsetAsync(a, 0, (size_t)rows * lda * 4, h->stream));
+      CU(cudaMemsetAsync(b, 0, (size_t)rows * ldb * 4, h->stream));
+      CU(cudaMemcpy2DAsync(a, (size_t)lda * 4, A, (size_t)ka * 4, (size_t)ka * 4, (size_t)rows, cudaMemcpyDeviceToDevice, h->stream));
+      CU(cudaMemcpy2DAsync(b, (size_t)ldb * 4, B, (size_t)nb * 4, (size_t)nb * 4, (size_t)rows, cudaMemcpyDeviceToDevice, h->stream));
+      h->p.tensor_cores = tensor_cores;
+      h->gemm_tn(a, lda, b, ldb, c, ldp, rows, ka, nb);
+      h->p.tensor_cores = saved;
+      CU(cudaMemcpy2DAsync(C, (size_t)nb * 4, c, (size_t)ldp * 4, (size_t)nb * 4, (size_t)ka, cudaMemcpyDeviceToDevice, h->stream));
+      CU(cudaStreamSynchronize(h->stream));
+    } catch (...) {
+      h->p.tensor_cores = saved;
+      cudaFree(a); cudaFree(b); cudaFree(c);
+      throw;
+    }
+    cudaFree(a); cudaFree(b); cudaFree(c);
     h->check_status();
   });
 }

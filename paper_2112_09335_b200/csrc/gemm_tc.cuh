@@ -700,6 +700,214 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Transposed product on the tensor cores:  part[s][Ka x Nb] = sum over the rows of split s of
+// A[r,:]^T B[r,:]  (the weight gradient P^T R, reduction over the node dimension).
+// Here the reduction index r is the MMA's K, and both operands are stored with their own index
+// (ka, nb) contiguous: "MN-major" operands.  A chunk is 32 rows; in shared memory it is laid out as
+// 128-byte swizzle rows of 32 consecutive columns: atom (g, q) holds rows 8q..8q+7 of column group g
+// (32 columns), 1024 bytes; successive column groups are 4096 bytes apart (the descriptor's leading
+// byte offset), successive groups of 8 rows 1024 bytes apart (its stride byte offset).  One MMA
+// consumes 8 rows (K = 8).  Same hi/lo split, same separate correction accumulator, same roles as
+// above (8 producer warps, one MMA warp); a CTA owns 128 columns of A (blockIdx.y) and one row
+// split (blockIdx.x) and writes its 128 x NT partial sum once, at the end.
+// ------------------------------------------------------------------------------------------------
+constexpr int kTnThreads = 9 * 32;
+constexpr int kTnRows = 32;                       // rows (reduction steps) per chunk
+
+__device__ __forceinline__ uint64_t operand_desc_mn(uint32_t smem_addr) {
+  const uint32_t lo = ((smem_addr >> 4) & 0x3fffu) | ((4096u >> 4) << 16);   // start address, LBO = 4096
+  const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);                // SBO = 1024, version 1, SWIZZLE_128B
+  return ((uint64_t)hi << 32) | lo;
+}
+__device__ __forceinline__ uint32_t instr_desc_mn(int nt) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(nt >> 3) << 17) |
+         ((uint32_t)(kBlockM >> 4) << 24);
+}
+// byte offset of float4 number c4 (columns 4 c4 .. 4 c4 + 3) of chunk row r in an MN-major tile
+__device__ __forceinline__ uint32_t swz_mn(int r, int c4) {
+  return (uint32_t)(c4 >> 3) * 4096u + (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u +
+         (uint32_t)(((c4 & 7) ^ (r & 7)) << 4);
+}
+
+template <int NT>
+struct TnCfg {
+  static constexpr int kGroupsB = (NT + 31) / 32;
+  static constexpr int kATile = 4 * 4096;                 // 128 columns x 32 rows, one of hi / lo
+  static constexpr int kBTile = kGroupsB * 4096;
+  static constexpr int kStage = 2 * kATile + 2 * kBTile;
+  static constexpr int kStagesTn = kStage > 72 * 1024 ? 2 : 3;
+  static constexpr uint32_t kTmemCols = 2 * NT <= 32 ? 32 : 2 * NT <= 64 ? 64 : 2 * NT <= 128 ? 128 : 2 * NT <= 256 ? 256 : 512;
+  static constexpr size_t kSmem = (size_t)kStagesTn * kStage + 1024;
+};
+
+template <int NT>
+__global__ void __launch_bounds__(kTnThreads, 1)
+k_gemm_tn_tc(const float* __restrict__ A, int lda, const float* __restrict__ B, int ldb, float* __restrict__ part, int ldp,
+             long long rows, long long rows_per_split, int Ka, int Nb, int* __restrict__ error_flag) {
+  using Cfg = TnCfg<NT>;
+  constexpr int S = Cfg::kStagesTn;
+  constexpr int A_PASSES = 4;                              // 1024 float4 / 256 threads
+  constexpr int B_F4 = kTnRows * (NT / 4);
+  constexpr int B_PASSES = (B_F4 + 255) / 256;
+  static_assert(NT % 16 == 0 && NT <= 256, "NT");
+
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2 * S + 1];       // full[S], empty[S], acc_full
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t smem_base = smem_u32(smem);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[S]), bar_acc = smem_u32(&bars[2 * S]);
+
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 256); mbar_init(bar_empty + 8 * s, 1); }
+    mbar_init(bar_acc, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                 "r"(Cfg::kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = tmem_base_slot;
+  volatile int* abortp = &abort_flag;
+
+  const long long r_begin = (long long)blockIdx.x * rows_per_split;
+  const long long r_end = min(rows, r_begin + rows_per_split);
+  const int total = r_end > r_begin ? (int)((r_end - r_begin + kTnRows - 1) / kTnRows) : 0;
+  const int ka0 = blockIdx.y * kBlockM;
+
+  if (warp < 8) {
+    // ---------------- producers ----------------
+    float4 ra[2][A_PASSES], rb[2][B_PASSES];
+    auto load_chunk = [&](int j, float4* pa, float4* pb) {
+      if (j >= total) return;
+      const long long r0 = r_begin + (long long)j * kTnRows;
+#pragma unroll
+      for (int i = 0; i < A_PASSES; ++i) {
+        const int f = tid + 256 * i, rr = f >> 5, c4 = f & 31;
+        const long long r = r0 + rr;
+        const int col = ka0 + 4 * c4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (r < r_end && col < Ka) v = *reinterpret_cast<const float4*>(A + r * lda + col);   // zero padding beyond Ka
+        pa[i] = v;
+      }
+#pragma unroll
+      for (int i = 0; i < B_PASSES; ++i) {
+        const int f = tid + 256 * i;
+        const int rr = f / (NT / 4), c4 = f % (NT / 4);
+        const long long r = r0 + rr;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (f < B_F4 && r < r_end && 4 * c4 < Nb) v = *reinterpret_cast<const float4*>(B + r * ldb + 4 * c4);
+        pb[i] = v;
+      }
+    };
+    auto store_chunk = [&](int stage, const float4* pa, const float4* pb) {
+      uint8_t* st = smem + (size_t)stage * Cfg::kStage;
+#pragma unroll
+      for (int i = 0; i < A_PASSES; ++i) {
+        const int f = tid + 256 * i, rr = f >> 5, c4 = f & 31;
+        float4 h, l;
+        split_tf32(pa[i].x, h.x, l.x); split_tf32(pa[i].y, h.y, l.y);
+        split_tf32(pa[i].z, h.z, l.z); split_tf32(pa[i].w, h.w, l.w);
+        const uint32_t off = swz_mn(rr, c4);
+        *reinterpret_cast<float4*>(st + off) = h;
+        *reinterpret_cast<float4*>(st + Cfg::kATile + off) = l;
+      }
+#pragma unroll
+      for (int i = 0; i < B_PASSES; ++i) {
+        const int f = tid + 256 * i;
+        if (f < B_F4) {
+          const int rr = f / (NT / 4), c4 = f % (NT / 4);
+          float4 h, l;
+          split_tf32(pb[i].x, h.x, l.x); split_tf32(pb[i].y, h.y, l.y);
+          split_tf32(pb[i].z, h.z, l.z); split_tf32(pb[i].w, h.w, l.w);
+          const uint32_t off = swz_mn(rr, c4);
+          *reinterpret_cast<float4*>(st + 2 * Cfg::kATile + off) = h;
+          *reinterpret_cast<float4*>(st + 2 * Cfg::kATile + Cfg::kBTile + off) = l;
+        }
+      }
+    };
+    load_chunk(0, ra[0], rb[0]);
+    load_chunk(1, ra[1], rb[1]);
+    for (int j = 0; j < total; ++j) {
+      const int stage = j % S;
+      if (j >= S && !mbar_wait_abortable(bar_empty + 8 * stage, ((j / S) - 1) & 1, abortp)) break;
+      if (j & 1) { store_chunk(stage, ra[1], rb[1]); load_chunk(j + 2, ra[1], rb[1]); }
+      else       { store_chunk(stage, ra[0], rb[0]); load_chunk(j + 2, ra[0], rb[0]); }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_arrive(bar_full + 8 * stage);
+    }
+  } else if (lane == 0) {
+    // ---------------- MMA issue ----------------
+    const uint32_t idesc = instr_desc_mn(NT);
+    for (int j = 0; j < total; ++j) {
+      const int stage = j % S;
+      if (!mbar_wait_abortable(bar_full + 8 * stage, (j / S) & 1, abortp)) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t a_hi = smem_base + stage * Cfg::kStage, a_lo = a_hi + Cfg::kATile;
+      const uint32_t b_hi = a_hi + 2 * Cfg::kATile, b_lo = b_hi + Cfg::kBTile;
+#pragma unroll
+      for (int ks = 0; ks < kTnRows / 8; ++ks) {
+        const uint32_t o = ks * 1024;              // the next group of 8 rows
+        const uint32_t first = (j > 0 || ks > 0) ? 1u : 0u;
+        mma_tf32(tmem_base + NT, operand_desc_mn(a_lo + o), operand_desc_mn(b_hi + o), idesc, first);   // corrections
+        mma_tf32(tmem_base + NT, operand_desc_mn(a_hi + o), operand_desc_mn(b_lo + o), idesc, 1u);
+        mma_tf32(tmem_base, operand_desc_mn(a_hi + o), operand_desc_mn(b_hi + o), idesc, first);        // main product
+      }
+      mma_commit(bar_empty + 8 * stage);
+      if (j + 1 == total) mma_commit(bar_acc);
+    }
+  }
+  __syncwarp();
+  // ---------------- epilogue: warps 0-3, one tensor-memory lane (= column of A) per thread ----------------
+  if (warp < 4) {
+    bool ok = true;
+    if (total > 0) ok = mbar_wait_abortable(bar_acc, 0, abortp);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const int ka = ka0 + warp * 32 + lane;
+    float* dst = part + ((long long)blockIdx.x * Ka + ka) * ldp;
+#pragma unroll 1
+    for (int cchunk = 0; cchunk < NT / 16; ++cchunk) {
+      uint32_t v[16], w[16];
+#pragma unroll
+      for (int q = 0; q < 16; ++q) v[q] = w[q] = 0u;
+      if (ok && total > 0) {
+        const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(cchunk * 16);
+        GTC_TMEM_LD16(v, taddr);
+        GTC_TMEM_LD16(w, taddr + (uint32_t)NT);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      }
+      if (ka < Ka) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int col = cchunk * 16 + q * 4;
+          if (col < ldp)
+            *reinterpret_cast<float4*>(dst + col) =
+                make_float4(__uint_as_float(v[q * 4]) + __uint_as_float(w[q * 4]),
+                            __uint_as_float(v[q * 4 + 1]) + __uint_as_float(w[q * 4 + 1]),
+                            __uint_as_float(v[q * 4 + 2]) + __uint_as_float(w[q * 4 + 2]),
+                            __uint_as_float(v[q * 4 + 3]) + __uint_as_float(w[q * 4 + 3]));
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (tid == 0 && abort_flag) atomicExch(error_flag, 1);
+  if (warp == 8) {
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(Cfg::kTmemCols) : "memory");
+  }
+}
+
 // dynamic shared memory of k_gemm_tc<NT>
 template <int NT>
 constexpr size_t smem_bytes() { return (size_t)kStages * (2 * kATileBytes + 2 * NT * kChunkK * 4) + 1024; }

@@ -39,3 +39,30 @@ def test_dense_product_against_fp64(handle, m, n, k, tensor_cores):
     assert np.isfinite(got).all()
     assert worst < 2e-6
     assert rel < 3e-6
+
+
+TN_SHAPES = [(50000, 128, 16), (30011, 256, 256), (20000, 100, 256), (40001, 256, 47), (8192, 128, 7), (100000, 16, 7),
+             (4096, 300, 40), (5000, 37, 129)]    # (rows, ka, nb)
+
+
+@pytest.mark.parametrize("tensor_cores", [1, 0])
+@pytest.mark.parametrize("rows,ka,nb", TN_SHAPES)
+def test_transposed_product_against_fp64(handle, rows, ka, nb, tensor_cores):
+    import torch
+    if ka * ((nb + 3) // 4 * 4) > 128 * 16 * 4 * 148:
+        pytest.skip("larger than this handle's partial-sum scratch")
+    rng = np.random.default_rng(rows + ka + nb)
+    a = rng.standard_normal((rows, ka)).astype(np.float32)
+    b = (rng.standard_normal((rows, nb)) * rng.choice([1e-3, 1.0, 30.0], size=(1, nb))).astype(np.float32)
+    ta, tb = torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda()
+    tc = torch.full((ka, nb), float("nan"), device="cuda")
+    handle.dense_product_tn(ta.data_ptr(), tb.data_ptr(), tc.data_ptr(), rows, ka, nb, tensor_cores)
+    got = tc.cpu().numpy().astype(np.float64)
+    want = a.astype(np.float64).T @ b.astype(np.float64)
+    scale = np.abs(a).astype(np.float64).T @ np.abs(b).astype(np.float64) + 1e-300
+    worst = float(np.max(np.abs(got - want) / scale))
+    rel = float(np.linalg.norm(got - want) / np.linalg.norm(want))
+    print(f"\n  rows={rows} ka={ka} nb={nb} tc={tensor_cores}: rel {rel:.2e}, worst elementwise/sum|a||b| {worst:.2e}")
+    assert np.isfinite(got).all()
+    assert worst < 2e-6
+    assert rel < 2e-4      # the sum over many rows cancels: relative to ||C|| the bound is loose, `worst` is the sharp one
