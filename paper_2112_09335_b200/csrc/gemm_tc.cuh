@@ -704,11 +704,12 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
 // Transposed product on the tensor cores:  part[s][Ka x Nb] = sum over the rows of split s of
 // A[r,:]^T B[r,:]  (the weight gradient P^T R, reduction over the node dimension).
 // Here the reduction index r is the MMA's K, and both operands are stored with their own index
-// (ka, nb) contiguous: "MN-major" operands.  A chunk is 32 rows; in shared memory it is laid out as
-// 128-byte swizzle rows of 32 consecutive columns: atom (g, q) holds rows 8q..8q+7 of column group g
-// (32 columns), 1024 bytes; successive column groups are 4096 bytes apart (the descriptor's leading
-// byte offset), successive groups of 8 rows 1024 bytes apart (its stride byte offset).  One MMA
-// consumes 8 rows (K = 8).  Same hi/lo split, same separate correction accumulator, same roles as
+// (ka, nb) contiguous: "MN-major" operands, for which 32-bit elements have exactly one shared-memory
+// form: 128-byte rows swizzled at 32-byte granularity.  A chunk is 32 rows; atom (g, q) holds rows
+// 4q..4q+3 of column group g (32 columns = 128 bytes per row), 512 bytes, and inside it the 32-byte
+// unit u of row r sits at unit u ^ (r mod 4); successive column groups are 4096 bytes apart (the
+// descriptor's leading byte offset), successive groups of 4 rows 512 bytes apart (its stride byte
+// offset).  One MMA consumes 8 rows (K = 8), i.e. two atoms.  Same hi/lo split, same separate correction accumulator, same roles as
 // above (8 producer warps, one MMA warp); a CTA owns 128 columns of A (blockIdx.y) and one row
 // split (blockIdx.x) and writes its 128 x NT partial sum once, at the end.
 // ------------------------------------------------------------------------------------------------
@@ -717,7 +718,7 @@ constexpr int kTnRows = 32;                       // rows (reduction steps) per 
 
 __device__ __forceinline__ uint64_t operand_desc_mn(uint32_t smem_addr) {
   const uint32_t lo = ((smem_addr >> 4) & 0x3fffu) | ((4096u >> 4) << 16);   // start address, LBO = 4096
-  const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);                // SBO = 1024, version 1, SWIZZLE_128B
+  const uint32_t hi = (512u >> 4) | (1u << 14) | (1u << 29);                 // SBO = 512, version 1, 128B swizzle / 32B base
   return ((uint64_t)hi << 32) | lo;
 }
 __device__ __forceinline__ uint32_t instr_desc_mn(int nt) {
@@ -726,8 +727,8 @@ __device__ __forceinline__ uint32_t instr_desc_mn(int nt) {
 }
 // byte offset of float4 number c4 (columns 4 c4 .. 4 c4 + 3) of chunk row r in an MN-major tile
 __device__ __forceinline__ uint32_t swz_mn(int r, int c4) {
-  return (uint32_t)(c4 >> 3) * 4096u + (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u +
-         (uint32_t)(((c4 & 7) ^ (r & 7)) << 4);
+  return (uint32_t)(c4 >> 3) * 4096u + (uint32_t)(r >> 2) * 512u + (uint32_t)(r & 3) * 128u +
+         (uint32_t)(((((c4 & 7) >> 1) ^ (r & 3)) << 5) | ((c4 & 1) << 4));
 }
 
 template <int NT>
