@@ -210,7 +210,8 @@ struct gcn_admm {
         else if (N <= 32) TC_WS(32)
         else if (N <= 48) TC_WS(48)
         else if (N <= 64) TC_WS(64)
-        else TC_WS(128)
+        else if (N <= 128) TC_WS(128)
+        else TC_WS(256)
 #undef TC_WS
         CU(cudaGetLastError());
         return;

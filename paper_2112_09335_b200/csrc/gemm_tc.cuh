@@ -491,8 +491,9 @@ inline size_t resident_smem_bytes(int K) {
 //               arrive on acc_empty[set]  (warp w reads lanes 32 (w mod 4) .. +31)
 //   warp 12     MMA: waits full[stage] (and, at the first chunk of a tile, acc_empty[set]), issues
 //               the twelve MMAs, commits to empty[stage] and, at the last chunk, to acc_full[set]
-// Two accumulator sets (main + correction each) alternate between consecutive tiles, so NT <= 128
-// (4 NT <= 512 columns of tensor memory); wider outputs use two column groups.
+// Up to 128 output columns, two accumulator sets (main + correction each) alternate between consecutive
+// tiles (4 NT <= 512 columns of tensor memory); from 129 to 256 columns there is room for one set, and
+// the MMAs of the next tile wait for the epilogue of the current one while the producers keep staging.
 // A wait that runs out raises a shared abort flag that every other wait polls; all roles then meet
 // at the closing barrier and tensor memory is released.
 // ------------------------------------------------------------------------------------------------
@@ -520,10 +521,12 @@ __device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parit
 
 template <int NT>
 struct WsCfg {
-  static constexpr int kStagesWs = NT > 64 ? 3 : 4;
+  static constexpr int kSets = NT > 128 ? 1 : 2;                        // accumulator sets (main + correction each)
+  static constexpr int kStagesWs = NT > 128 ? 2 : NT > 64 ? 3 : 4;
   static constexpr int kBTile = NT * kChunkK * 4;                       // one of hi / lo
   static constexpr int kStage = 2 * kATileBytes + 2 * kBTile;
-  static constexpr uint32_t kTmemCols = 4 * NT <= 64 ? 64 : 4 * NT <= 128 ? 128 : 4 * NT <= 256 ? 256 : 512;
+  static constexpr int kAccCols = kSets * 2 * NT;
+  static constexpr uint32_t kTmemCols = kAccCols <= 64 ? 64 : kAccCols <= 128 ? 128 : kAccCols <= 256 ? 256 : 512;
   static constexpr size_t kSmem = (size_t)kStagesWs * kStage + 1024;
 };
 
@@ -535,7 +538,8 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
   constexpr int S = Cfg::kStagesWs;
   constexpr int B_PASSES = (NT + 31) / 32;
   constexpr int A_PASSES = kBlockM / 32;
-  static_assert(NT <= 128 && NT % 16 == 0, "NT");
+  constexpr int SETS = Cfg::kSets;
+  static_assert(NT <= 256 && NT % 16 == 0, "NT");
   if (skip != nullptr && *skip) return;
 
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -640,8 +644,8 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
     if (lane == 0) {
       const uint32_t idesc = instr_desc(NT);
       for (int j = 0; j < total; ++j) {
-        const int stage = j % S, kc = j % kc_count, tile_i = j / kc_count, set = tile_i & 1;
-        if (kc == 0 && tile_i >= 2 && !mbar_wait_abortable(bar_acc_empty + 8 * set, ((tile_i >> 1) - 1) & 1, abortp)) break;
+        const int stage = j % S, kc = j % kc_count, tile_i = j / kc_count, set = tile_i % SETS;
+        if (kc == 0 && tile_i >= SETS && !mbar_wait_abortable(bar_acc_empty + 8 * set, ((tile_i / SETS) - 1) & 1, abortp)) break;
         if (!mbar_wait_abortable(bar_full + 8 * stage, (j / S) & 1, abortp)) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t a_hi = smem_base + stage * Cfg::kStage, a_lo = a_hi + kATileBytes;
@@ -663,8 +667,8 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
     // ---------------- epilogue ----------------
     const int quarter = warp & 3;
     for (int tile_i = 0; tile_i < my_tiles; ++tile_i) {
-      const int set = tile_i & 1;
-      if (!mbar_wait_abortable(bar_acc_full + 8 * set, (tile_i >> 1) & 1, abortp)) break;
+      const int set = tile_i % SETS;
+      if (!mbar_wait_abortable(bar_acc_full + 8 * set, (tile_i / SETS) & 1, abortp)) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const long long row = (long long)(blockIdx.x + tile_i * gridDim.x) * kBlockM + quarter * 32 + lane;
 #pragma unroll 1
