@@ -1,0 +1,94 @@
+"""The largest workload at full size (2.45 M nodes, ~62 M edges, 100-256-256-47, 64 communities), in the
+launch configuration bench.py times.  A full oracle pass is out of reach there, so sampled outputs are
+checked against rows the fp64 oracle computes one by one (oracle/sampled_rows.py): propagation rows, the
+hidden Z block updates (given the accepted theta, whose decision is logged), the output-layer rows and
+the dual rows; plus properties that hold at any size (no exhausted search, every accepted q >= 1)."""
+import numpy as np
+import pytest
+
+from oracle.sampled_rows import SampledRows
+from paper_2112_09335_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def rows_close(got, want, scale, tol):
+    err = np.abs(np.asarray(got, dtype=np.float64) - want)
+    return float(np.max(err / (scale + 1e-30))), tol
+
+
+def test_sampled_rows_at_full_size():
+    import torch
+    wl = inputs.make_workload(4)
+    g = binding.GcnAdmm(wl.n, wl.row_ptr, wl.col_idx, wl.X, wl.y, wl.train_mask, wl.widths, wl.n_comm, wl.community,
+                        wl.w_init, nu=wl.nu, rho=wl.rho)
+    try:
+        L, M = len(wl.widths) - 1, wl.n_comm
+        sr = SampledRows(wl.n, wl.row_ptr, wl.col_idx, wl.y, wl.train_mask, wl.widths, wl.nu, wl.rho)
+        rng = np.random.default_rng(5)
+        deg = np.diff(wl.row_ptr)
+        train_rows = np.flatnonzero(wl.train_mask)
+        rows = np.unique(np.concatenate([rng.choice(wl.n, 12, replace=False), rng.choice(train_rows, 4, replace=False),
+                                         [int(np.argmax(deg)), int(np.argmin(deg))]]))
+        # ---- propagation rows ----
+        x = torch.randn(wl.n, 32, device="cuda", generator=torch.Generator(device="cuda").manual_seed(1))
+        out = torch.empty_like(x)
+        g.propagate(x.data_ptr(), 32, out=out.data_ptr())
+        torch.cuda.synchronize()
+        xh = x.cpu().numpy()
+        want = sr.propagate_rows(xh, rows)
+        mag = np.zeros_like(want)
+        for k, i in enumerate(rows):
+            c, v = sr.adj_row(int(i))
+            mag[k] = v @ np.abs(xh[c])
+        worst, _ = rows_close(out[torch.from_numpy(rows).cuda()].cpu().numpy(), want, mag, 0)
+        assert worst < 2e-6, worst
+        del x, out, xh
+
+        # ---- a state with every term active: three passes from the forward start ----
+        g.step(3)
+        dec = g.decisions()
+        assert (dec["trial_w"] != -2).all() and (dec["trial_z"] != -2).all()
+        ok = dec["trial_w"] >= 0
+        assert (dec["q_w"][ok] >= 1.0).all()
+        okz = dec["trial_z"] >= 0
+        assert (dec["q_z"][okz] >= 1.0).all()
+
+        def fetch():
+            Z = [wl.X] + [g.get_state(binding.ST_Z, l) for l in range(1, L + 1)]
+            W = [None] + [g.get_state(binding.ST_W, l) for l in range(1, L + 1)]
+            return Z, W, g.get_state(binding.ST_U)
+
+        report = {}
+        for l in range(1, L):                      # hidden Z blocks: Z_new = Z - grad / theta_{comm(row)}
+            Z, W, U = fetch()
+            g.step_block(binding.PHASE_Z, l)
+            theta = g.get_state(binding.ST_THETA, l)
+            trial = g.decisions()["trial_z"][0, l - 1]
+            got = g.get_state(binding.ST_Z, l)[rows]
+            grad = sr.grad_Z_rows(l, rows, Z, W, U)
+            comm = wl.community[rows]
+            stepped = trial[comm] >= 0
+            want = Z[l][rows].astype(np.float64) - np.where(stepped[:, None], grad / theta[comm][:, None], 0.0)
+            assert stepped.any()
+            rel = np.linalg.norm(got - want) / np.linalg.norm(want)
+            rel_step = np.linalg.norm((got - Z[l][rows]) - (want - Z[l][rows])) / max(np.linalg.norm(want - Z[l][rows]), 1e-300)
+            report[f"Z{l}"] = (rel, rel_step)
+            assert rel < 1e-5 and rel_step < 5e-3, (l, rel, rel_step)
+        Z, W, U = fetch()                            # output layer rows, Eq. (7)
+        g.step_block(binding.PHASE_Z, L)
+        got = g.get_state(binding.ST_Z, L)[rows]
+        want = sr.ZL_rows(rows, Z, W, U)
+        rel = np.linalg.norm(got - want) / np.linalg.norm(want)
+        report[f"Z{L}"] = (rel, 0.0)
+        assert rel < 1e-5, rel
+        Z, W, U = fetch()                            # dual rows, Eq. (3)
+        g.step_block(binding.PHASE_U, 0)
+        got = g.get_state(binding.ST_U)[rows]
+        want = sr.U_rows(rows, Z, W, U)
+        rel = np.linalg.norm(got - want) / np.linalg.norm(want)
+        report["U"] = (rel, 0.0)
+        assert rel < 1e-5, rel
+        print("\n  full size, sampled rows:", {k: (f"{a:.1e}", f"{b:.1e}") for k, (a, b) in report.items()})
+    finally:
+        g.destroy()

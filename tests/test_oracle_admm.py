@@ -381,3 +381,22 @@ def test_large_nu_pulls_hidden_layers_to_the_network():
         o.iterate()
     target = np.maximum((o.At @ o.Z[0]) @ o.W[1], 0)
     assert np.linalg.norm(o.Z[1] - target) < 0.5 * before
+
+
+def test_sampled_row_evaluator_matches_the_full_oracle():
+    """oracle/sampled_rows.py (used where a full pass is out of reach) against the full oracle."""
+    from oracle.sampled_rows import SampledRows
+    pr, o = make(31)
+    sr = SampledRows(pr["n"], pr["row_ptr"], pr["col_idx"], pr["y"], pr["mask"], pr["widths"], o.p.nu, o.p.rho)
+    rows = np.arange(pr["n"])
+    At = dense_At(pr)
+    np.testing.assert_allclose(sr.propagate_rows(o.Z[1], rows), At @ o.Z[1], atol=1e-13)
+    for l in range(1, o.L + 1):
+        np.testing.assert_allclose(sr.H_rows(l, rows, o.Z, o.W), At @ o.Z[l - 1] @ o.W[l], atol=1e-12)
+    for l in range(1, o.L):
+        full = np.zeros_like(o.Z[l])
+        for m in range(o.M):
+            full[o.V[m]] = o.grad_psi(l, m)
+        np.testing.assert_allclose(sr.grad_Z_rows(l, rows, o.Z, o.W, o.U), full, atol=1e-12)
+    np.testing.assert_allclose(sr.ZL_rows(rows, o.Z, o.W, o.U), o.update_ZL(o.W), atol=1e-12)
+    np.testing.assert_allclose(sr.U_rows(rows, o.Z, o.W, o.U), o.update_U(o.W, o.Z), atol=1e-13)
