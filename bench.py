@@ -162,6 +162,22 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def max_over_ranks(value, dist, device):
+    """Largest `value` over the ranks of the default process group (the value itself without one)."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(steps, ms, world):
+    """Whole-job iterations per second of `world` independent replicas that each ran `steps` iterations,
+    timed as the slowest replica's `ms`."""
+    return world * steps / (ms * 1e-3)
+
+
 def kernel_table(prof, iters, peaks):
     """Per kernel kind: launches and ms per iteration, achieved GB/s and TFLOP/s on algorithmic work."""
     rows = []
@@ -225,10 +241,7 @@ def run_ours(args):
     ms = ev0.elapsed_time(ev1)
     launches = g.launches() - launches0
     clocks = sampler.stop() if rank == 0 else None
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, dist, "cuda")
     obj = g.objective()
     dec = g.decisions()
     exhausted = int((dec["trial_w"] == -2).sum() + (dec["trial_z"] == -2).sum())
@@ -261,10 +274,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
     d2h = sum(w.nbytes for w in ws) + 48
-    if dist is not None:
-        t = torch.tensor([e2e_s], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = max_over_ranks(e2e_s, dist, "cuda")
     g2.destroy()
 
     if rank != 0:
@@ -272,7 +282,7 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    value = world * args.steps / (ms * 1e-3)
+    value = aggregate_value(args.steps, ms, world)
     dominant = table[0]
     alu_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12   # fp32 FMA TFLOP/s
     if dominant["kernel"].startswith("gemm"):
