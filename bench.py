@@ -285,19 +285,27 @@ def run_ours(args):
     value = aggregate_value(args.steps, ms, world)
     dominant = table[0]
     alu_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12   # fp32 FMA TFLOP/s
-    if dominant["kernel"].startswith("gemm"):
-        roofline = dict(bound="alu", achieved=dominant["tflops"], peak=alu_peak, unit="TFLOP/s",
-                        frac=dominant["tflops"] / alu_peak, traffic=None,
-                        peak_source="148 SMs x 128 fp32 lanes x 2 flop x max SM clock")
-    else:
-        traffic = None
-        if dominant["kernel"] == "spmm@256":
-            traffic = NCU_SPMM256["dram_bytes"] * (2 * wl.n_edges + wl.n) / NCU_SPMM256["nnz"]
-        roofline = dict(bound="hbm", achieved=dominant["gbs"], peak=peaks["hbm_gbs"], unit="GB/s",
-                        frac=dominant["gbs"] / peaks["hbm_gbs"], traffic=traffic, peak_source=peaks["source"],
-                        note=("gather kernel: every stored entry pulls a full operand row through L2 (nnz x ld x 4 B, "
-                              "about 23x the algorithmic bytes at mean degree 50), so it runs at the L2-to-SM rate, "
-                              "not at the HBM rate; algorithmic bytes = 4 nnz + 8 N + 8 N ld"))
+    # fp32-equivalent peak of the three-pass TF32 product: TF32 dense = bf16 dense x (1.1 / 2.25) nominal ratio, / 3
+    tc_peak = peaks["bf16_tflops"] * (1.1 / 2.25) / 3.0
+
+    def bound_of(row):
+        k = row["kernel"]
+        if k.startswith("gemm_tc") or k.startswith("gemm_tn_tc"):
+            return "tensor", row["tflops"], tc_peak, "TFLOP/s"
+        if k.startswith("gemm"):
+            return "alu", row["tflops"], alu_peak, "TFLOP/s"
+        return "hbm", row["gbs"], peaks["hbm_gbs"], "GB/s"
+
+    bound, achieved, peak, unit = bound_of(dominant)
+    roofline = dict(bound=bound, achieved=achieved, peak=peak, unit=unit, frac=achieved / peak, traffic=None,
+                    peak_source=(peaks["source"] if bound == "hbm" else
+                                 "148 SMs x 128 fp32 lanes x 2 flop x max SM clock" if bound == "alu" else
+                                 peaks["source"] + " bf16 x (1.1/2.25) / 3 passes"))
+    if dominant["kernel"] == "spmm@256":
+        roofline["traffic"] = NCU_SPMM256["dram_bytes"] * (2 * wl.n_edges + wl.n) / NCU_SPMM256["nnz"]
+        roofline["note"] = ("gather kernel: every stored entry pulls a full operand row through L2 (nnz x ld x 4 B, about "
+                            "23x the algorithmic bytes at mean degree 50), so it runs at the L2-to-SM rate, not at the HBM "
+                            "rate; algorithmic bytes = 4 nnz + 8 N + 8 N ld")
     roofline.update(kernel=dominant["kernel"], ms_per_launch=dominant["ms_per_iter"] / max(dominant["launches_per_iter"], 1e-9),
                     share_of_kernel_time=dominant["share"])
 
@@ -311,7 +319,8 @@ def run_ours(args):
                 roofline=roofline,
                 kernels=[dict(kernel=r["kernel"], ms_per_iter=round(r["ms_per_iter"], 4), share=round(r["share"], 4),
                               launches_per_iter=round(r["launches_per_iter"], 2), gbs=round(r["gbs"], 1),
-                              tflops=round(r["tflops"], 2)) for r in table if r["share"] >= 0.002],
+                              tflops=round(r["tflops"], 2), bound=bound_of(r)[0],
+                              frac=round(bound_of(r)[1] / bound_of(r)[2], 3)) for r in table if r["share"] >= 0.002],
                 objective=dict(L_rho=obj[0], R=obj[1], train_acc=obj[5], exhausted_searches=exhausted,
                                e2e_L_rho=obj2[0]))
     if world == 1 and not args.no_cpu_baseline:

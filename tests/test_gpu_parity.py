@@ -199,3 +199,24 @@ def test_ten_iterations(case, dual_mode):
             assert abs(g.get_state(binding.ST_TAU, l)[0] - o.tau[l]) <= 1e-12 * o.tau[l]
     finally:
         g.destroy()
+
+
+def test_ten_iterations_without_tensor_cores():
+    """The fp32 FMA kernels (tensor_cores = 0) stay a supported path: same ten-pass check on one case."""
+    wl = inputs.make_workload(3, scale=0.012)
+    g, o = make_pair(wl)
+    g.destroy()
+    g = binding.GcnAdmm(wl.n, wl.row_ptr, wl.col_idx, wl.X, wl.y, wl.train_mask, wl.widths, wl.n_comm, wl.community,
+                        wl.w_init, nu=wl.nu, rho=wl.rho, tensor_cores=0)
+    try:
+        g.step(10)
+        dec = g.decisions()
+        o.forced_tol = 1e-4
+        for k in range(10):
+            rec = o.iterate(forced_from(dec, k, o.L, o.M))
+            assert all(r["ok"] for r in list(rec["W"].values()) + list(rec["Z"].values())), k
+        for l in range(1, o.L + 1):
+            assert relerr(g.get_state(binding.ST_W, l), o.W[l]) <= ITER_TOL
+            assert relerr(g.get_state(binding.ST_Z, l), o.Z[l]) <= ITER_TOL
+    finally:
+        g.destroy()
