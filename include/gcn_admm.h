@@ -58,6 +58,9 @@ enum {
  *                  cores as an error-compensated TF32 product (three passes, fp32 accumulation,
  *                  relative error of a few 1e-7 of sum |a||b|); 2: the same product with its earlier, unsplit
  *                  scheduling (kept for comparison); 0: fp32 FMA kernels everywhere
+ *  spmm_ring       0: propagation gathers neighbour rows into registers; 1: rows of 68..256 floats are
+ *                  kept in flight in a shared-memory ring filled with cp.async instead (same result; both
+ *                  forms run at the same ~10 TB/s of gathered bytes on B200, the ring is kept for comparison)
  *  w_init          L host pointers to row-major C_{l-1} x C_l matrices (required)
  *  device          CUDA device ordinal;  stream: a cudaStream_t owned by the caller (NULL = the
  *                  default stream) */
@@ -70,13 +73,14 @@ typedef struct {
   float loss_scale;
   int dual_mode;
   int tensor_cores;
+  int spmm_ring;
   const float* const* w_init;
   int device;
   void* stream;
 } gcn_admm_params;
 
 /* Fills *p with the defaults: nu = rho = 1e-3, tau0 = theta0 = 1, growth 2, shrink 0.5,
- * 40 trials, 30 FISTA iterations, loss_scale 1, dual_mode 0, tensor_cores 1, device 0, stream NULL,
+ * 40 trials, 30 FISTA iterations, loss_scale 1, dual_mode 0, tensor_cores 1, spmm_ring 0, device 0, stream NULL,
  * w_init NULL. */
 void gcn_admm_default_params(gcn_admm_params* p);
 

@@ -170,6 +170,25 @@ struct gcn_admm {
     char name[48];
     std::snprintf(name, sizeof name, "spmm@%d", ldx);
     Scope sc(this, name, 1, 4.0 * gi.nnz + 8.0 * n + 8.0 * (double)n * ldx, 2.0 * (double)gi.nnz * ldx);
+    if (p.spmm_ring && ld4 > 16 && ld4 <= 64) {
+      // rows of 17..64 float4: gathered rows in flight in a shared-memory ring (see k_spmm_ring)
+      CU(cudaMemsetAsync(row_counter, 0, sizeof(int), stream));
+      constexpr int kRingDepth = 16, kRingWarps = 4;
+#define RING_CASE(V)                                                                                          \
+  {                                                                                                           \
+    const size_t smem = (size_t)kRingWarps * kRingDepth * (V) * 32 * sizeof(float4);                          \
+    CU(cudaFuncSetAttribute(gk::k_spmm_ring<V, kRingDepth>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+    int occ = 1;                                                                                              \
+    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gk::k_spmm_ring<V, kRingDepth>, kRingWarps * 32, smem)); \
+    const unsigned grid = (unsigned)std::min<long long>(cdiv(n, (long long)gk::kGrab * kRingWarps), (long long)kSmCount * std::max(occ, 1)); \
+    gk::k_spmm_ring<V, kRingDepth><<<grid, kRingWarps * 32, smem, stream>>>(d_row_ptr, d_col, d_dinv, x4, o4, nn, ld4, row_counter); \
+  }
+      if (ld4 <= 32) RING_CASE(1)
+      else RING_CASE(2)
+#undef RING_CASE
+      CU(cudaGetLastError());
+      return;
+    }
     // 64-thread blocks: rows differ widely in length, small blocks keep the SMs evenly loaded
 #define SPMM_CASE(G, V, UN)                                                                    \
   {                                                                                            \
@@ -816,6 +835,7 @@ void gcn_admm_default_params(gcn_admm_params* p) {
   p->loss_scale = 1.f;
   p->dual_mode = 0;
   p->tensor_cores = 1;
+  p->spmm_ring = 0;
   p->w_init = nullptr;
   p->device = 0;
   p->stream = nullptr;

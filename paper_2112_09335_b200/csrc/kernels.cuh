@@ -127,6 +127,139 @@ k_spmm(const int* __restrict__ row_ptr, const int* __restrict__ col, const float
   }
 }
 
+// Propagation with the gathered rows in flight in shared memory instead of registers.
+// The register-held form above keeps UN x V 16-byte loads per lane in flight, and the register
+// file caps how many warps can do that; measured, it stalls on load latency at ~45 % of the L2
+// rate.  Here a warp owns a ring of D row slots in shared memory: the row of stored entry q is
+// fetched with cp.async into slot q mod D while entry q - D, fetched D steps earlier, is read back
+// (each lane reads the bytes it copied itself) and accumulated, so a warp keeps D whole rows in
+// flight at the cost of a handful of registers.  A warp takes kGrab consecutive rows at a time from
+// a global counter (`row_counter`, zero at launch) and walks their stored entries as one stream, so
+// the ring drains once per grab, not once per row; column indices are prefetched two chunks of 32
+// ahead and their weights dinv[col] one chunk ahead.  V = float4 per lane (ld <= 128 V).
+constexpr int kGrab = 16;
+
+template <int V, int D>
+__global__ void __launch_bounds__(128)
+k_spmm_ring(const int* __restrict__ row_ptr, const int* __restrict__ col, const float* __restrict__ dinv,
+            const float4* __restrict__ x, float4* __restrict__ out, int n, int ld4, int* __restrict__ row_counter) {
+  static_assert(D <= 32, "the lag must stay within two chunks of 32");
+  extern __shared__ __align__(16) float4 ring_all[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  float4* ring = ring_all + (size_t)warp * D * V * 32;
+  const uint32_t ring_s = (uint32_t)__cvta_generic_to_shared(ring);
+  for (;;) {
+    int row_base = 0;
+    if (lane == 0) row_base = atomicAdd(row_counter, kGrab);
+    row_base = __shfl_sync(0xffffffffu, row_base, 0);
+    if (row_base >= n) break;
+    const int rows_here = min(kGrab, n - row_base);
+    // lane t holds the end position and the scale of row row_base + t
+    int rp_lane = 0;
+    float di_lane = 0.f;
+    if (lane < rows_here) { rp_lane = row_ptr[row_base + lane + 1]; di_lane = dinv[row_base + lane]; }
+    const int p0 = row_ptr[row_base];
+    const int p1 = __shfl_sync(0xffffffffu, rp_lane, rows_here - 1);
+    const int total = p1 - p0;
+    int crow = 0;                                       // row (relative) being accumulated
+    int crow_end = __shfl_sync(0xffffffffu, rp_lane, 0);
+    float4 acc[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    int c_cur = 0, c_nxt = 0, c_nxt2 = 0, cur_chunk = -1;
+    float w_cur = 0.f, w_prev = 0.f, w_nxt = 0.f;
+    if (p0 + lane < p1) c_nxt = col[p0 + lane];
+    if (p0 + 32 + lane < p1) c_nxt2 = col[p0 + 32 + lane];
+    if (p0 + lane < p1) w_nxt = dinv[c_nxt];
+
+    auto finish_row = [&]() {
+      const float di = __shfl_sync(0xffffffffu, di_lane, crow);
+#pragma unroll
+      for (int v = 0; v < V; ++v) {
+        const int f = lane + 32 * v;
+        if (f < ld4)
+          out[(long long)(row_base + crow) * ld4 + f] =
+              make_float4(di * acc[v].x, di * acc[v].y, di * acc[v].z, di * acc[v].w);
+        acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    };
+
+    // entries move in batches of kBatch: one commit / one wait per batch, the batch's reads independent
+    constexpr int kBatch = 8;
+    static_assert(D % kBatch == 0 && 32 % kBatch == 0, "batching");
+    constexpr int kLagBatches = D / kBatch;
+    const int n_batches = (total + kBatch - 1) / kBatch;
+    for (int bq = 0; bq < n_batches + kLagBatches; ++bq) {
+      if (bq >= kLagBatches) {              // consume batch bq - kLagBatches (the oldest group in flight)
+        asm volatile("cp.async.wait_group %0;" ::"n"(kLagBatches - 1) : "memory");
+        const int q0 = (bq - kLagBatches) * kBatch;
+        float wj[kBatch];
+#pragma unroll
+        for (int t = 0; t < kBatch; ++t) {
+          const int qc = q0 + t;
+          const float wa = __shfl_sync(0xffffffffu, w_cur, qc & 31), wb = __shfl_sync(0xffffffffu, w_prev, qc & 31);
+          wj[t] = ((qc >> 5) == cur_chunk) ? wa : wb;
+        }
+        float4 xv[kBatch][V];
+#pragma unroll
+        for (int t = 0; t < kBatch; ++t)
+#pragma unroll
+          for (int v = 0; v < V; ++v) {
+            const int f = lane + 32 * v;
+            xv[t][v] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (f < ld4 && q0 + t < total) xv[t][v] = ring[(size_t)((q0 + t) % D) * V * 32 + f];
+          }
+#pragma unroll
+        for (int t = 0; t < kBatch; ++t) {
+          const int qc = q0 + t;
+          if (qc < total) {
+            while (p0 + qc >= crow_end) {   // entry belongs to a later row: close the finished one(s)
+              finish_row();
+              ++crow;
+              crow_end = __shfl_sync(0xffffffffu, rp_lane, crow);
+            }
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+              acc[v].x = fmaf(wj[t], xv[t][v].x, acc[v].x); acc[v].y = fmaf(wj[t], xv[t][v].y, acc[v].y);
+              acc[v].z = fmaf(wj[t], xv[t][v].z, acc[v].z); acc[v].w = fmaf(wj[t], xv[t][v].w, acc[v].w);
+            }
+          }
+        }
+      }
+      if (bq < n_batches) {                 // issue batch bq
+        const int q0 = bq * kBatch;
+        if ((q0 & 31) == 0) {               // the next chunk of 32 entries becomes current
+          w_prev = w_cur;
+          c_cur = c_nxt; w_cur = w_nxt;
+          c_nxt = c_nxt2;
+          cur_chunk = q0 >> 5;
+          const int a1 = p0 + q0 + 32 + lane, a2 = p0 + q0 + 64 + lane;
+          w_nxt = (a1 < p1) ? dinv[c_nxt] : 0.f;
+          c_nxt2 = (a2 < p1) ? col[a2] : 0;
+        }
+#pragma unroll
+        for (int t = 0; t < kBatch; ++t) {
+          const int q = q0 + t;
+          const int cj = __shfl_sync(0xffffffffu, c_cur, q & 31);
+          if (q < total) {
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+              const int f = lane + 32 * v;
+              if (f < ld4)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ring_s + (uint32_t)(((q % D) * V * 32 + f) * 16)),
+                             "l"(x + (long long)cj * ld4 + f)
+                             : "memory");
+            }
+          }
+        }
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    finish_row();                           // the last row of the grab (every row stores its self loop)
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+  }
+}
+
 // ------------------------------------------------------------------------------------------
 // Dense products.
 //   k_gemm_nn : C[M x N] = A[M x K] B[K x N]          (H = P W, D = P grad, G = S W^T, T = G W)
