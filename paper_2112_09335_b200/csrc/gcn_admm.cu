@@ -208,11 +208,11 @@ struct gcn_admm {
 
   // C = A B.  B is handed over twice: row-major K x N (ldb) for the fp32-ALU kernels and K-major
   // N x K (Bk, ldbk; may be NULL) for the tensor-core kernel, which is used whenever it applies
-  // (at most 256 output columns; K capped because its accumulator error grows with K).
+  // (K capped at 2048 because its accumulator error grows with K, about 2.5e-9 K of the magnitude).
   void gemm_nn(const float* A, int lda, const float* B, int ldb, const float* Bk, int ldbk, float* Cm, int ldc,
                long long Mr, int N, int K, const int* skip = nullptr) {
     char name[48];
-    if (p.tensor_cores && Bk != nullptr && N <= 256 && K >= 8 && K <= 512 && Mr >= 512) {
+    if (p.tensor_cores && Bk != nullptr && K >= 8 && K <= 2048 && Mr >= 512 && (p.tensor_cores == 1 || (N <= 256 && K <= 512))) {
       std::snprintf(name, sizeof name, "gemm_tc@%dx%d", K, N);
       Scope sc(this, name, 1, 4.0 * ((double)Mr * (lda + ldc) + (double)K * ldb), 2.0 * (double)Mr * N * K);
       const int tiles = (int)cdiv(Mr, gtc::kBlockM);
@@ -295,11 +295,16 @@ struct gcn_admm {
     int splits = 1;
     long long rps = rows;
     char name[48];
-    if (p.tensor_cores == 1 && Nb <= 256 && rows >= 4096) {
+    if (p.tensor_cores == 1 && rows >= 4096) {
       std::snprintf(name, sizeof name, "gemm_tn_tc@%dx%d", Ka, Nb);
       Scope sc(this, name, 2, 4.0 * ((double)rows * (lda + ldb) + (double)Ka * ldp), 2.0 * (double)rows * Ka * Nb);
+      const int nt_tn = Nb <= 16 ? 16 : Nb <= 32 ? 32 : Nb <= 48 ? 48 : Nb <= 64 ? 64 : Nb <= 128 ? 128 : 256;
+      const int nb_groups = (int)cdiv(Nb, nt_tn);
       const int groups = (int)cdiv(Ka, gtc::kBlockM);
-      splits = (int)std::max<long long>(1, std::min<long long>(kSmCount / groups, cdiv(rows, 256)));
+      // at most 2048 rows (256 MMAs) per accumulator: the tensor core rounds the running sum toward zero at
+      // every MMA, so long sums are cut into splits whose partial results are added in fp64
+      splits = (int)std::max<long long>(std::max(1, kSmCount / (groups * nb_groups)), cdiv(rows, 2048));
+      splits = (int)std::min<long long>(splits, cdiv(rows, 256));
       splits = (int)std::min<long long>(splits, (long long)(part_elems / ((size_t)Ka * ldp)));
       rps = cdiv(rows, splits);
       splits = (int)cdiv(rows, rps);
@@ -307,7 +312,7 @@ struct gcn_admm {
   {                                                                                                            \
     const size_t smem = gtc::TnCfg<NT>::kSmem;                                                                 \
     CU(cudaFuncSetAttribute(gtc::k_gemm_tn_tc<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));   \
-    dim3 grid((unsigned)splits, (unsigned)groups);                                                             \
+    dim3 grid((unsigned)splits, (unsigned)groups, (unsigned)nb_groups);                                        \
     gtc::k_gemm_tn_tc<NT><<<grid, gtc::kTnThreads, smem, stream>>>(A, lda, B, ldb, part, ldp, rows, rps, Ka, Nb, tc_error); \
   }
       if (Nb <= 16) TN_TC(16)
@@ -734,7 +739,9 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
     grad_t_elems = std::max(grad_t_elems, (size_t)h->C[l] * h->ld[l - 1]);
     h->part_elems = std::max(h->part_elems, ge * 4 * kSmCount);
   }
-  h->part_elems = std::min<size_t>(h->part_elems, (size_t)64 << 20);   // at most 256 MB of partial sums
+  for (int l = 1; l <= L; ++l)   // room for one split per 2048 rows (tensor-core form of the transposed product)
+    h->part_elems = std::max(h->part_elems, (size_t)h->C[l - 1] * h->ld[l] * (size_t)cdiv(n, 2048));
+  h->part_elems = std::min<size_t>(h->part_elems, (size_t)256 << 20);   // at most 1 GB of partial sums
   h->part_elems = std::max(h->part_elems, grad_elems);
   h->U = h->alloc<float>(rows * h->ld[L]);
   h->B0 = h->alloc<float>(rows * h->max_ld);

@@ -714,8 +714,8 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
 // unit u of row r sits at unit u ^ (r mod 4); successive column groups are 4096 bytes apart (the
 // descriptor's leading byte offset), successive groups of 4 rows 512 bytes apart (its stride byte
 // offset).  One MMA consumes 8 rows (K = 8), i.e. two atoms.  Same hi/lo split, same separate correction accumulator, same roles as
-// above (8 producer warps, one MMA warp); a CTA owns 128 columns of A (blockIdx.y) and one row
-// split (blockIdx.x) and writes its 128 x NT partial sum once, at the end.
+// above (8 producer warps, one MMA warp); a CTA owns 128 columns of A (blockIdx.y), NT columns of B
+// (blockIdx.z) and one row split (blockIdx.x) and writes its 128 x NT partial sum once, at the end.
 // ------------------------------------------------------------------------------------------------
 constexpr int kTnThreads = 9 * 32;
 constexpr int kTnRows = 32;                       // rows (reduction steps) per chunk
@@ -788,6 +788,7 @@ k_gemm_tn_tc(const float* __restrict__ A, int lda, const float* __restrict__ B, 
   const long long r_end = min(rows, r_begin + rows_per_split);
   const int total = r_end > r_begin ? (int)((r_end - r_begin + kTnRows - 1) / kTnRows) : 0;
   const int ka0 = blockIdx.y * kBlockM;
+  const int nb0 = blockIdx.z * NT;                 // first column of B (and of the partial sum) of this CTA
 
   if (warp < 8) {
     // ---------------- producers ----------------
@@ -810,7 +811,7 @@ k_gemm_tn_tc(const float* __restrict__ A, int lda, const float* __restrict__ B, 
         const int rr = f / (NT / 4), c4 = f % (NT / 4);
         const long long r = r0 + rr;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (f < B_F4 && r < r_end && 4 * c4 < Nb) v = *reinterpret_cast<const float4*>(B + r * ldb + 4 * c4);
+        if (f < B_F4 && r < r_end && nb0 + 4 * c4 < Nb) v = *reinterpret_cast<const float4*>(B + r * ldb + nb0 + 4 * c4);
         pb[i] = v;
       }
     };
@@ -893,7 +894,7 @@ k_gemm_tn_tc(const float* __restrict__ A, int lda, const float* __restrict__ B, 
       if (ka < Ka) {
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          const int col = cchunk * 16 + q * 4;
+          const int col = nb0 + cchunk * 16 + q * 4;
           if (col < ldp)
             *reinterpret_cast<float4*>(dst + col) =
                 make_float4(__uint_as_float(v[q * 4]) + __uint_as_float(w[q * 4]),
