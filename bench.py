@@ -342,7 +342,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=WORKLOAD_INDEX, help="workload index 0..4 (default: the largest)")
+    ap.add_argument("--config", type=int, default=WORKLOAD_INDEX, help="workload index 0..5 (default 4, the largest; 5 = the paper-experiment-shaped one)")
     ap.add_argument("--scale", type=float, default=1.0, help="shrink the workload (profiling captures only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

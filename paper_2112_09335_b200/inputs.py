@@ -5,7 +5,7 @@ labels, masks, initial weights and a community assignment.  Both the CUDA
 library's tests/benchmark and the CPU oracle's tests are fed from here, so the
 two implementations see the same numbers without sharing any arithmetic.
 
-Five workload shapes are provided (``CONFIGS``).  They are synthetic stand-ins
+Six workload shapes are provided (``CONFIGS``; the sixth follows the sizes of the paper's own experiment).  They are synthetic stand-ins
 with the node counts, degree distributions, feature shapes and label structure
 of small citation graphs, a medium citation graph and two large co-purchase /
 product graphs; no item of any public dataset is reproduced.  ``scale`` shrinks
@@ -81,6 +81,12 @@ CONFIGS = [
     dict(name="powerlaw-xlarge", n=2449029, kind="dcsbm", blocks=47, edges=61900000, alpha=1.0,
          draw_factor=1.222, feat="normal", c0=100, classes=47, label="block",
          train_p=0.08, widths=[100, 256, 256, 47], n_comm=64, n_iters=20),
+    # shaped like the paper's own speed-up experiment (Section 4.1, Table 2): 13,752 nodes, 767 features,
+    # 1000 hidden units, 10 classes, 1000 training nodes, 3 communities; the paper gives no edge count, so the
+    # mean degree (30) and the feature density (0.3) are free choices of this build
+    dict(name="table2-shaped", n=13752, kind="dcsbm", blocks=10, edges=206280, alpha=1.5,
+         draw_factor=1.068, feat="bow", feat_p=0.3, c0=767, classes=10, label="block",
+         train=1000, widths=[767, 1000, 10], n_comm=3, n_iters=50),
 ]
 
 
@@ -158,7 +164,7 @@ def glorot(rng, fan_in, fan_out):
 
 
 def make_workload(index: int, scale: float = 1.0, n_comm: int | None = None) -> Workload:
-    """Build config ``index`` (0..4).  ``scale`` < 1 shrinks node and edge counts."""
+    """Build config ``index`` (0..5).  ``scale`` < 1 shrinks node and edge counts."""
     cfg = CONFIGS[index]
     rng = np.random.Generator(np.random.PCG64(BASE_SEED + index))
     n = max(int(round(cfg["n"] * scale)), 4 * cfg["blocks"])

@@ -21,7 +21,8 @@ def small_cases():
             ("cfg1", lambda: inputs.make_workload(1)),
             ("cfg2@0.15", lambda: inputs.make_workload(2, scale=0.15)),
             ("cfg3@0.012", lambda: inputs.make_workload(3, scale=0.012)),
-            ("cfg4@0.001", lambda: inputs.make_workload(4, scale=0.001))]
+            ("cfg4@0.001", lambda: inputs.make_workload(4, scale=0.001)),
+            ("table2@0.12", lambda: inputs.make_workload(5, scale=0.12))]
 
 
 @pytest.fixture(scope="module", params=small_cases(), ids=lambda c: c[0])
@@ -60,7 +61,8 @@ def test_propagation_row_for_row(case, width):
 def test_initial_state_is_the_forward_pass(case):
     wl, g, o = case
     for l in range(1, o.L + 1):
-        assert relerr(g.get_state(binding.ST_Z, l), o.Z[l]) < 2e-6
+        # chained tensor-core products: about 2.5e-9 * K per product (K up to 1000 here)
+        assert relerr(g.get_state(binding.ST_Z, l), o.Z[l]) < 1e-5
         assert np.array_equal(g.get_state(binding.ST_W, l), wl.w_init[l - 1])
     assert not g.get_state(binding.ST_U).any()
     go, oo = g.objective(), o.objective()
@@ -68,7 +70,7 @@ def test_initial_state_is_the_forward_pass(case):
     assert abs(go[2]) <= 1e-12 and abs(go[4]) <= 1e-12      # residuals vanish at the forward pass
     logits, labels = g.predict()
     ol, olab = o.predict()
-    assert relerr(logits, ol) < 2e-6
+    assert relerr(logits, ol) < 1e-5
     gap = np.sort(ol, axis=1)
     clear = (gap[:, -1] - gap[:, -2]) > 1e-5 * np.abs(gap[:, -1]) if ol.shape[1] > 1 else np.ones(wl.n, bool)
     assert np.array_equal(labels[clear], olab[clear])
