@@ -209,6 +209,8 @@ def run_ours(args):
     peaks = measured_peaks()
 
     wl = inputs.make_workload(args.config, scale=args.scale)
+    # a stream of our own (not the default stream): the library can then record a pass as a CUDA graph
+    torch.cuda.set_stream(torch.cuda.Stream())
     stream = torch.cuda.current_stream()
 
     def make(host_arrays=None):
@@ -216,7 +218,7 @@ def run_ours(args):
                                   community=wl.community)
         return binding.GcnAdmm(wl.n, src["row_ptr"], src["col_idx"], src["X"], src["y"], src["train_mask"], wl.widths,
                                wl.n_comm, src["community"], wl.w_init, nu=wl.nu, rho=wl.rho, device=local,
-                               stream=stream.cuda_stream)
+                               stream=stream.cuda_stream, dual_mode=args.dual_mode, use_graph=0 if args.no_graph else 1)
 
     def barrier():
         if dist is not None:
@@ -311,7 +313,8 @@ def run_ours(args):
 
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32",
-                data="synthetic", config=config_dict(wl, dict(parallelism="replicas only" if world > 1 else "single GPU")),
+                data="synthetic", config=config_dict(wl, dict(parallelism="replicas only" if world > 1 else "single GPU", dual_mode=args.dual_mode,
+                                          cuda_graph=not args.no_graph)),
                 clocks=clocks, gpu_launches=int(launches),
                 e2e=dict(value=world * args.steps / e2e_s, unit=UNIT, h2d_bytes_per_step=h2d / args.steps,
                          d2h_bytes_per_step=d2h / args.steps, seconds=e2e_s,
@@ -345,6 +348,8 @@ def main():
     ap.add_argument("--config", type=int, default=WORKLOAD_INDEX, help="workload index 0..5 (default 4, the largest; 5 = the paper-experiment-shaped one)")
     ap.add_argument("--scale", type=float, default=1.0, help="shrink the workload (profiling captures only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--dual-mode", type=int, default=0, help="0: Eq. 3 as printed (default), 1: textbook dual update")
+    ap.add_argument("--no-graph", action="store_true", help="plain launches instead of CUDA-graph replay")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

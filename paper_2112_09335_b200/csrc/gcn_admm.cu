@@ -143,10 +143,12 @@ struct gcn_admm {
   size_t part_elems = 0;
   SearchCtl *ctl_w = nullptr, *ctl_z = nullptr;   // [L+1], [(L+1) * M]
   double *sums_w = nullptr, *sums_z = nullptr, *acc_w = nullptr, *acc_z = nullptr, *obj = nullptr;
-  int *n_active = nullptr, *status = nullptr, *row_counter = nullptr;
+  int *n_active = nullptr, *status = nullptr, *row_counter = nullptr, *d_pass = nullptr;
+  cudaGraphExec_t pass_graph = nullptr;   // one pass of Algorithm 1, recorded once and replayed
   int *log_trial_w = nullptr, *log_trial_z = nullptr;
   double *log_q_w = nullptr, *log_q_z = nullptr;
   long long log_count = 0;
+  long long launches_per_pass = 0;
   bool fresh = false;        // P_l, H_l agree with the stored W, Z
   std::string err;
   std::vector<int> ix_cache[16];
@@ -364,17 +366,20 @@ struct gcn_admm {
 
   int n_passes() const { return (p.bt_max_trials + gk::kCand - 1) / gk::kCand; }
 
-  int* log_slot_trial_w() { return log_trial_w + (log_count % kLogPasses) * L; }
-  double* log_slot_q_w() { return log_q_w + (log_count % kLogPasses) * L; }
-  int* log_slot_trial_z() { return log_trial_z + (log_count % kLogPasses) * (long long)std::max(L - 1, 0) * M; }
-  double* log_slot_q_z() { return log_q_z + (log_count % kLogPasses) * (long long)std::max(L - 1, 0) * M; }
+  long long z_per_pass() const { return (long long)std::max(L - 1, 0) * M; }
 
   void begin_log_pass() {
-    const long long zc = (long long)std::max(L - 1, 0) * M;
+    const long long zc = z_per_pass();
     Scope sc(this, "small", zc > 0 ? 2 : 1, 0.0, 0.0);
-    gk::k_fill_int<<<1, 64, 0, stream>>>(log_slot_trial_w(), L, -3);
-    if (zc > 0) gk::k_fill_int<<<grid_for(zc), 256, 0, stream>>>(log_slot_trial_z(), zc, -3);
+    gk::k_log_clear<<<1, 64, 0, stream>>>(log_trial_w, d_pass, L, kLogPasses);
+    if (zc > 0) gk::k_log_clear<<<grid_for(zc), 256, 0, stream>>>(log_trial_z, d_pass, zc, kLogPasses);
     CU(cudaGetLastError());
+  }
+  void end_log_pass() {
+    Scope sc(this, "small", 1, 0.0, 0.0);
+    gk::k_pass_advance<<<1, 1, 0, stream>>>(d_pass);
+    CU(cudaGetLastError());
+    ++log_count;
   }
 
   // ---- W_l block (Section 3.1) --------------------------------------------------------
@@ -423,7 +428,7 @@ struct gcn_admm {
     CU(cudaGetLastError());
     {
       Scope sc(this, "small", 2, 0.0, 0.0);
-      gk::k_log_decisions<<<1, 32, 0, stream>>>(ctl, 1, log_slot_trial_w() + (l - 1), log_slot_q_w() + (l - 1));
+      gk::k_log_decisions<<<1, 32, 0, stream>>>(ctl, 1, log_trial_w, log_q_w, d_pass, L, l - 1, kLogPasses);
       gk::k_apply_w<<<(unsigned)cdiv((long long)Kp * Cn, 256), 256, 0, stream>>>(W[l], Wt[l], grad, Kp, Cn, ldc,
                                                                                ld[l - 1], ctl);
     }
@@ -520,8 +525,8 @@ struct gcn_admm {
     CU(cudaGetLastError());
     {
       Scope sc(this, "small", 1, 0.0, 0.0);
-      gk::k_log_decisions<<<(unsigned)cdiv(M, 128), 128, 0, stream>>>(ctl, M, log_slot_trial_z() + (size_t)(l - 1) * M,
-                                                                    log_slot_q_z() + (size_t)(l - 1) * M);
+      gk::k_log_decisions<<<(unsigned)cdiv(M, 128), 128, 0, stream>>>(ctl, M, log_trial_z, log_q_z, d_pass, z_per_pass(),
+                                                                      (long long)(l - 1) * M, kLogPasses);
     }
     Scope sc(this, "apply_z", 1, 12.0 * (double)n * ldl, 0.0);
     gk::k_apply_z<<<grid_for(n * (ldl / 4)), 256, 0, stream>>>((float4*)Z[l], (const float4*)B2, ldl / 4, n, d_row_comm, ctl);
@@ -561,7 +566,7 @@ struct gcn_admm {
     update_output(p.dual_mode == 0, true);
     refresh();
     if (p.dual_mode != 0) dual_from_stored();
-    ++log_count;
+    end_log_pass();
   }
 
   // logits of Problem 1's forward pass with the stored W, left in B0 (N x ld_L)
@@ -763,6 +768,8 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
   h->n_active = h->alloc<int>(1);
   h->status = h->alloc<int>(1);
   h->row_counter = h->alloc<int>(1);
+  h->d_pass = h->alloc<int>(1);
+  CU(cudaMemset(h->d_pass, 0, sizeof(int)));
   h->log_trial_w = h->alloc<int>((size_t)kLogPasses * L);
   h->log_q_w = h->alloc<double>((size_t)kLogPasses * L);
   h->log_trial_z = h->alloc<int>((size_t)kLogPasses * std::max(L - 1, 0) * n_comm);
@@ -843,6 +850,7 @@ void gcn_admm_default_params(gcn_admm_params* p) {
   p->dual_mode = 0;
   p->tensor_cores = 1;
   p->spmm_ring = 0;
+  p->use_graph = 1;
   p->w_init = nullptr;
   p->device = 0;
   p->stream = nullptr;
@@ -894,6 +902,7 @@ void gcn_admm_destroy(gcn_admm* h) {
   if (cudaSetDevice(h->p.device) == cudaSuccess) {
     cudaStreamSynchronize(h->stream);
     h->collect_profile();
+    if (h->pass_graph) cudaGraphExecDestroy(h->pass_graph);
     for (cudaEvent_t e : h->event_pool) cudaEventDestroy(e);
     for (void* q : h->owned) cudaFree(q);
   }
@@ -907,7 +916,39 @@ int gcn_admm_step(gcn_admm* h, int n_iters) {
   return guarded(h, [&] {
     if (n_iters < 0) throw Fail{GCN_ADMM_ERR_ARG, "n_iters must be >= 0"};
     h->log_count = 0;
-    for (int k = 0; k < n_iters; ++k) h->iterate();
+    CU(cudaMemsetAsync(h->d_pass, 0, sizeof(int), h->stream));
+    // A pass is a fixed sequence of launches (every decision is taken on the device), so on a stream
+    // that can be captured it is recorded once and replayed: the small workloads are launch-bound.
+    const bool replay = h->p.use_graph && h->stream != nullptr && !h->profiling && n_iters >= 2;
+    if (!replay) {
+      for (int k = 0; k < n_iters; ++k) h->iterate();
+      return;
+    }
+    if (!h->fresh) h->refresh();
+    if (h->pass_graph == nullptr) {
+      cudaGraph_t graph = nullptr;
+      CU(cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
+      const long long launches_before = h->launches, log_before = h->log_count;
+      try {
+        h->iterate();
+      } catch (...) {
+        cudaStreamEndCapture(h->stream, &graph);
+        if (graph) cudaGraphDestroy(graph);
+        throw;
+      }
+      CU(cudaStreamEndCapture(h->stream, &graph));
+      h->launches_per_pass = h->launches - launches_before;
+      h->launches = launches_before;       // recording launched nothing
+      h->log_count = log_before;
+      cudaError_t e = cudaGraphInstantiate(&h->pass_graph, graph, 0);
+      cudaGraphDestroy(graph);
+      if (e != cudaSuccess) throw Fail{GCN_ADMM_ERR_CUDA, std::string("cudaGraphInstantiate: ") + cudaGetErrorString(e)};
+    }
+    for (int k = 0; k < n_iters; ++k) {
+      CU(cudaGraphLaunch(h->pass_graph, h->stream));
+      h->launches += h->launches_per_pass;
+      ++h->log_count;
+    }
   });
 }
 
@@ -918,6 +959,7 @@ int gcn_admm_step_block(gcn_admm* h, int phase, int layer) {
       if (layer < 1 || layer > L) throw Fail{GCN_ADMM_ERR_ARG, "layer out of range"};
     if (!h->fresh) h->refresh();
     h->log_count = 0;
+    CU(cudaMemsetAsync(h->d_pass, 0, sizeof(int), h->stream));
     h->begin_log_pass();
     if (phase == GCN_ADMM_PHASE_W) {
       h->update_W(layer);
@@ -930,7 +972,7 @@ int gcn_admm_step_block(gcn_admm* h, int phase, int layer) {
     } else {
       throw Fail{GCN_ADMM_ERR_ARG, "unknown phase"};
     }
-    ++h->log_count;
+    h->end_log_pass();
   });
 }
 

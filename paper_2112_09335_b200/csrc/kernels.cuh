@@ -753,14 +753,28 @@ __global__ void k_search_decide(SearchCtl* ctl, int count, double* __restrict__ 
   for (int j = 0; j < acc_per; ++j) acc[i * acc_per + j] = 0.0;
 }
 
-// Copies the decision of each search into the log of this pass.
-__global__ void k_log_decisions(const SearchCtl* __restrict__ ctl, int count, int* __restrict__ trial,
-                                double* __restrict__ q) {
+// The decision log is a ring of `ring` passes; the slot in use is *pass mod ring, with the pass counter
+// kept on the device so that a recorded launch sequence stays valid from one pass to the next.
+// Copies the decision of each search into the slot of the current pass.
+__global__ void k_log_decisions(const SearchCtl* __restrict__ ctl, int count, int* __restrict__ trial_base,
+                                double* __restrict__ q_base, const int* __restrict__ pass, long long per_pass,
+                                long long offset, int ring) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= count) return;
-  trial[i] = ctl[i].trial;
-  q[i] = ctl[i].q;
+  const long long at = (long long)(*pass % ring) * per_pass + offset + i;
+  trial_base[at] = ctl[i].trial;
+  q_base[at] = ctl[i].q;
 }
+
+// Marks every entry of the current pass's slot as "not run".
+__global__ void k_log_clear(int* __restrict__ trial_base, const int* __restrict__ pass, long long per_pass, int ring) {
+  const long long at0 = (long long)(*pass % ring) * per_pass;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < per_pass;
+       i += (long long)gridDim.x * blockDim.x)
+    trial_base[at0 + i] = -3;
+}
+
+__global__ void k_pass_advance(int* __restrict__ pass) { *pass += 1; }
 
 // W <- W - grad / tau (and its transpose copy), C_prev x C matrices with padded leading dimensions.
 __global__ void k_apply_w(float* __restrict__ W, float* __restrict__ Wt, const float* __restrict__ grad,
