@@ -218,7 +218,7 @@ def run_ours(args):
                                   community=wl.community)
         return binding.GcnAdmm(wl.n, src["row_ptr"], src["col_idx"], src["X"], src["y"], src["train_mask"], wl.widths,
                                wl.n_comm, src["community"], wl.w_init, nu=wl.nu, rho=wl.rho, device=local,
-                               stream=stream.cuda_stream, dual_mode=args.dual_mode, use_graph=0 if args.no_graph else 1)
+                               stream=stream.cuda_stream, dual_mode=args.dual_mode, use_graph=0 if args.no_graph else 2)
 
     def barrier():
         if dist is not None:
@@ -314,7 +314,7 @@ def run_ours(args):
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32",
                 data="synthetic", config=config_dict(wl, dict(parallelism="replicas only" if world > 1 else "single GPU", dual_mode=args.dual_mode,
-                                          cuda_graph=not args.no_graph)),
+                                          cuda_graph="off" if args.no_graph else "auto (small problems only)")),
                 clocks=clocks, gpu_launches=int(launches),
                 e2e=dict(value=world * args.steps / e2e_s, unit=UNIT, h2d_bytes_per_step=h2d / args.steps,
                          d2h_bytes_per_step=d2h / args.steps, seconds=e2e_s,

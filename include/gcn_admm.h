@@ -62,7 +62,9 @@ enum {
  *                  kept in flight in a shared-memory ring filled with cp.async instead (same result; both
  *                  forms run at the same ~10 TB/s of gathered bytes on B200, the ring is kept for comparison)
  *  use_graph       1: gcn_admm_step records one pass as a CUDA graph on first use and replays it (only when
- *                  the handle's stream is not the default stream and profiling is off); 0: plain launches
+ *                  the handle's stream is not the default stream and profiling is off); 2: the same, but
+ *                  only for problems small enough to be launch-bound (N x widest layer < 2^25);
+ *                  0: plain launches
  *  w_init          L host pointers to row-major C_{l-1} x C_l matrices (required)
  *  device          CUDA device ordinal;  stream: a cudaStream_t owned by the caller (NULL = the
  *                  default stream) */
@@ -83,7 +85,7 @@ typedef struct {
 } gcn_admm_params;
 
 /* Fills *p with the defaults: nu = rho = 1e-3, tau0 = theta0 = 1, growth 2, shrink 0.5,
- * 40 trials, 30 FISTA iterations, loss_scale 1, dual_mode 0, tensor_cores 1, spmm_ring 0, use_graph 1, device 0, stream NULL,
+ * 40 trials, 30 FISTA iterations, loss_scale 1, dual_mode 0, tensor_cores 1, spmm_ring 0, use_graph 2, device 0, stream NULL,
  * w_init NULL. */
 void gcn_admm_default_params(gcn_admm_params* p);
 

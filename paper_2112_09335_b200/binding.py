@@ -101,7 +101,7 @@ class GcnAdmm:
 
     def __init__(self, n, row_ptr, col_idx, X, y, train_mask, widths, n_comm, community, w_init, nu=1e-3, rho=1e-3,
                  tau0=1.0, theta0=1.0, bt_growth=2.0, bt_shrink=0.5, bt_max_trials=40, fista_iters=30,
-                 loss_scale=1.0, dual_mode=0, tensor_cores=1, spmm_ring=0, use_graph=1, device=0, stream=0):
+                 loss_scale=1.0, dual_mode=0, tensor_cores=1, spmm_ring=0, use_graph=2, device=0, stream=0):
         lib = load()
         self._lib = lib
         self._h = C.c_void_p()

@@ -850,7 +850,7 @@ void gcn_admm_default_params(gcn_admm_params* p) {
   p->dual_mode = 0;
   p->tensor_cores = 1;
   p->spmm_ring = 0;
-  p->use_graph = 1;
+  p->use_graph = 2;
   p->w_init = nullptr;
   p->device = 0;
   p->stream = nullptr;
@@ -919,7 +919,9 @@ int gcn_admm_step(gcn_admm* h, int n_iters) {
     CU(cudaMemsetAsync(h->d_pass, 0, sizeof(int), h->stream));
     // A pass is a fixed sequence of launches (every decision is taken on the device), so on a stream
     // that can be captured it is recorded once and replayed: the small workloads are launch-bound.
-    const bool replay = h->p.use_graph && h->stream != nullptr && !h->profiling && n_iters >= 2;
+    // use_graph 1: always; 2: only where a pass is short enough for launch overhead to matter
+    const bool wanted = h->p.use_graph == 1 || (h->p.use_graph == 2 && h->n * (long long)h->max_ld < (1LL << 25));
+    const bool replay = wanted && h->stream != nullptr && !h->profiling && n_iters >= 2;
     if (!replay) {
       for (int k = 0; k < n_iters; ++k) h->iterate();
       return;
