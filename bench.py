@@ -218,7 +218,7 @@ def run_ours(args):
                                   community=wl.community)
         return binding.GcnAdmm(wl.n, src["row_ptr"], src["col_idx"], src["X"], src["y"], src["train_mask"], wl.widths,
                                wl.n_comm, src["community"], wl.w_init, nu=wl.nu, rho=wl.rho, device=local,
-                               stream=stream.cuda_stream, dual_mode=args.dual_mode, use_graph=0 if args.no_graph else 2)
+                               stream=stream.cuda_stream, dual_mode=args.dual_mode, use_graph=0 if args.no_graph else 2, schedule=args.schedule)
 
     def barrier():
         if dist is not None:
@@ -313,7 +313,7 @@ def run_ours(args):
 
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32",
-                data="synthetic", config=config_dict(wl, dict(parallelism="replicas only" if world > 1 else "single GPU", dual_mode=args.dual_mode,
+                data="synthetic", config=config_dict(wl, dict(parallelism="replicas only" if world > 1 else "single GPU", dual_mode=args.dual_mode, schedule=args.schedule,
                                           cuda_graph="off" if args.no_graph else "auto (small problems only)")),
                 clocks=clocks, gpu_launches=int(launches),
                 e2e=dict(value=world * args.steps / e2e_s, unit=UNIT, h2d_bytes_per_step=h2d / args.steps,
@@ -349,6 +349,7 @@ def main():
     ap.add_argument("--scale", type=float, default=1.0, help="shrink the workload (profiling captures only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--dual-mode", type=int, default=0, help="0: Eq. 3 as printed (default), 1: textbook dual update")
+    ap.add_argument("--schedule", type=int, default=0, help="0: Algorithm 1 (default), 1: the serial schedule")
     ap.add_argument("--no-graph", action="store_true", help="plain launches instead of CUDA-graph replay")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -65,6 +65,9 @@ enum {
  *                  the handle's stream is not the default stream and profiling is off); 2: the same, but
  *                  only for problems small enough to be launch-bound (N x widest layer < 2^25);
  *                  0: plain launches
+ *  schedule        0: Algorithm 1 (every W_l, then every Z_{l,m}, then U; Jacobi inside a pass);
+ *                  1: the serial schedule of Section 4.1 (W_1, Z_1, .., W_L, Z_L, U one after the other,
+ *                  each block reading the latest value of all others; the dual uses the new iterates)
  *  w_init          L host pointers to row-major C_{l-1} x C_l matrices (required)
  *  device          CUDA device ordinal;  stream: a cudaStream_t owned by the caller (NULL = the
  *                  default stream) */
@@ -79,13 +82,14 @@ typedef struct {
   int tensor_cores;
   int spmm_ring;
   int use_graph;
+  int schedule;
   const float* const* w_init;
   int device;
   void* stream;
 } gcn_admm_params;
 
 /* Fills *p with the defaults: nu = rho = 1e-3, tau0 = theta0 = 1, growth 2, shrink 0.5,
- * 40 trials, 30 FISTA iterations, loss_scale 1, dual_mode 0, tensor_cores 1, spmm_ring 0, use_graph 2, device 0, stream NULL,
+ * 40 trials, 30 FISTA iterations, loss_scale 1, dual_mode 0, tensor_cores 1, spmm_ring 0, use_graph 2, schedule 0, device 0, stream NULL,
  * w_init NULL. */
 void gcn_admm_default_params(gcn_admm_params* p);
 

@@ -24,6 +24,7 @@ Where each function comes from (sections / equations of the paper):
 * ``OracleADMM.update_ZL``        Eq. (7), solved row by row with FISTA (Beck & Teboulle 2009).
 * ``OracleADMM.update_U``         Eq. (3).
 * ``OracleADMM.iterate``          Algorithm 1 (W blocks, then Z blocks, then U, all Jacobi).
+* ``OracleADMM.iterate_sequential``  the serial schedule of Section 4.1 (one block after the other).
 * ``OracleADMM.objective``        Eq. (1) in its full-graph form.
 * ``OracleADMM.predict``          forward pass of Problem 1 with the current W.
 
@@ -45,6 +46,8 @@ is UNPINNED by the paper, they are stated choices):
   dual_mode 1 is the textbook update with the k+1 iterates.
 * initial state: given W, Z from the forward pass of Problem 1, U = 0, tau = tau0, theta = theta0.
 * index lists are ascending and unique; nodes are ordered by (community, original id).
+* serial schedule: block order W_1, Z_1, .., W_L, Z_L, U with the latest values everywhere (the paper only
+  says that the layers are trained sequentially).
 """
 
 from __future__ import annotations
@@ -432,6 +435,32 @@ class OracleADMM:
         else:
             Un = self.update_U(Wn, Zn)
         self.W, self.tau, self.Z, self.theta, self.U = Wn, taun, Zn, thetan, Un
+        return rec
+
+    def iterate_sequential(self, forced=None, trace=None):
+        """The serial schedule of Section 4.1 ("layers trained sequentially"): the same block updates as
+        Algorithm 1, but taken one after the other in the order W_1, Z_1, W_2, Z_2, .., W_L, Z_L, U, each
+        reading the latest value of every other block (the communities of one layer still move together,
+        from the same Z_l).  ``trace``, when a list, receives L_rho after every block."""
+        L, M = self.L, self.M
+        rec = dict(W={}, Z={})
+        fW = (forced or {}).get("W", {})
+        fZ = (forced or {}).get("Z", {})
+        for l in range(1, L + 1):
+            self.W[l], self.tau[l], rec["W"][l] = self.update_W(l, forced=fW.get(l))
+            if trace is not None:
+                trace.append(("W", l, self.objective()[0]))
+            if l < L:
+                Zl = self.Z[l].copy()
+                for m in range(M):
+                    Zlm, self.theta[l][m], rec["Z"][(l, m)] = self.update_Z(l, m, self.W, forced=fZ.get((l, m)))
+                    Zl[self.V[m]] = Zlm
+                self.Z[l] = Zl
+            else:
+                self.Z[L] = self.update_ZL(self.W)
+            if trace is not None:
+                trace.append(("Z", l, self.objective()[0]))
+        self.U = self.update_U(self.W, self.Z)
         return rec
 
     # ---- reporting --------------------------------------------------------------------

@@ -558,7 +558,27 @@ struct gcn_admm {
     fresh = true;
   }
 
+  // The serial schedule of Section 4.1: the same block updates, one after the other in the order
+  // W_1, Z_1, .., W_L, Z_L, U, each reading the latest value of every other block.
+  void iterate_sequential() {
+    if (!fresh) refresh();
+    begin_log_pass();
+    for (int l = 1; l <= L; ++l) {
+      if (l >= 2) {   // Z_{l-1} has just moved: P_l and H_l follow it (H_{l+1} still matches the untouched Z_l)
+        spmm(Z[l - 1], P[l], ld[l - 1]);
+        gemm_nn(P[l], ld[l - 1], W[l], ld[l], Wt[l], ld[l - 1], H[l], ld[l], n, C[l], C[l - 1]);
+      }
+      update_W(l);
+      if (l < L) update_Z_hidden(l);
+      else update_output(false, true);
+    }
+    refresh();
+    dual_from_stored();
+    end_log_pass();
+  }
+
   void iterate() {   // Algorithm 1, one pass
+    if (p.schedule == 1) { iterate_sequential(); return; }
     if (!fresh) refresh();
     begin_log_pass();
     for (int l = 1; l <= L; ++l) update_W(l);
@@ -851,6 +871,7 @@ void gcn_admm_default_params(gcn_admm_params* p) {
   p->tensor_cores = 1;
   p->spmm_ring = 0;
   p->use_graph = 2;
+  p->schedule = 0;
   p->w_init = nullptr;
   p->device = 0;
   p->stream = nullptr;
@@ -871,7 +892,7 @@ int gcn_admm_create(gcn_admm** out, long long n, const long long* row_ptr, const
   for (int l = 0; l < n_layers; ++l)
     if (!p->w_init[l]) { g_create_error = "w_init holds a NULL pointer"; return GCN_ADMM_ERR_ARG; }
   if (!(p->nu > 0.f) || !(p->rho > 0.f) || !(p->bt_growth > 1.f) || !(p->bt_shrink > 0.f) || p->bt_max_trials < 1 ||
-      p->bt_max_trials > 64 || p->fista_iters < 0 || !(p->tau0 > 0.f) || !(p->theta0 > 0.f) || !(p->loss_scale > 0.f)) {
+      p->bt_max_trials > 64 || p->fista_iters < 0 || p->schedule < 0 || p->schedule > 1 || !(p->tau0 > 0.f) || !(p->theta0 > 0.f) || !(p->loss_scale > 0.f)) {
     g_create_error = "a parameter is out of range";
     return GCN_ADMM_ERR_ARG;
   }

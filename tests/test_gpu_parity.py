@@ -222,3 +222,30 @@ def test_ten_iterations_without_tensor_cores():
             assert relerr(g.get_state(binding.ST_Z, l), o.Z[l]) <= ITER_TOL
     finally:
         g.destroy()
+
+
+@pytest.mark.parametrize("name,make_wl", small_cases()[:2] + small_cases()[3:4], ids=lambda c: c if isinstance(c, str) else "")
+def test_ten_iterations_serial_schedule(name, make_wl):
+    """schedule = 1 (Section 4.1's serial ADMM: blocks one after the other) against the oracle's serial pass."""
+    wl = make_wl()
+    o = make_oracle(wl)
+    g = binding.GcnAdmm(wl.n, wl.row_ptr, wl.col_idx, wl.X, wl.y, wl.train_mask, wl.widths, wl.n_comm, wl.community,
+                        wl.w_init, nu=wl.nu, rho=wl.rho, schedule=1)
+    try:
+        g.step(10)
+        dec = g.decisions()
+        o.forced_tol = 1e-4
+        for k in range(10):
+            rec = o.iterate_sequential(forced_from(dec, k, o.L, o.M))
+            bad = [(key, r) for key, r in list(rec["W"].items()) + list(rec["Z"].items()) if not r["ok"]]
+            assert not bad, (k, bad[:2])
+        worst = 0.0
+        for l in range(1, o.L + 1):
+            worst = max(worst, relerr(g.get_state(binding.ST_W, l), o.W[l]), relerr(g.get_state(binding.ST_Z, l), o.Z[l]))
+        eu = relerr(g.get_state(binding.ST_U), o.U)
+        go, oo = g.objective(), o.objective()
+        print(f"\n  serial {name}: worst W/Z rel {worst:.2e}  U rel {eu:.2e}  L_rho {go[0]:.6g} vs {oo[0]:.6g}")
+        assert worst <= ITER_TOL and eu <= ITER_TOL
+        assert abs(go[0] - oo[0]) <= ITER_TOL * np.abs(oo[1:5]).sum()
+    finally:
+        g.destroy()

@@ -400,3 +400,41 @@ def test_sampled_row_evaluator_matches_the_full_oracle():
         np.testing.assert_allclose(sr.grad_Z_rows(l, rows, o.Z, o.W, o.U), full, atol=1e-12)
     np.testing.assert_allclose(sr.ZL_rows(rows, o.Z, o.W, o.U), o.update_ZL(o.W), atol=1e-12)
     np.testing.assert_allclose(sr.U_rows(rows, o.Z, o.W, o.U), o.update_U(o.W, o.Z), atol=1e-13)
+
+
+@pytest.mark.parametrize("seed,n_comm", [(41, 1), (42, 3)])
+def test_sequential_schedule_descends_block_by_block(seed, n_comm):
+    """In the serial schedule every accepted W / hidden-Z step is a majorisation step on the augmented
+    Lagrangian as a function of that block with all other blocks at their latest values, so L_rho of Eq. 1
+    cannot go up across such a block (with one community; with several, the communities of a layer move
+    together from the same point and the bound holds per community objective, so a small slack is allowed).
+    A schedule that read stale values would not have this property."""
+    pr, o = make(seed, n_comm=n_comm)
+    prev = o.objective()[0]
+    for it in range(3):
+        trace = []
+        o.iterate_sequential(trace=trace)
+        for kind, l, val in trace:
+            hidden_or_w = kind == "W" or l < o.L
+            slack = (1e-12 if n_comm == 1 else 5e-3) * max(1.0, abs(prev))
+            if hidden_or_w:
+                assert val <= prev + slack, (it, kind, l, prev, val)
+            prev = val
+        prev = o.objective()[0]       # after the dual step
+
+
+def test_sequential_schedule_uses_latest_values():
+    """One pass by hand: W_1 from the old state, Z_1 with the new W_1 and the old W_2, W_2 with the new Z_1."""
+    pr, o = make(43)
+    pr, ref = make(43)
+    o.iterate_sequential()
+    W1, t, _ = ref.update_W(1)
+    ref.W[1], ref.tau[1] = W1, t
+    Z1 = ref.Z[1].copy()
+    for m in range(ref.M):
+        Z1[ref.V[m]], ref.theta[1][m], _ = ref.update_Z(1, m, ref.W)
+    ref.Z[1] = Z1
+    W2, t, _ = ref.update_W(2)
+    np.testing.assert_array_equal(o.W[1], W1)
+    np.testing.assert_array_equal(o.Z[1], Z1)
+    np.testing.assert_array_equal(o.W[2], W2)
