@@ -158,7 +158,8 @@ class GcnAdmm:
         return np.array(out[:])
 
     def weights(self, layer):
-        out = np.empty((self.widths[layer - 1], self.widths[layer]), dtype=np.float32)
+        shape = (self.widths[layer - 1], self.widths[layer]) if 1 <= layer <= self.L else (1, 1)   # the library rejects it
+        out = np.empty(shape, dtype=np.float32)
         self._check(self._lib.gcn_admm_weights(self._h, layer, _ptr(out)))
         return out
 
@@ -202,6 +203,8 @@ class GcnAdmm:
         return np.ctypeslib.as_array(data, shape=(length.value,)).copy()
 
     def _state_shape(self, which, layer):
+        if which in (ST_W, ST_Z) and not 1 <= layer <= self.L:
+            return (1,), np.float32            # out of range: left to the library to reject
         if which == ST_W:
             return (self.widths[layer - 1], self.widths[layer]), np.float32
         if which == ST_Z:

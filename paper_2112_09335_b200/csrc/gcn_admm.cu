@@ -393,7 +393,7 @@ struct gcn_admm {
       Scope sc(this, "small", 3, 0.0, 0.0);
       gk::k_transpose_small<<<(unsigned)cdiv((long long)Kp * Cn, 256), 256, 0, stream>>>(grad, ldc, grad_t, ld[l - 1], Kp, Cn);
       gk::k_two_sumsq<<<1, 1024, 0, stream>>>(grad, W[l], (long long)Kp * ldc, sums_w);
-      gk::k_search_begin<<<1, 32, 0, stream>>>(ctl, 1, sums_w, 2, p.bt_shrink, p.bt_growth, acc_w, gk::kCand, nullptr);
+      gk::k_search_begin<<<1, 32, 0, stream>>>(ctl, 1, sums_w, 2, p.bt_shrink, p.bt_growth, acc_w, gk::kCand, nullptr, status);
       CU(cudaGetLastError());
     }
     gemm_nn(P[l], ld[l - 1], grad, ldc, grad_t, ld[l - 1], B1, ldc, n, Cn, Kp, &ctl->done);   // D = P_l grad
@@ -457,7 +457,7 @@ struct gcn_admm {
     {
       Scope sc(this, "small", 1, 0.0, 0.0);
       gk::k_search_begin<<<(unsigned)cdiv(M, 128), 128, 0, stream>>>(ctl, M, sums_z, 3, p.bt_shrink, p.bt_growth, acc_z,
-                                                                     per, n_active);
+                                                                     per, n_active, status);
       CU(cudaGetLastError());
     }
     gemm_nn(B2, ldl, W[l + 1], ldn, Wt[l + 1], ldl, B1, ldn, n, C[l + 1], C[l]);         // T = G W_{l+1}

@@ -660,7 +660,7 @@ __device__ __forceinline__ void set_candidates(SearchCtl* c, double growth) {
 // Starts `count` searches: sums[i*stride + 0] = ||grad||^2, sums[i*stride + 1] = ||x||^2.
 __global__ void k_search_begin(SearchCtl* ctl, int count, const double* __restrict__ sums, int stride,
                                double shrink, double growth, double* __restrict__ acc, int acc_per,
-                               int* __restrict__ n_active) {
+                               int* __restrict__ n_active, int* __restrict__ status) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= count) return;
   SearchCtl* c = ctl + i;
@@ -672,7 +672,9 @@ __global__ void k_search_begin(SearchCtl* ctl, int count, const double* __restri
   for (int j = 0; j < acc_per; ++j) acc[i * acc_per + j] = 0.0;
   if (!(c->gg > 1e-24 * c->xx)) {          // zero up to rounding (also catches NaN): skip
     c->done = 1;
-    c->trial = (c->gg == c->gg) ? -1 : -2;
+    const bool finite = (c->gg == c->gg) && (c->xx == c->xx) && c->gg < 1.0e300 && c->xx < 1.0e300;
+    c->trial = finite ? -1 : -2;
+    if (!finite) atomicOr(status, 1);     // a NaN or an infinity reached the gradient or the block itself
     return;
   }
   c->done = 0;
