@@ -670,14 +670,24 @@ int guarded(gcn_admm* h, F&& body) {
   }
 }
 
+// View of `count` elements on the host: the caller's buffer itself when it is host memory, a copy when
+// it lives on the device.
 template <typename T>
-std::vector<T> to_host(const T* p, size_t count) {
-  std::vector<T> v(count);
-  if (count == 0) return v;
-  if (is_device_pointer(p)) CU(cudaMemcpy(v.data(), p, count * sizeof(T), cudaMemcpyDeviceToHost));
-  else std::memcpy(v.data(), p, count * sizeof(T));
-  return v;
-}
+struct HostView {
+  std::vector<T> copy;
+  const T* ptr = nullptr;
+  HostView(const T* p, size_t count) {
+    if (count > 0 && is_device_pointer(p)) {
+      copy.resize(count);
+      CU(cudaMemcpy(copy.data(), p, count * sizeof(T), cudaMemcpyDeviceToHost));
+      ptr = copy.data();
+    } else {
+      ptr = p;
+    }
+  }
+  const T* data() const { return ptr; }
+  const T& operator[](size_t i) const { return ptr[i]; }
+};
 
 template <typename T>
 T* upload(gcn_admm* h, const std::vector<T>& v) {
@@ -705,17 +715,17 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
     if (h->ld[l] / 4 > 256) throw Fail{GCN_ADMM_ERR_WIDTHS, "layer widths above 1024 are supported for C_0 only"};
 
   // host copies of the graph-side inputs, then the index tables
-  std::vector<long long> rp = to_host(row_ptr, (size_t)n + 1);
+  HostView<long long> rp(row_ptr, (size_t)n + 1);
   if (rp[n] < 0 || rp[0] != 0) throw Fail{GCN_ADMM_ERR_GRAPH, "row_ptr must start at 0 and be ascending"};
-  std::vector<int> ci = to_host(col_idx, (size_t)rp[n]);
-  std::vector<int> comm = to_host(community, (size_t)n);
-  std::vector<int> yy = to_host(y, (size_t)n);
-  std::vector<unsigned char> tm = to_host(train_mask, (size_t)n);
+  HostView<int> ci(col_idx, (size_t)rp[n]);
+  HostView<int> comm(community, (size_t)n);
+  HostView<int> yy(y, (size_t)n);
+  HostView<unsigned char> tm(train_mask, (size_t)n);
   std::string msg;
   const int rc = gcn_admm_host::build_graph_index(n, rp.data(), ci.data(), n_comm, comm.data(), h->gi, msg);
   if (rc == gcn_admm_host::IDX_BAD_GRAPH) throw Fail{GCN_ADMM_ERR_GRAPH, msg};
   if (rc == gcn_admm_host::IDX_BAD_COMMUNITY) throw Fail{GCN_ADMM_ERR_COMMUNITY, msg};
-  { std::vector<long long>().swap(rp); std::vector<int>().swap(ci); }
+  { std::vector<long long>().swap(rp.copy); std::vector<int>().swap(ci.copy); }
   const GraphIndex& g = h->gi;
   std::vector<int> y_new(n);
   std::vector<unsigned char> t_new(n);
@@ -741,7 +751,9 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
   h->d_dinv = upload(h, g.dinv);
   {
     std::vector<unsigned short> cc(g.col.size());
-    for (size_t e = 0; e < cc.size(); ++e) cc[e] = (unsigned short)g.row_comm[g.col[e]];
+    const long long n_entries = (long long)cc.size();
+#pragma omp parallel for schedule(static)
+    for (long long e = 0; e < n_entries; ++e) cc[e] = (unsigned short)g.row_comm[g.col[e]];
     h->d_col_comm = upload(h, cc);
   }
   h->d_y = upload(h, y_new);

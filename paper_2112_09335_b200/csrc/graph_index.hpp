@@ -33,20 +33,28 @@ inline int build_graph_index(long long n, const long long* row_ptr, const int* c
   for (long long i = 0; i < n; ++i)
     if (row_ptr[i + 1] < row_ptr[i]) { err = "row_ptr is not ascending"; return IDX_BAD_GRAPH; }
   if (row_ptr[n] + n > 2147483647LL) { err = "more than 2^31-1 stored entries"; return IDX_BAD_GRAPH; }
+  // Symmetry: every entry above the diagonal must have its mirror below it (a binary search in the
+  // sorted row), and there must be as many entries below as above; rows hold no duplicates, so the
+  // mirrors found are distinct and the counts then force every lower entry to be one of them.
   int bad = 0;
-#pragma omp parallel for schedule(dynamic, 4096) reduction(| : bad)
+  long long upper = 0, lower = 0;
+#pragma omp parallel for schedule(dynamic, 4096) reduction(| : bad) reduction(+ : upper, lower)
   for (long long i = 0; i < n; ++i) {
     for (long long p = row_ptr[i]; p < row_ptr[i + 1]; ++p) {
       const int j = col_idx[p];
       if (j < 0 || j >= n) { bad |= 1; continue; }
       if (p > row_ptr[i] && col_idx[p - 1] >= j) bad |= 2;
-      if (j != i) {  // symmetric: i must be stored in row j
+      if (j > i) {
+        ++upper;
         const int* lo = col_idx + row_ptr[j];
         const int* hi = col_idx + row_ptr[j + 1];
         if (!std::binary_search(lo, hi, (int)i)) bad |= 4;
+      } else if (j < i) {
+        ++lower;
       }
     }
   }
+  if (upper != lower) bad |= 4;
   if (bad & 1) { err = "column index out of range"; return IDX_BAD_GRAPH; }
   if (bad & 2) { err = "columns of a row are not strictly ascending"; return IDX_BAD_GRAPH; }
   if (bad & 4) { err = "adjacency is not symmetric"; return IDX_BAD_GRAPH; }
@@ -78,13 +86,15 @@ inline int build_graph_index(long long n, const long long* row_ptr, const int* c
   // A + I in new ids: row lengths, then columns (self loops of the input dropped, one identity)
   g.row_ptr.assign(n + 1, 0);
   g.dinv.resize(n);
+#pragma omp parallel for schedule(static)
   for (long long i = 0; i < n; ++i) {
     const long long o = g.perm[i];
     int deg = 0;
     for (long long p = row_ptr[o]; p < row_ptr[o + 1]; ++p) deg += (col_idx[p] != o);
-    g.row_ptr[i + 1] = g.row_ptr[i] + deg + 1;
+    g.row_ptr[i + 1] = deg + 1;
     g.dinv[i] = (float)(1.0 / std::sqrt((double)deg + 1.0));
   }
+  for (long long i = 0; i < n; ++i) g.row_ptr[i + 1] += g.row_ptr[i];
   g.nnz = g.row_ptr[n];
   g.col.resize(g.nnz);
   g.seg_row_ptr.assign(n + 1, 0);
