@@ -68,6 +68,11 @@ enum {
  *  schedule        0: Algorithm 1 (every W_l, then every Z_{l,m}, then U; Jacobi inside a pass);
  *                  1: the serial schedule of Section 4.1 (W_1, Z_1, .., W_L, Z_L, U one after the other,
  *                  each block reading the latest value of all others; the dual uses the new iterates)
+ *  long_row        rows of A + I with more stored entries than this are cut into work items of at most
+ *                  this many entries, each walked by a warp of its own, and the items' sums are added up
+ *                  in a fixed order afterwards (the paper's graphs have power-law degrees; a hub row
+ *                  walked by one warp would outlast the rest of the launch).  Same sums up to fp32
+ *                  rounding order.  0: the default, 256; a value above the longest row switches it off
  *  w_init          L host pointers to row-major C_{l-1} x C_l matrices (required)
  *  device          CUDA device ordinal;  stream: a cudaStream_t owned by the caller (NULL = the
  *                  default stream) */
@@ -83,13 +88,15 @@ typedef struct {
   int spmm_ring;
   int use_graph;
   int schedule;
+  int long_row;
   const float* const* w_init;
   int device;
   void* stream;
 } gcn_admm_params;
 
 /* Fills *p with the defaults: nu = rho = 1e-3, tau0 = theta0 = 1, growth 2, shrink 0.5,
- * 40 trials, 30 FISTA iterations, loss_scale 1, dual_mode 0, tensor_cores 1, spmm_ring 0, use_graph 2, schedule 0, device 0, stream NULL,
+ * 40 trials, 30 FISTA iterations, loss_scale 1, dual_mode 0, tensor_cores 1, spmm_ring 0, use_graph 2, schedule 0, long_row 0, device 0,
+ * stream NULL,
  * w_init NULL. */
 void gcn_admm_default_params(gcn_admm_params* p);
 

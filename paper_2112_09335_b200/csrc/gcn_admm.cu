@@ -2,6 +2,7 @@
 // kernels.cuh.  See include/gcn_admm.h for the contract of every entry point.
 #include "../../include/gcn_admm.h"
 
+#include <climits>
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -25,6 +26,7 @@ namespace {
 
 constexpr int kLogPasses = 256;
 constexpr int kSmCount = 148;
+constexpr int kDefaultLongRow = 256;   // stored entries one warp walks before a row is cut into items
 
 thread_local std::string g_create_error;
 
@@ -131,6 +133,11 @@ struct gcn_admm {
   int* d_y = nullptr;
   float* d_dinv = nullptr;
   unsigned short* d_col_comm = nullptr;   // community of every stored column
+  // rows too long for one warp, cut into items (see gcn_admm_host::LongRowTables)
+  int4 *d_items = nullptr, *d_split = nullptr, *d_long_rows = nullptr;
+  int n_items = 0, n_split = 0, n_long = 0, long_len = 0;
+  float* item_sums = nullptr;             // n_items x max_ld
+  size_t item_sums_elems = 0;
   unsigned char* d_train = nullptr;
 
   std::vector<float*> W, Wt, Z, P, H;   // 1..L
@@ -191,11 +198,16 @@ struct gcn_admm {
       CU(cudaGetLastError());
       return;
     }
-    // 64-thread blocks: rows differ widely in length, small blocks keep the SMs evenly loaded
+    // 64-thread blocks: rows differ widely in length, small blocks keep the SMs evenly loaded.
+    // Long rows go as items unless the operand is wider than the item buffer was sized for (a
+    // caller's matrix wider than every layer): then they are walked whole, slower but the same sums.
+    const bool cut = n_items > 0 && (size_t)n_items * ldx <= item_sums_elems;
+    const int items_used = cut ? n_items : 0;
 #define SPMM_CASE(G, V, UN)                                                                    \
   {                                                                                            \
-    const long long threads = n * (G);                                                         \
-    gk::k_spmm<G, V, UN><<<(unsigned)cdiv(threads, 64), 64, 0, stream>>>(d_row_ptr, d_col, d_dinv, x4, o4, nn, ld4); \
+    const long long threads = (n + items_used) * (G);                                          \
+    gk::k_spmm<G, V, UN><<<(unsigned)cdiv(threads, 64), 64, 0, stream>>>(d_row_ptr, d_col, d_dinv, x4, o4, nn, ld4, \
+        d_items, items_used, cut ? long_len : INT_MAX, reinterpret_cast<float4*>(item_sums));  \
   }
     if (ld4 <= 1) SPMM_CASE(1, 1, 4)
     else if (ld4 <= 2) SPMM_CASE(2, 1, 4)
@@ -206,6 +218,11 @@ struct gcn_admm {
     else SPMM_CASE(32, 2, 4)
 #undef SPMM_CASE
     CU(cudaGetLastError());
+    if (cut) {
+      gk::k_spmm_long_rows<<<(unsigned)n_long, 64, 0, stream>>>(d_long_rows, reinterpret_cast<const float4*>(item_sums), o4, ld4);
+      CU(cudaGetLastError());
+      ++launches;   // booked with the propagation it completes
+    }
   }
 
   // C = A B.  B is handed over twice: row-major K x N (ldb) for the fp32-ALU kernels and K-major
@@ -477,10 +494,16 @@ struct gcn_admm {
     CU(cudaMemsetAsync(row_counter, 0, sizeof(int), stream));                                             \
     int occ = 1;                                                                                          \
     CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gk::k_score_z<V, OUT>, warps * 32, dyn));      \
-    const unsigned grid = (unsigned)std::min<long long>(cdiv(n, warps), (long long)kSmCount * std::max(occ, 1)); \
+    const unsigned grid = (unsigned)std::min<long long>(cdiv(n + n_items, warps), (long long)kSmCount * std::max(occ, 1)); \
     gk::k_score_z<V, OUT><<<grid, warps * 32, dyn, stream>>>(d_row_ptr, d_col, d_col_comm, d_dinv,        \
         (const float4*)B1, (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0, ld4, (int)n, ctl, M, \
-        acc_z, n_active, use_smem, row_counter);                                                          \
+        acc_z, n_active, use_smem, row_counter, d_items, n_items, long_len, reinterpret_cast<float4*>(item_sums)); \
+    if (n_split > 0) {                                                                                    \
+      gk::k_score_z_split<V, OUT><<<(unsigned)cdiv(n_split, warps), warps * 32, 0, stream>>>(d_split, n_split, d_dinv, \
+          reinterpret_cast<const float4*>(item_sums), (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0, \
+          ld4, ctl, acc_z, n_active);                                                                     \
+      ++launches;                                                                                         \
+    }                                                                                                     \
   }
 #define SCORE_Z_ANY(OUT)                    \
   {                                         \
@@ -758,6 +781,18 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
   }
   h->d_y = upload(h, y_new);
   h->d_train = upload(h, t_new);
+  {
+    h->long_len = p.long_row > 0 ? p.long_row : kDefaultLongRow;
+    gcn_admm_host::LongRowTables lt;
+    gcn_admm_host::build_long_row_tables(g, h->long_len, lt);
+    static_assert(sizeof(gcn_admm_host::Quad) == sizeof(int4), "tables are uploaded as int4");
+    h->n_items = (int)lt.items.size();
+    h->n_split = (int)lt.split.size();
+    h->n_long = (int)lt.rows.size();
+    h->d_items = reinterpret_cast<int4*>(upload(h, lt.items));
+    h->d_split = reinterpret_cast<int4*>(upload(h, lt.split));
+    h->d_long_rows = reinterpret_cast<int4*>(upload(h, lt.rows));
+  }
 
   const int L = n_layers;
   const size_t rows = (size_t)n;
@@ -784,6 +819,8 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
   h->B0 = h->alloc<float>(rows * h->max_ld);
   h->B1 = h->alloc<float>(rows * h->max_ld);
   h->B2 = h->alloc<float>(rows * h->max_ld);
+  h->item_sums_elems = std::max<size_t>(1, (size_t)h->n_items * h->max_ld);
+  h->item_sums = h->alloc<float>(h->item_sums_elems);
   h->grad = h->alloc<float>(grad_elems);
   h->grad_t = h->alloc<float>(grad_t_elems);
   h->tc_error = h->alloc<int>(1);
@@ -884,6 +921,7 @@ void gcn_admm_default_params(gcn_admm_params* p) {
   p->spmm_ring = 0;
   p->use_graph = 2;
   p->schedule = 0;
+  p->long_row = 0;
   p->w_init = nullptr;
   p->device = 0;
   p->stream = nullptr;
@@ -904,7 +942,7 @@ int gcn_admm_create(gcn_admm** out, long long n, const long long* row_ptr, const
   for (int l = 0; l < n_layers; ++l)
     if (!p->w_init[l]) { g_create_error = "w_init holds a NULL pointer"; return GCN_ADMM_ERR_ARG; }
   if (!(p->nu > 0.f) || !(p->rho > 0.f) || !(p->bt_growth > 1.f) || !(p->bt_shrink > 0.f) || p->bt_max_trials < 1 ||
-      p->bt_max_trials > 64 || p->fista_iters < 0 || p->schedule < 0 || p->schedule > 1 || !(p->tau0 > 0.f) || !(p->theta0 > 0.f) || !(p->loss_scale > 0.f)) {
+      p->bt_max_trials > 64 || p->fista_iters < 0 || p->schedule < 0 || p->schedule > 1 || p->long_row < 0 || !(p->tau0 > 0.f) || !(p->theta0 > 0.f) || !(p->loss_scale > 0.f)) {
     g_create_error = "a parameter is out of range";
     return GCN_ADMM_ERR_ARG;
   }

@@ -131,6 +131,79 @@ inline int build_graph_index(long long n, const long long* row_ptr, const int* c
   return IDX_OK;
 }
 
+// ------------------------------------------------------------------------------------------
+// Work items for long rows.  Row lengths follow a power law, and a warp walks the stored entries
+// of its row one after the other: a row of thousands of entries keeps one warp busy long after
+// every other row is done.  Rows with more than `limit` stored entries are therefore cut into
+// items of at most `limit` entries, each handled by a warp of its own.  Cuts fall between
+// community segments wherever a segment fits (an item of whole segments can be scored without
+// help in the Z search); a segment longer than `limit` is cut into even pieces whose partial
+// sums are put together afterwards.
+//   items[k] = {row, first entry, one past the last entry, split}   split = -1: whole segments,
+//                                                                   else index into `split`
+//   split[s] = {row, community, first item, number of items}        (pieces are consecutive items)
+//   rows[r]  = {row, first item, number of items, 0}                (items of a row are consecutive)
+// ------------------------------------------------------------------------------------------
+struct Quad { int x, y, z, w; };
+struct LongRowTables {
+  std::vector<Quad> items, split, rows;
+};
+
+template <typename ItemFn, typename SplitFn>
+inline void walk_long_row(const GraphIndex& g, int row, int limit, ItemFn&& item, SplitFn&& split) {
+  int group_beg = g.row_ptr[row];
+  for (int s = g.seg_row_ptr[row]; s < g.seg_row_ptr[row + 1]; ++s) {
+    const int sb = g.seg_begin[s], se = g.seg_begin[s + 1], len = se - sb;
+    if (len > limit) {
+      if (sb > group_beg) item(group_beg, sb, false);
+      const int pieces = (len + limit - 1) / limit;
+      split(g.seg_comm[s], pieces);
+      for (int k = 0; k < pieces; ++k)
+        item(sb + (int)((long long)len * k / pieces), sb + (int)((long long)len * (k + 1) / pieces), true);
+      group_beg = se;
+    } else if (se - group_beg > limit) {
+      item(group_beg, sb, false);
+      group_beg = sb;
+    }
+  }
+  if (group_beg < g.row_ptr[row + 1]) item(group_beg, g.row_ptr[row + 1], false);
+}
+
+inline void build_long_row_tables(const GraphIndex& g, int limit, LongRowTables& t) {
+  t.items.clear(); t.split.clear(); t.rows.clear();
+  std::vector<int> long_rows;
+  for (long long i = 0; i < g.n; ++i)
+    if (g.row_ptr[i + 1] - g.row_ptr[i] > limit) long_rows.push_back((int)i);
+  const long long nl = (long long)long_rows.size();
+  if (nl == 0) return;
+  std::vector<long long> item_at(nl + 1, 0), split_at(nl + 1, 0);
+#pragma omp parallel for schedule(dynamic, 256)
+  for (long long r = 0; r < nl; ++r) {
+    long long ni = 0, ns = 0;
+    walk_long_row(g, long_rows[r], limit, [&](int, int, bool) { ++ni; }, [&](int, int) { ++ns; });
+    item_at[r + 1] = ni;
+    split_at[r + 1] = ns;
+  }
+  for (long long r = 0; r < nl; ++r) { item_at[r + 1] += item_at[r]; split_at[r + 1] += split_at[r]; }
+  t.items.resize((size_t)item_at[nl]);
+  t.split.resize((size_t)split_at[nl]);
+  t.rows.resize((size_t)nl);
+#pragma omp parallel for schedule(dynamic, 256)
+  for (long long r = 0; r < nl; ++r) {
+    const int row = long_rows[r];
+    long long ni = item_at[r], ns = split_at[r];
+    int cur_split = -1;
+    walk_long_row(
+        g, row, limit,
+        [&](int b, int e, bool piece) { t.items[(size_t)ni++] = Quad{row, b, e, piece ? cur_split : -1}; },
+        [&](int comm, int pieces) {
+          cur_split = (int)ns;
+          t.split[(size_t)ns++] = Quad{row, comm, (int)ni, pieces};
+        });
+    t.rows[(size_t)r] = Quad{row, (int)item_at[r], (int)(item_at[r + 1] - item_at[r]), 0};
+  }
+}
+
 // First-order neighbour rows of community m: new ids outside V_m adjacent to V_m, ascending.
 inline std::vector<int> halo1_of(const GraphIndex& g, int m) {
   std::vector<int> out;

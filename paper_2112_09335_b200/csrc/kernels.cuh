@@ -69,17 +69,35 @@ __device__ __forceinline__ double block_sum(double v, double* sh) {
 // Propagation  out = A~ x,  A~_ij = dinv_i dinv_j on the pattern of A + I (Problem 1).
 // G lanes share one row; each lane owns the float4 columns lane, lane+G, .. of a block of
 // G*V float4 columns; wider rows loop over column blocks.
+// A lane group walks its stored entries one after the other, so a row of thousands of entries
+// (row lengths follow a power law) would keep one warp busy long after the rest of the grid is
+// done.  Rows longer than `long_len` are therefore not handled as rows: they come as `n_items`
+// items {row, first entry, one past the last} (first in the grid), whose partial sums go to
+// `scratch` (one padded row per item) and are added up, in item order, by k_spmm_long_rows.
 // ------------------------------------------------------------------------------------------
 template <int G, int V, int UN>
 __global__ void __launch_bounds__(256)
 k_spmm(const int* __restrict__ row_ptr, const int* __restrict__ col, const float* __restrict__ dinv,
-       const float4* __restrict__ x, float4* __restrict__ out, int n, int ld4) {
+       const float4* __restrict__ x, float4* __restrict__ out, int n, int ld4,
+       const int4* __restrict__ items, int n_items, int long_len, float4* __restrict__ scratch) {
   const int lane = threadIdx.x & 31;
   const int gl = lane & (G - 1);
   const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << (lane & ~(G - 1)));
-  const long long row = ((long long)blockIdx.x * blockDim.x + threadIdx.x) / G;
-  if (row >= n) return;
-  const int rs = row_ptr[row], re = row_ptr[row + 1];
+  const long long unit = ((long long)blockIdx.x * blockDim.x + threadIdx.x) / G;
+  if (unit >= (long long)n + n_items) return;
+  long long row;
+  int rs, re;
+  float4* dst;
+  if (unit < n_items) {
+    const int4 it = items[unit];
+    row = it.x; rs = it.y; re = it.z;
+    dst = scratch + unit * ld4;
+  } else {
+    row = unit - n_items;
+    rs = row_ptr[row]; re = row_ptr[row + 1];
+    if (re - rs > long_len) return;
+    dst = out + row * ld4;
+  }
   const float di = dinv[row];
   for (int cb = 0; cb < ld4; cb += G * V) {
     float4 acc[V];
@@ -122,8 +140,23 @@ k_spmm(const int* __restrict__ row_ptr, const int* __restrict__ col, const float
     for (int v = 0; v < V; ++v) {
       const int f = cb + gl + G * v;
       if (f < ld4)
-        out[row * ld4 + f] = make_float4(di * acc[v].x, di * acc[v].y, di * acc[v].z, di * acc[v].w);
+        dst[f] = make_float4(di * acc[v].x, di * acc[v].y, di * acc[v].z, di * acc[v].w);
     }
+  }
+}
+
+// Rows that k_spmm handled as items: out[row] = sum of the row's item sums, in item order.
+// rows[r] = {row, first item, number of items}; one block per row.
+__global__ void k_spmm_long_rows(const int4* __restrict__ rows, const float4* __restrict__ scratch,
+                                 float4* __restrict__ out, int ld4) {
+  const int4 r = rows[blockIdx.x];
+  for (int f = threadIdx.x; f < ld4; f += blockDim.x) {
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int k = 0; k < r.z; ++k) {
+      const float4 v = scratch[(long long)(r.y + k) * ld4 + f];
+      s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+    out[(long long)r.x * ld4 + f] = s;
   }
 }
 
@@ -885,13 +918,66 @@ __device__ __forceinline__ float warp_sum2(float v0, float v1, int lane) {
 // Sums are kept per warp in shared memory (no atomics on the hot path) and added to `acc` once per
 // block; with too many communities for that (use_smem == 0) they go to `acc` directly.
 // V = float4 columns per lane (width <= 128 V).  Persistent grid; `row_counter` must be zero at launch.
+//
+// Rows longer than `long_len` come as `n_items` items {row, first entry, one past the last, split}
+// (see k_spmm): an item of whole community segments (split < 0) is scored like a short row; an
+// item that is one piece of a segment too long for one warp only leaves its part of K_m[i],
+// unscaled, in `scratch` (one padded row per item), and k_score_z_split scores the sum of the pieces.
+
+// Scores one finished K_m[i] (k, still without the factor di) against the row's a, b.
+template <int V, bool OUT>
+__device__ __forceinline__ void score_segment(const float4 (&k)[V], float di, const float4 (&a)[V],
+                                              const float4 (&b)[V], const SearchCtl* __restrict__ ctl,
+                                              int cur, int lane, double* mine, bool plain_add) {
+  if (OUT) {
+    float p1 = 0.f, p2 = 0.f;
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+      const float kx = di * k[v].x, ky = di * k[v].y, kz = di * k[v].z, kw = di * k[v].w;
+      p1 += kx * a[v].x + ky * a[v].y + kz * a[v].z + kw * a[v].w;
+      p2 += kx * kx + ky * ky + kz * kz + kw * kw;
+    }
+    const float r = warp_sum2(p1, p2, lane);
+    if ((lane & 15) == 0) {
+      double* dst = mine + cur * 2 + (lane >> 4);
+      if (plain_add) *dst += (double)r; else atomicAdd(dst, (double)r);
+    }
+  } else {
+    float inv[kCand], part[kCand];
+#pragma unroll
+    for (int j = 0; j < kCand; ++j) { inv[j] = ctl[cur].inv_cand[j]; part[j] = 0.f; }
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+      const float kk[4] = {di * k[v].x, di * k[v].y, di * k[v].z, di * k[v].w};
+      const float hh[4] = {a[v].x, a[v].y, a[v].z, a[v].w};
+      const float zz[4] = {b[v].x, b[v].y, b[v].z, b[v].w};
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const float e0 = zz[c] - relu(hh[c]);
+#pragma unroll
+        for (int j = 0; j < kCand; ++j) {
+          const float df = relu_drop(hh[c], kk[c] * inv[j]);
+          part[j] = fmaf(df, fmaf(2.f, e0, df), part[j]);
+        }
+      }
+    }
+    static_assert(kCand == 4, "warp_sum4 reduces exactly four candidates");
+    const float r = warp_sum4(part[0], part[1], part[2], part[3], lane);
+    if ((lane & 7) == 0) {
+      double* dst = mine + cur * kCand + (lane >> 3);
+      if (plain_add) *dst += (double)r; else atomicAdd(dst, (double)r);
+    }
+  }
+}
+
 template <int V, bool OUT>
 __global__ void __launch_bounds__(256)
 k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
           const unsigned short* __restrict__ col_comm, const float* __restrict__ dinv,
           const float4* __restrict__ T, const float4* __restrict__ Hn, const float4* __restrict__ Zn,
           const float4* __restrict__ Rn, int ld4, int n, const SearchCtl* __restrict__ ctl, int n_comm,
-          double* __restrict__ acc, const int* __restrict__ n_active, int use_smem, int* __restrict__ row_counter) {
+          double* __restrict__ acc, const int* __restrict__ n_active, int use_smem, int* __restrict__ row_counter,
+          const int4* __restrict__ items, int n_items, int long_len, float4* __restrict__ scratch) {
   if (*n_active <= 0) return;
   constexpr int PER = OUT ? 2 : kCand;
   extern __shared__ double s_acc[];
@@ -903,21 +989,34 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
     __syncthreads();
     mine = s_acc + (size_t)warp * n_comm * PER;
   }
-  // rows are handed out four at a time from a global counter: row lengths follow a power law, a
-  // static deal leaves most warps waiting at the closing barrier for the unlucky ones
+  const bool plain_add = use_smem != 0;
+  const int n_units = n + n_items;
+  // units (items first, then rows) are handed out four at a time from a global counter: row lengths
+  // follow a power law, a static deal leaves most warps waiting at the closing barrier for the unlucky ones
   for (;;) {
-    int row_base = 0;
-    if (lane == 0) row_base = atomicAdd(row_counter, 4);
-    row_base = __shfl_sync(0xffffffffu, row_base, 0);
-    if (row_base >= n) break;
-    const int row_end = min(n, row_base + 4);
-  for (int row = row_base; row < row_end; ++row) {
+    int unit_base = 0;
+    if (lane == 0) unit_base = atomicAdd(row_counter, 4);
+    unit_base = __shfl_sync(0xffffffffu, unit_base, 0);
+    if (unit_base >= n_units) break;
+    const int unit_end = min(n_units, unit_base + 4);
+  for (int unit = unit_base; unit < unit_end; ++unit) {
+    int row, rs, re;
+    bool piece = false;
+    if (unit < n_items) {
+      const int4 it = items[unit];
+      row = it.x; rs = it.y; re = it.z;
+      piece = it.w >= 0;
+    } else {
+      row = unit - n_items;
+      rs = row_ptr[row]; re = row_ptr[row + 1];
+      if (re - rs > long_len) continue;
+    }
     float4 a[V], b[V];   // OUT: a = R' ; else a = h, b = z
 #pragma unroll
     for (int v = 0; v < V; ++v) {
       const int f = lane + 32 * v;
       a[v] = b[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (f < ld4) {
+      if (f < ld4 && !piece) {
         if (OUT) a[v] = Rn[(long long)row * ld4 + f];
         else { a[v] = Hn[(long long)row * ld4 + f]; b[v] = Zn[(long long)row * ld4 + f]; }
       }
@@ -931,48 +1030,17 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
 
     auto finish_segment = [&]() {
       if (!cur_on) return;
-      if (OUT) {
-        float p1 = 0.f, p2 = 0.f;
+      if (piece) {
 #pragma unroll
         for (int v = 0; v < V; ++v) {
-          const float kx = di * k[v].x, ky = di * k[v].y, kz = di * k[v].z, kw = di * k[v].w;
-          p1 += kx * a[v].x + ky * a[v].y + kz * a[v].z + kw * a[v].w;
-          p2 += kx * kx + ky * ky + kz * kz + kw * kw;
+          const int f = lane + 32 * v;
+          if (f < ld4) scratch[(long long)unit * ld4 + f] = k[v];
         }
-        const float r = warp_sum2(p1, p2, lane);
-        if ((lane & 15) == 0) {
-          double* dst = mine + cur * 2 + (lane >> 4);
-          if (use_smem) *dst += (double)r; else atomicAdd(dst, (double)r);
-        }
-      } else {
-        float inv[kCand], part[kCand];
-#pragma unroll
-        for (int j = 0; j < kCand; ++j) { inv[j] = ctl[cur].inv_cand[j]; part[j] = 0.f; }
-#pragma unroll
-        for (int v = 0; v < V; ++v) {
-          const float kk[4] = {di * k[v].x, di * k[v].y, di * k[v].z, di * k[v].w};
-          const float hh[4] = {a[v].x, a[v].y, a[v].z, a[v].w};
-          const float zz[4] = {b[v].x, b[v].y, b[v].z, b[v].w};
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const float e0 = zz[c] - relu(hh[c]);
-#pragma unroll
-            for (int j = 0; j < kCand; ++j) {
-              const float df = relu_drop(hh[c], kk[c] * inv[j]);
-              part[j] = fmaf(df, fmaf(2.f, e0, df), part[j]);
-            }
-          }
-        }
-        static_assert(kCand == 4, "warp_sum4 reduces exactly four candidates");
-        const float r = warp_sum4(part[0], part[1], part[2], part[3], lane);
-        if ((lane & 7) == 0) {
-          double* dst = mine + cur * kCand + (lane >> 3);
-          if (use_smem) *dst += (double)r; else atomicAdd(dst, (double)r);
-        }
+        return;
       }
+      score_segment<V, OUT>(k, di, a, b, ctl, cur, lane, mine, plain_add);
     };
 
-    const int rs = row_ptr[row], re = row_ptr[row + 1];
     for (int base = rs; base < re; base += 32) {
       const int idx = base + lane;
       int c = 0, m = -1;
@@ -1033,6 +1101,37 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
       if (t != 0.0) atomicAdd(acc + i, t);
     }
   }
+}
+
+// Segments that k_score_z handled in pieces: K_m[i] = sum of the pieces (item order), then scored
+// as above.  split[s] = {row, community, first item, number of items}; one warp per entry.
+template <int V, bool OUT>
+__global__ void __launch_bounds__(256)
+k_score_z_split(const int4* __restrict__ split, int n_split, const float* __restrict__ dinv,
+                const float4* __restrict__ scratch, const float4* __restrict__ Hn, const float4* __restrict__ Zn,
+                const float4* __restrict__ Rn, int ld4, const SearchCtl* __restrict__ ctl,
+                double* __restrict__ acc, const int* __restrict__ n_active) {
+  if (*n_active <= 0) return;
+  const int lane = threadIdx.x & 31;
+  const int s = (int)(((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+  if (s >= n_split) return;
+  const int4 sp = split[s];
+  if (ctl[sp.y].done) return;
+  float4 a[V], b[V], k[V];
+#pragma unroll
+  for (int v = 0; v < V; ++v) {
+    const int f = lane + 32 * v;
+    a[v] = b[v] = k[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (f < ld4) {
+      if (OUT) a[v] = Rn[(long long)sp.x * ld4 + f];
+      else { a[v] = Hn[(long long)sp.x * ld4 + f]; b[v] = Zn[(long long)sp.x * ld4 + f]; }
+      for (int q = 0; q < sp.w; ++q) {
+        const float4 t = scratch[(long long)(sp.z + q) * ld4 + f];
+        k[v].x += t.x; k[v].y += t.y; k[v].z += t.z; k[v].w += t.w;
+      }
+    }
+  }
+  score_segment<V, OUT>(k, dinv[sp.x], a, b, ctl, sp.y, lane, acc, false);
 }
 
 // Z_l[i,:] <- Z_l[i,:] - G[i,:] / theta_{comm(i)}   (Eq. 10)

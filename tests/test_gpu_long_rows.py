@@ -1,0 +1,86 @@
+"""Long rows cut into work items (`long_row`): with a limit of a few entries almost every row of the
+small parity cases goes through the item path (propagation items, whole-segment items and split
+segments of the Z scoring), and the results must still match the fp64 oracle and the uncut path."""
+import numpy as np
+import pytest
+
+from oracle import gcn_admm_oracle as orc
+from paper_2112_09335_b200 import binding, inputs
+from parity_utils import forced_from, make_oracle, relerr
+
+pytestmark = pytest.mark.gpu
+
+CASES = [("cfg0/3", lambda: inputs.make_workload(0), 3),
+         ("cfg0/1", lambda: inputs.make_workload(0), 1),
+         ("cfg2@0.15/3", lambda: inputs.make_workload(2, scale=0.15), 3),
+         ("cfg3@0.012/8", lambda: inputs.make_workload(3, scale=0.012), 8),
+         ("cfg4@0.001/5", lambda: inputs.make_workload(4, scale=0.001), 5),
+         ("cfg3@0.012 M=1/6", lambda: inputs.make_workload(3, scale=0.012, n_comm=1), 6)]
+
+
+def handle(wl, **kw):
+    return binding.GcnAdmm(wl.n, wl.row_ptr, wl.col_idx, wl.X, wl.y, wl.train_mask, wl.widths, wl.n_comm, wl.community,
+                           wl.w_init, nu=wl.nu, rho=wl.rho, **kw)
+
+
+@pytest.fixture(scope="module", params=CASES, ids=lambda c: c[0])
+def case(request):
+    name, make, limit = request.param
+    wl = make()
+    deg = np.diff(np.asarray(wl.row_ptr)) + 1
+    assert (deg > limit).mean() > 0.3, "the case must send a good share of its rows through the item path"
+    g = handle(wl, long_row=limit)
+    yield wl, g, limit
+    g.destroy()
+
+
+@pytest.mark.parametrize("width", [1, 5, 47, 128, 256, 300])
+def test_propagation_with_cut_rows(case, width):
+    wl, g, _ = case
+    At = orc.normalized_adjacency(wl.n, wl.row_ptr, wl.col_idx)
+    x = np.random.default_rng(width).standard_normal((wl.n, width)).astype(np.float32)
+    got = g.propagate(x)
+    want = At @ x.astype(np.float64)
+    scale = abs(At) @ np.abs(x.astype(np.float64)) + 1e-30
+    assert np.max(np.abs(got - want) / scale) < 1e-6
+
+
+def test_three_passes_equal_the_uncut_path(case):
+    """Same decisions, same step-size ratios and the same iterates (to rounding order) as with whole rows."""
+    wl, _, limit = case
+    a, b = handle(wl, long_row=limit), handle(wl, long_row=1 << 30)
+    try:
+        a.step(3)
+        b.step(3)
+        da, db = a.decisions(), b.decisions()
+        assert np.array_equal(da["trial_w"], db["trial_w"]) and np.array_equal(da["trial_z"], db["trial_z"])
+        np.testing.assert_allclose(da["q_z"], db["q_z"], rtol=2e-4, atol=1e-6)
+        for l in range(1, a.L + 1):
+            assert relerr(a.get_state(binding.ST_W, l), b.get_state(binding.ST_W, l)) < 1e-5
+            assert relerr(a.get_state(binding.ST_Z, l), b.get_state(binding.ST_Z, l)) < 1e-5
+        assert relerr(a.get_state(binding.ST_U), b.get_state(binding.ST_U)) < 1e-5
+    finally:
+        a.destroy()
+        b.destroy()
+
+
+@pytest.mark.parametrize("schedule", [0, 1])
+def test_ten_iterations_with_cut_rows(case, schedule):
+    wl, _, limit = case
+    g = handle(wl, long_row=limit, schedule=schedule)
+    o = make_oracle(wl)
+    try:
+        g.step(10)
+        dec = g.decisions()
+        assert (dec["trial_w"] >= -1).all() and (dec["trial_z"] >= -1).all()
+        o.forced_tol = 1e-4
+        for k in range(10):
+            forced = forced_from(dec, k, o.L, o.M)
+            rec = o.iterate_sequential(forced) if schedule else o.iterate(forced)
+            assert all(r["ok"] for r in list(rec["W"].values()) + list(rec["Z"].values())), k
+        for l in range(1, o.L + 1):
+            assert relerr(g.get_state(binding.ST_W, l), o.W[l]) <= 1e-3
+            assert relerr(g.get_state(binding.ST_Z, l), o.Z[l]) <= 1e-3
+        assert relerr(g.get_state(binding.ST_U), o.U) <= 1e-3
+    finally:
+        g.destroy()
