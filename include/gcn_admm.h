@@ -57,7 +57,10 @@ enum {
  *  tensor_cores    1: dense products with at most 256 output columns and K <= 512 run on the tensor
  *                  cores as an error-compensated TF32 product (three passes, fp32 accumulation,
  *                  relative error of a few 1e-7 of sum |a||b|); 2: the same product with its earlier, unsplit
- *                  scheduling (kept for comparison); 0: fp32 FMA kernels everywhere
+ *                  scheduling (kept for comparison); 0: fp32 FMA kernels everywhere.  With 1, products of
+ *                  16384 rows or more first split the weight operand once into the staged layout and
+ *                  fetch it with bulk copies (smaller ones re-split it per row tile, which is cheaper
+ *                  than another launch); 3: the same kernels, pre-split at every size
  *  spmm_ring       0: propagation gathers neighbour rows into registers; 1: rows of 68..256 floats are
  *                  kept in flight in a shared-memory ring filled with cp.async instead (same result; both
  *                  forms run at the same ~10 TB/s of gathered bytes on B200, the ring is kept for comparison)

@@ -26,6 +26,7 @@ namespace {
 
 constexpr int kLogPasses = 256;
 constexpr int kSmCount = 148;
+constexpr long long kImageMinRows = 16384;   // row count from which the weight operand is pre-split
 constexpr int kDefaultLongRow = 256;   // stored entries one warp walks before a row is cut into items
 
 thread_local std::string g_create_error;
@@ -146,6 +147,8 @@ struct gcn_admm {
   float* grad = nullptr;     // max over l of C_{l-1} x ld_l
   float* grad_t = nullptr;   // its transpose, C_l x ld_{l-1} (K-major operand of the tensor-core product)
   int* tc_error = nullptr;   // raised by a tensor-core product whose bounded wait ran out
+  uint8_t* b_image = nullptr;   // split weight operand in the staged layout (see gtc::k_split_b)
+  size_t b_image_bytes = 0;
   float* part = nullptr;     // split partial sums of the transposed product
   size_t part_elems = 0;
   SearchCtl *ctl_w = nullptr, *ctl_z = nullptr;   // [L+1], [(L+1) * M]
@@ -231,18 +234,30 @@ struct gcn_admm {
   void gemm_nn(const float* A, int lda, const float* B, int ldb, const float* Bk, int ldbk, float* Cm, int ldc,
                long long Mr, int N, int K, const int* skip = nullptr) {
     char name[48];
-    if (p.tensor_cores && Bk != nullptr && K >= 8 && K <= 2048 && Mr >= 512 && (p.tensor_cores == 1 || (N <= 256 && K <= 512))) {
+    if (p.tensor_cores && Bk != nullptr && K >= 8 && K <= 2048 && Mr >= 512 && (p.tensor_cores == 1 || p.tensor_cores == 3 || (N <= 256 && K <= 512))) {
       std::snprintf(name, sizeof name, "gemm_tc@%dx%d", K, N);
       Scope sc(this, name, 1, 4.0 * ((double)Mr * (lda + ldc) + (double)K * ldb), 2.0 * (double)Mr * N * K);
       const int tiles = (int)cdiv(Mr, gtc::kBlockM);
-      if (p.tensor_cores == 1) {   // role-split kernel: producers / MMA issue / epilogue overlap
+      if (p.tensor_cores == 1 || p.tensor_cores == 3) {   // role-split kernel: producers / MMA issue / epilogue overlap
+      // With many row tiles the weight operand is split once into an image of the staged layout and
+      // fetched by bulk copies; with few (launch-bound problems) the extra launch costs more than the
+      // producers' repeated work.  tensor_cores = 3 takes the image at every size.
 #define TC_WS(NT)                                                                                              \
   {                                                                                                            \
     const size_t smem = gtc::WsCfg<NT>::kSmem;                                                                 \
     const int groups = (int)cdiv(N, NT);                                                                       \
-    CU(cudaFuncSetAttribute(gtc::k_gemm_tc_ws<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));   \
+    const size_t image_bytes = (size_t)groups * cdiv(K, gtc::kChunkK) * 2 * (NT) * gtc::kChunkK * 4;            \
     dim3 grid((unsigned)std::max(1, std::min(tiles, kSmCount / groups)), (unsigned)groups);                    \
-    gtc::k_gemm_tc_ws<NT><<<grid, gtc::kWsThreads, smem, stream>>>(A, lda, Bk, ldbk, Cm, ldc, (int)Mr, N, K, skip, tc_error); \
+    if ((p.tensor_cores == 3 || Mr >= kImageMinRows) && image_bytes <= b_image_bytes) {                        \
+      const long long work = (long long)groups * cdiv(K, gtc::kChunkK) * (NT) * 8;                             \
+      gtc::k_split_b<<<(unsigned)std::min<long long>(cdiv(work, 256), 4 * kSmCount), 256, 0, stream>>>(Bk, ldbk, N, K, NT, b_image); \
+      ++launches;                                                                                              \
+      CU(cudaFuncSetAttribute(gtc::k_gemm_tc_ws<NT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+      gtc::k_gemm_tc_ws<NT, true><<<grid, gtc::kWsThreads, smem, stream>>>(A, lda, Bk, ldbk, Cm, ldc, (int)Mr, N, K, skip, tc_error, b_image); \
+    } else {                                                                                                   \
+      CU(cudaFuncSetAttribute(gtc::k_gemm_tc_ws<NT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+      gtc::k_gemm_tc_ws<NT, false><<<grid, gtc::kWsThreads, smem, stream>>>(A, lda, Bk, ldbk, Cm, ldc, (int)Mr, N, K, skip, tc_error, nullptr); \
+    }                                                                                                          \
   }
         if (N <= 16) TC_WS(16)
         else if (N <= 32) TC_WS(32)
@@ -314,7 +329,7 @@ struct gcn_admm {
     int splits = 1;
     long long rps = rows;
     char name[48];
-    if (p.tensor_cores == 1 && rows >= 4096) {
+    if ((p.tensor_cores == 1 || p.tensor_cores == 3) && rows >= 4096) {
       std::snprintf(name, sizeof name, "gemm_tn_tc@%dx%d", Ka, Nb);
       Scope sc(this, name, 2, 4.0 * ((double)rows * (lda + ldb) + (double)Ka * ldp), 2.0 * (double)rows * Ka * Nb);
       const int nt_tn = Nb <= 16 ? 16 : Nb <= 32 ? 32 : Nb <= 48 ? 48 : Nb <= 64 ? 64 : Nb <= 128 ? 128 : 256;
@@ -824,6 +839,8 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
   h->grad = h->alloc<float>(grad_elems);
   h->grad_t = h->alloc<float>(grad_t_elems);
   h->tc_error = h->alloc<int>(1);
+  h->b_image_bytes = (size_t)16 << 20;   // e.g. 1024 columns x 2048 K
+  h->b_image = h->alloc<uint8_t>(h->b_image_bytes);
   CU(cudaMemset(h->tc_error, 0, sizeof(int)));
   CU(cudaMemset(h->grad_t, 0, grad_t_elems * sizeof(float)));
   h->part = h->alloc<float>(h->part_elems);

@@ -530,10 +530,36 @@ struct WsCfg {
   static constexpr size_t kSmem = (size_t)kStagesWs * kStage + 1024;
 };
 
-template <int NT>
+// The weight operand split once, in the layout the MMA descriptors read: for column group g and K
+// chunk kc, the 128-byte-swizzled NT x 32 tile of B_hi followed by that of B_lo, one contiguous block
+// of 2 * NT * 128 bytes at block index g * chunks + kc.  With it (IMG = true) a stage's B tiles arrive
+// by one bulk copy issued by one thread, and the producers stage A only; without it they load, split
+// and store B again for every 128-row tile.
+__global__ void k_split_b(const float* __restrict__ Bk, int ldbk, int N, int K, int nt, uint8_t* __restrict__ image) {
+  const int kc_count = (K + kChunkK - 1) / kChunkK;
+  const int groups = (N + nt - 1) / nt;
+  const long long total = (long long)groups * kc_count * nt * 8;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const int c16 = (int)(i & 7);
+    const int nrow = (int)((i >> 3) % nt);
+    const long long blk = i / (8LL * nt);
+    const int kc = (int)(blk % kc_count), g = (int)(blk / kc_count);
+    const int k0 = kc * kChunkK + c16 * 4, n = g * nt + nrow;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (n < N && k0 < K) v = *reinterpret_cast<const float4*>(Bk + (long long)n * ldbk + k0);
+    float4 h, l;
+    split_tf32(v.x, h.x, l.x); split_tf32(v.y, h.y, l.y); split_tf32(v.z, h.z, l.z); split_tf32(v.w, h.w, l.w);
+    uint8_t* dst = image + (size_t)blk * (size_t)(2 * nt * kChunkK * 4) + swz(nrow, c16);
+    *reinterpret_cast<float4*>(dst) = h;
+    *reinterpret_cast<float4*>(dst + (size_t)nt * kChunkK * 4) = l;
+  }
+}
+
+template <int NT, bool IMG>
 __global__ void __launch_bounds__(kWsThreads, 1)
 k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk, int ldbk, float* __restrict__ C, int ldc,
-             int M, int N, int K, const int* __restrict__ skip, int* __restrict__ error_flag) {
+             int M, int N, int K, const int* __restrict__ skip, int* __restrict__ error_flag,
+             const uint8_t* __restrict__ b_image) {
   using Cfg = WsCfg<NT>;
   constexpr int S = Cfg::kStagesWs;
   constexpr int B_PASSES = (NT + 31) / 32;
@@ -580,7 +606,7 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
   if (warp < 8) {
     // ---------------- producers ----------------
     const int ld_c16 = tid & 7, ld_row = tid >> 3;
-    float4 ra[2][A_PASSES], rb[2][B_PASSES];
+    float4 ra[2][A_PASSES], rb[2][IMG ? 1 : B_PASSES];
     auto load_chunk = [&](int j, float4* pa, float4* pb) {
       if (j >= total) return;
       const int tile = blockIdx.x + (j / kc_count) * gridDim.x, kc = j % kc_count;
@@ -595,14 +621,16 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
         }
         pa[i] = v;
       }
+      if (!IMG) {
 #pragma unroll
-      for (int i = 0; i < B_PASSES; ++i) {
-        const int nrow = ld_row + 32 * i;
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (nrow < n_loc && k0 < K) {
-          v = *reinterpret_cast<const float4*>(Bk + (long long)(n0 + nrow) * ldbk + k0);
+        for (int i = 0; i < B_PASSES; ++i) {
+          const int nrow = ld_row + 32 * i;
+          float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (nrow < n_loc && k0 < K) {
+            v = *reinterpret_cast<const float4*>(Bk + (long long)(n0 + nrow) * ldbk + k0);
+          }
+          pb[i] = v;
         }
-        pb[i] = v;
       }
     };
     auto store_chunk = [&](int stage, const float4* pa, const float4* pb) {
@@ -616,16 +644,18 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
         *reinterpret_cast<float4*>(st + off) = h;
         *reinterpret_cast<float4*>(st + kATileBytes + off) = l;
       }
+      if (!IMG) {
 #pragma unroll
-      for (int i = 0; i < B_PASSES; ++i) {
-        const int nrow = ld_row + 32 * i;
-        if (nrow < NT) {
-          float4 h, l;
-          split_tf32(pb[i].x, h.x, l.x); split_tf32(pb[i].y, h.y, l.y);
-          split_tf32(pb[i].z, h.z, l.z); split_tf32(pb[i].w, h.w, l.w);
-          const uint32_t off = swz(nrow, ld_c16);
-          *reinterpret_cast<float4*>(st + 2 * kATileBytes + off) = h;
-          *reinterpret_cast<float4*>(st + 2 * kATileBytes + Cfg::kBTile + off) = l;
+        for (int i = 0; i < B_PASSES; ++i) {
+          const int nrow = ld_row + 32 * i;
+          if (nrow < NT) {
+            float4 h, l;
+            split_tf32(pb[i].x, h.x, l.x); split_tf32(pb[i].y, h.y, l.y);
+            split_tf32(pb[i].z, h.z, l.z); split_tf32(pb[i].w, h.w, l.w);
+            const uint32_t off = swz(nrow, ld_c16);
+            *reinterpret_cast<float4*>(st + 2 * kATileBytes + off) = h;
+            *reinterpret_cast<float4*>(st + 2 * kATileBytes + Cfg::kBTile + off) = l;
+          }
         }
       }
     };
@@ -634,6 +664,17 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
     for (int j = 0; j < total; ++j) {
       const int stage = j % S;
       if (j >= S && !mbar_wait_abortable(bar_empty + 8 * stage, ((j / S) - 1) & 1, abortp)) break;
+      if (IMG && tid == 0) {
+        // the stage is free (its MMAs have retired): fetch both B tiles of this chunk with one bulk copy
+        // that reports its bytes to the stage's full barrier; this thread's own arrival comes below
+        const uint32_t bytes = 2u * (uint32_t)Cfg::kBTile;
+        const uint8_t* src = b_image + ((size_t)blockIdx.y * kc_count + (size_t)(j % kc_count)) * bytes;
+        const uint32_t dst = smem_base + (uint32_t)stage * Cfg::kStage + 2u * kATileBytes;
+        asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar_full + 8 * stage), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(dst), "l"(src), "r"(bytes), "r"(bar_full + 8 * stage)
+                     : "memory");
+      }
       if (j & 1) { store_chunk(stage, ra[1], rb[1]); load_chunk(j + 2, ra[1], rb[1]); }
       else       { store_chunk(stage, ra[0], rb[0]); load_chunk(j + 2, ra[0], rb[0]); }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

@@ -8,7 +8,7 @@ from paper_2112_09335_b200 import binding, inputs
 pytestmark = pytest.mark.gpu
 
 SHAPES = [(1000, 16, 128), (5000, 256, 256), (4097, 256, 100), (3000, 47, 256), (2049, 16, 1433), (700, 5, 37),
-          (130, 256, 8), (40000, 128, 500), (777, 3, 128), (12345, 40, 256), (9000, 1000, 767), (6000, 10, 1000), (3000, 300, 64)]    # (m, n, k)
+          (130, 256, 8), (40000, 128, 500), (33000, 256, 256), (20001, 47, 256), (16384, 256, 100), (777, 3, 128), (12345, 40, 256), (9000, 1000, 767), (6000, 10, 1000), (3000, 300, 64)]    # (m, n, k)
 
 
 @pytest.fixture(scope="module")
@@ -20,7 +20,7 @@ def handle():
     g.destroy()
 
 
-@pytest.mark.parametrize("tensor_cores", [1, 2, 0])
+@pytest.mark.parametrize("tensor_cores", [1, 3, 2, 0])     # 3: weight operand pre-split at every size (1 does so from 16384 rows)
 @pytest.mark.parametrize("m,n,k", SHAPES)
 def test_dense_product_against_fp64(handle, m, n, k, tensor_cores):
     import torch

@@ -203,13 +203,15 @@ def test_ten_iterations(case, dual_mode):
         g.destroy()
 
 
-def test_ten_iterations_without_tensor_cores():
-    """The fp32 FMA kernels (tensor_cores = 0) stay a supported path: same ten-pass check on one case."""
+@pytest.mark.parametrize("tensor_cores", [0, 3])
+def test_ten_iterations_other_product_kernels(tensor_cores):
+    """The fp32 FMA kernels (tensor_cores = 0) stay a supported path, and the pre-split weight operand
+    (3; taken by default only from 16384 rows) must give the same iterates: same ten-pass check on one case."""
     wl = inputs.make_workload(3, scale=0.012)
     g, o = make_pair(wl)
     g.destroy()
     g = binding.GcnAdmm(wl.n, wl.row_ptr, wl.col_idx, wl.X, wl.y, wl.train_mask, wl.widths, wl.n_comm, wl.community,
-                        wl.w_init, nu=wl.nu, rho=wl.rho, tensor_cores=0)
+                        wl.w_init, nu=wl.nu, rho=wl.rho, tensor_cores=tensor_cores)
     try:
         g.step(10)
         dec = g.decisions()
