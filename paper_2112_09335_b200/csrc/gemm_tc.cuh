@@ -527,7 +527,7 @@ struct WsCfg {
   static constexpr int kStage = 2 * kATileBytes + 2 * kBTile;
   static constexpr int kAccCols = kSets * 2 * NT;
   static constexpr uint32_t kTmemCols = kAccCols <= 64 ? 64 : kAccCols <= 128 ? 128 : kAccCols <= 256 ? 256 : 512;
-  static constexpr size_t kSmem = (size_t)kStagesWs * kStage + 1024;
+  static constexpr size_t kSmem = (size_t)kStagesWs * kStage + 4 * 4096 + 1024;   // + the epilogue warps' buffers
 };
 
 // The weight operand split once, in the layout the MMA descriptors read: for column group g and K
@@ -606,7 +606,8 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
   if (warp < 8) {
     // ---------------- producers ----------------
     const int ld_c16 = tid & 7, ld_row = tid >> 3;
-    float4 ra[2][A_PASSES], rb[2][IMG ? 1 : B_PASSES];
+    constexpr int DEPTH = IMG ? 4 : 2;   // chunks a thread holds in registers ahead of the one it stores
+    float4 ra[DEPTH][A_PASSES], rb[DEPTH][IMG ? 1 : B_PASSES];
     auto load_chunk = [&](int j, float4* pa, float4* pb) {
       if (j >= total) return;
       const int tile = blockIdx.x + (j / kc_count) * gridDim.x, kc = j % kc_count;
@@ -659,26 +660,32 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
         }
       }
     };
-    load_chunk(0, ra[0], rb[0]);
-    load_chunk(1, ra[1], rb[1]);
-    for (int j = 0; j < total; ++j) {
-      const int stage = j % S;
-      if (j >= S && !mbar_wait_abortable(bar_empty + 8 * stage, ((j / S) - 1) & 1, abortp)) break;
-      if (IMG && tid == 0) {
-        // the stage is free (its MMAs have retired): fetch both B tiles of this chunk with one bulk copy
-        // that reports its bytes to the stage's full barrier; this thread's own arrival comes below
-        const uint32_t bytes = 2u * (uint32_t)Cfg::kBTile;
-        const uint8_t* src = b_image + ((size_t)blockIdx.y * kc_count + (size_t)(j % kc_count)) * bytes;
-        const uint32_t dst = smem_base + (uint32_t)stage * Cfg::kStage + 2u * kATileBytes;
-        asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar_full + 8 * stage), "r"(bytes) : "memory");
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     ::"r"(dst), "l"(src), "r"(bytes), "r"(bar_full + 8 * stage)
-                     : "memory");
+#pragma unroll
+    for (int d = 0; d < DEPTH; ++d) load_chunk(d, ra[d], rb[d]);
+    bool stop = false;
+    for (int j0 = 0; j0 < total && !stop; j0 += DEPTH) {
+#pragma unroll
+      for (int d = 0; d < DEPTH; ++d) {
+        const int j = j0 + d;
+        if (j >= total) break;
+        const int stage = j % S;
+        if (j >= S && !mbar_wait_abortable(bar_empty + 8 * stage, ((j / S) - 1) & 1, abortp)) { stop = true; break; }
+        if (IMG && tid == 0) {
+          // the stage is free (its MMAs have retired): fetch both B tiles of this chunk with one bulk copy
+          // that reports its bytes to the stage's full barrier; this thread's own arrival comes below
+          const uint32_t bytes = 2u * (uint32_t)Cfg::kBTile;
+          const uint8_t* src = b_image + ((size_t)blockIdx.y * kc_count + (size_t)(j % kc_count)) * bytes;
+          const uint32_t dst = smem_base + (uint32_t)stage * Cfg::kStage + 2u * kATileBytes;
+          asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar_full + 8 * stage), "r"(bytes) : "memory");
+          asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                       ::"r"(dst), "l"(src), "r"(bytes), "r"(bar_full + 8 * stage)
+                       : "memory");
+        }
+        store_chunk(stage, ra[d], rb[d]);
+        load_chunk(j + DEPTH, ra[d], rb[d]);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(bar_full + 8 * stage);
       }
-      if (j & 1) { store_chunk(stage, ra[1], rb[1]); load_chunk(j + 2, ra[1], rb[1]); }
-      else       { store_chunk(stage, ra[0], rb[0]); load_chunk(j + 2, ra[0], rb[0]); }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      mbar_arrive(bar_full + 8 * stage);
     }
   } else if (warp == 12) {
     // ---------------- MMA issue ----------------
@@ -706,31 +713,49 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
     }
   } else {
     // ---------------- epilogue ----------------
+    // In tensor memory a lane holds one row, so a direct store would have the 32 lanes of a warp write
+    // 16 bytes each to 32 different rows.  The sums of CW columns go through a per-warp buffer in shared
+    // memory instead (128-byte rows, 16-byte slots XORed with the row index) and leave as whole lines:
+    // 32 / (CW/4) rows of CW contiguous floats per store instruction.
     const int quarter = warp & 3;
+    constexpr int CW = (NT % 32 == 0) ? 32 : 16;      // columns per step
+    constexpr int SLOTS = CW / 4;                      // float4 per row and step
+    constexpr int ROWS_PER_STORE = 32 / SLOTS;
+    uint8_t* tbuf = smem + (size_t)S * Cfg::kStage + (size_t)quarter * 4096;
     for (int tile_i = 0; tile_i < my_tiles; ++tile_i) {
       const int set = tile_i % SETS;
       if (!mbar_wait_abortable(bar_acc_full + 8 * set, (tile_i / SETS) & 1, abortp)) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const long long row = (long long)(blockIdx.x + tile_i * gridDim.x) * kBlockM + quarter * 32 + lane;
+      const long long row0 = (long long)(blockIdx.x + tile_i * gridDim.x) * kBlockM + quarter * 32;
 #pragma unroll 1
-      for (int cchunk = 0; cchunk < NT / 16; ++cchunk) {
-        uint32_t v[16], w[16];
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(set * 2 * NT + cchunk * 16);
-        GTC_TMEM_LD16(v, taddr);
-        GTC_TMEM_LD16(w, taddr + (uint32_t)NT);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (row < M) {
+      for (int cstep = 0; cstep < NT / CW; ++cstep) {
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(set * 2 * NT + cstep * CW);
+#pragma unroll
+        for (int half = 0; half < CW / 16; ++half) {
+          uint32_t v[16], w[16];
+          GTC_TMEM_LD16(v, taddr + (uint32_t)(half * 16));
+          GTC_TMEM_LD16(w, taddr + (uint32_t)(NT + half * 16));
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
-            const int col = n0 + cchunk * 16 + q * 4;
-            if (col < ldc)
-              *reinterpret_cast<float4*>(C + row * ldc + col) =
-                  make_float4(__uint_as_float(v[q * 4]) + __uint_as_float(w[q * 4]),
-                              __uint_as_float(v[q * 4 + 1]) + __uint_as_float(w[q * 4 + 1]),
-                              __uint_as_float(v[q * 4 + 2]) + __uint_as_float(w[q * 4 + 2]),
-                              __uint_as_float(v[q * 4 + 3]) + __uint_as_float(w[q * 4 + 3]));
+            const int slot = (half * 4 + q) ^ (lane & (SLOTS - 1));
+            *reinterpret_cast<float4*>(tbuf + lane * 128 + slot * 16) =
+                make_float4(__uint_as_float(v[q * 4]) + __uint_as_float(w[q * 4]),
+                            __uint_as_float(v[q * 4 + 1]) + __uint_as_float(w[q * 4 + 1]),
+                            __uint_as_float(v[q * 4 + 2]) + __uint_as_float(w[q * 4 + 2]),
+                            __uint_as_float(v[q * 4 + 3]) + __uint_as_float(w[q * 4 + 3]));
           }
         }
+        __syncwarp();
+        const int c4 = lane & (SLOTS - 1);
+        const int col = n0 + cstep * CW + c4 * 4;
+#pragma unroll
+        for (int i = 0; i < SLOTS; ++i) {
+          const int r = i * ROWS_PER_STORE + lane / SLOTS;
+          const float4 val = *reinterpret_cast<const float4*>(tbuf + r * 128 + ((c4 ^ (r & (SLOTS - 1))) * 16));
+          if (row0 + r < M && col < ldc) *reinterpret_cast<float4*>(C + (row0 + r) * ldc + col) = val;
+        }
+        __syncwarp();
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       mbar_arrive(bar_acc_empty + 8 * set);
