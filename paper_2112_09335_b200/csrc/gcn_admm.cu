@@ -140,6 +140,7 @@ struct gcn_admm {
   float* item_sums = nullptr;             // n_items x max_ld
   size_t item_sums_elems = 0;
   unsigned char* d_train = nullptr;
+  int* d_train_rows = nullptr;            // new ids of the training rows, ascending
 
   std::vector<float*> W, Wt, Z, P, H;   // 1..L
   float* U = nullptr;
@@ -218,7 +219,7 @@ struct gcn_admm {
     else if (ld4 <= 8) SPMM_CASE(8, 1, 8)
     else if (ld4 <= 16) SPMM_CASE(16, 1, 8)
     else if (ld4 <= 32) SPMM_CASE(32, 1, 4)
-    else SPMM_CASE(32, 2, 4)
+    else SPMM_CASE(32, 2, 2)   // two neighbours in flight per lane beat four (fewer registers, more warps): measured
 #undef SPMM_CASE
     CU(cudaGetLastError());
     if (cut) {
@@ -502,15 +503,15 @@ struct gcn_admm {
     const size_t smem = (size_t)warps * M * per * sizeof(double);
     const int use_smem = smem <= 96 * 1024;
     const size_t dyn = use_smem ? smem : 0;
-#define SCORE_Z(V, OUT)                                                                                   \
+#define SCORE_Z_U(V, OUT, UNZ)                                                                                 \
   {                                                                                                       \
     if (dyn > 48 * 1024)                                                                                  \
-      CU(cudaFuncSetAttribute(gk::k_score_z<V, OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn)); \
+      CU(cudaFuncSetAttribute(gk::k_score_z<V, OUT, UNZ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn)); \
     CU(cudaMemsetAsync(row_counter, 0, sizeof(int), stream));                                             \
     int occ = 1;                                                                                          \
-    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gk::k_score_z<V, OUT>, warps * 32, dyn));      \
+    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gk::k_score_z<V, OUT, UNZ>, warps * 32, dyn));      \
     const unsigned grid = (unsigned)std::min<long long>(cdiv(n + n_items, warps), (long long)kSmCount * std::max(occ, 1)); \
-    gk::k_score_z<V, OUT><<<grid, warps * 32, dyn, stream>>>(d_row_ptr, d_col, d_col_comm, d_dinv,        \
+    gk::k_score_z<V, OUT, UNZ><<<grid, warps * 32, dyn, stream>>>(d_row_ptr, d_col, d_col_comm, d_dinv,        \
         (const float4*)B1, (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0, ld4, (int)n, ctl, M, \
         acc_z, n_active, use_smem, row_counter, d_items, n_items, long_len, reinterpret_cast<float4*>(item_sums)); \
     if (n_split > 0) {                                                                                    \
@@ -519,6 +520,11 @@ struct gcn_admm {
           ld4, ctl, acc_z, n_active);                                                                     \
       ++launches;                                                                                         \
     }                                                                                                     \
+  }
+#define SCORE_Z(V, OUT)                                     \
+  {                                                         \
+    if (OUT) SCORE_Z_U(V, OUT, 4)                           \
+    else SCORE_Z_U(V, OUT, 2)                               \
   }
 #define SCORE_Z_ANY(OUT)                    \
   {                                         \
@@ -560,6 +566,7 @@ struct gcn_admm {
     }
 #undef SCORE_Z_ANY
 #undef SCORE_Z
+#undef SCORE_Z_U
     CU(cudaGetLastError());
     {
       Scope sc(this, "small", 1, 0.0, 0.0);
@@ -575,10 +582,18 @@ struct gcn_admm {
   void update_output(bool dual_now, bool update_z) {
     const int warps = 8;
     Scope sc(this, "output_rows", 1, 4.0 * (double)n * ld[L] * (3 + (update_z ? 1 : 0) + (dual_now ? 1 : 0)), 0.0);
-    gk::k_output_rows<<<(unsigned)cdiv(n, warps), warps * 32, 0, stream>>>(Z[L], U, H[L], ld[L], C[L], (int)n, d_y, d_train,
-                                                                           p.rho, p.loss_scale, p.fista_iters,
-                                                                           dual_now ? 1 : 0, update_z ? 1 : 0);
+    // rows without a loss term: closed form, plain sweep; training rows: one warp each (FISTA)
+    gk::k_output_plain<<<grid_for(n * (ld[L] / 4)), 256, 0, stream>>>((float4*)Z[L], (float4*)U, (const float4*)H[L],
+                                                                      ld[L] / 4, n, d_train, p.rho, dual_now ? 1 : 0,
+                                                                      update_z ? 1 : 0);
     CU(cudaGetLastError());
+    if (n_train > 0) {
+      gk::k_output_rows<<<(unsigned)cdiv(n_train, warps), warps * 32, 0, stream>>>(
+          Z[L], U, H[L], ld[L], C[L], n_train, d_y, d_train, p.rho, p.loss_scale, p.fista_iters, dual_now ? 1 : 0,
+          update_z ? 1 : 0, d_train_rows);
+      CU(cudaGetLastError());
+      ++launches;
+    }
   }
 
   void dual_from_stored() {   // U + rho (Z_L - H_L) with H_L = A~ Z_{L-1} W_L of the stored iterates
@@ -796,6 +811,13 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
   }
   h->d_y = upload(h, y_new);
   h->d_train = upload(h, t_new);
+  {
+    std::vector<int> tr;
+    tr.reserve((size_t)h->n_train);
+    for (long long i = 0; i < n; ++i)
+      if (t_new[i]) tr.push_back((int)i);
+    h->d_train_rows = upload(h, tr);
+  }
   {
     h->long_len = p.long_row > 0 ? p.long_row : kDefaultLongRow;
     gcn_admm_host::LongRowTables lt;

@@ -970,7 +970,7 @@ __device__ __forceinline__ void score_segment(const float4 (&k)[V], float di, co
   }
 }
 
-template <int V, bool OUT>
+template <int V, bool OUT, int UN>
 __global__ void __launch_bounds__(256)
 k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
           const unsigned short* __restrict__ col_comm, const float* __restrict__ dinv,
@@ -1052,19 +1052,19 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
         else w = dinv[c];
       }
       const int cnt = min(32, re - base);
-      for (int t = 0; t < cnt; t += 4) {
-        int cj[4], mj[4];
-        float wj[4];
+      for (int t = 0; t < cnt; t += UN) {
+        int cj[UN], mj[UN];
+        float wj[UN];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < UN; ++u) {
           cj[u] = __shfl_sync(0xffffffffu, c, (t + u) & 31);
           mj[u] = __shfl_sync(0xffffffffu, m, (t + u) & 31);
           wj[u] = __shfl_sync(0xffffffffu, w, (t + u) & 31);
           if (t + u >= cnt) mj[u] = -1;
         }
-        float4 xv[4][V];
+        float4 xv[UN][V];
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
+        for (int u = 0; u < UN; ++u)
 #pragma unroll
           for (int v = 0; v < V; ++v) {
             const int f = lane + 32 * v;
@@ -1072,7 +1072,7 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
             if (mj[u] >= 0 && mj[u] < 0x10000 && f < ld4) xv[u][v] = __ldg(T + (long long)cj[u] * ld4 + f);
           }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < UN; ++u) {
           if (mj[u] < 0) continue;                       // past the end of the row (warp-uniform)
           const int mm = mj[u] & 0xffff;
           if (mm != cur) {
@@ -1134,6 +1134,29 @@ k_score_z_split(const int4* __restrict__ split, int n_split, const float* __rest
   score_segment<V, OUT>(k, dinv[sp.x], a, b, ctl, sp.y, lane, acc, false);
 }
 
+// The rows of Eq. 7 without a loss term (not in the training set) have the closed form
+// z = q - u / rho; with dual_now, U <- u + rho (z_old - q) first (Eq. 3 as printed).  Plain
+// elementwise sweep; training rows are skipped (k_output_rows visits them).
+__global__ void k_output_plain(float4* __restrict__ ZL, float4* __restrict__ U, const float4* __restrict__ HL, int ld4,
+                               long long n, const unsigned char* __restrict__ train, float rho, int dual_now,
+                               int update_z) {
+  const long long total = n * ld4;
+  const float inv_rho = 1.f / rho;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total;
+       e += (long long)gridDim.x * blockDim.x) {
+    if (train[e / ld4]) continue;
+    const float4 q = HL[e], u = U[e];
+    if (dual_now) {
+      const float4 z = ZL[e];
+      U[e] = make_float4(fmaf(rho, z.x - q.x, u.x), fmaf(rho, z.y - q.y, u.y), fmaf(rho, z.z - q.z, u.z),
+                         fmaf(rho, z.w - q.w, u.w));
+    }
+    if (update_z)
+      ZL[e] = make_float4(fmaf(-u.x, inv_rho, q.x), fmaf(-u.y, inv_rho, q.y), fmaf(-u.z, inv_rho, q.z),
+                          fmaf(-u.w, inv_rho, q.w));
+  }
+}
+
 // Z_l[i,:] <- Z_l[i,:] - G[i,:] / theta_{comm(i)}   (Eq. 10)
 __global__ void k_apply_z(float4* __restrict__ Z, const float4* __restrict__ G, int ld4, long long n,
                           const int* __restrict__ row_comm, const SearchCtl* __restrict__ ctl) {
@@ -1154,14 +1177,17 @@ __global__ void k_apply_z(float4* __restrict__ Z, const float4* __restrict__ G, 
 //   q = row of A~ Z_{L-1}^k W_L^{k+1};  training rows: FISTA on
 //   loss_scale * CE(z, y) + <u, z - q> + (rho/2)||z - q||^2 ;  other rows: z = q - u / rho.
 //   dual_now != 0: U <- u + rho (z_old - q) in the same sweep (Eq. 3 as printed).
+// `rows` (may be NULL = every row) lists the rows to visit: the training rows, when the rest is
+// left to k_output_plain.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 k_output_rows(float* __restrict__ ZL, float* __restrict__ U, const float* __restrict__ HL, int ld, int C,
               int n, const int* __restrict__ y, const unsigned char* __restrict__ train, float rho,
-              float loss_scale, int iters, int dual_now, int update_z) {
+              float loss_scale, int iters, int dual_now, int update_z, const int* __restrict__ rows) {
   const int lane = threadIdx.x & 31;
-  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (row >= n) return;
+  const int slot = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (slot >= n) return;
+  const int row = rows != nullptr ? rows[slot] : slot;
   float q[kMaxClassesPerLane], u[kMaxClassesPerLane], z[kMaxClassesPerLane];
   const long long base = (long long)row * ld;
 #pragma unroll
