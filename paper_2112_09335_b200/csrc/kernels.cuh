@@ -30,10 +30,12 @@ struct SearchCtl {
 __device__ __forceinline__ float relu(float x) { return x > 0.f ? x : 0.f; }
 
 // relu(h) - relu(h - s) without forming h - s when both sides are active, so that a step s far
-// below the rounding unit of h still registers exactly.
-__device__ __forceinline__ float relu_drop(float h, float s) {
-  const bool on0 = h > 0.f, on1 = h > s;
-  return on0 ? (on1 ? s : h) : (on1 ? s - h : 0.f);
+// below the rounding unit of h still registers exactly.  With pos = max(h, 0) and neg = max(-h, 0)
+// (one of them is zero) the drop is min(s + neg, pos): for h > 0 that is min(s, h), for h <= 0 it
+// is min(s - h, 0).  The caller forms pos and neg once per element and passes s = k * inv as the
+// two factors, so a candidate costs one fused multiply-add and one minimum.
+__device__ __forceinline__ float relu_drop(float k, float inv, float neg, float pos) {
+  return fminf(fmaf(k, inv, neg), pos);
 }
 
 __device__ __forceinline__ double warp_sum(double v) {
@@ -649,11 +651,12 @@ k_score_w_hidden(const float4* __restrict__ H, const float4* __restrict__ D, con
     for (int j = 0; j < kCand; ++j) part[j] = 0.f;
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
-      const float e0 = z[c] - relu(h[c]);
+      const float pos = fmaxf(h[c], 0.f), neg = fmaxf(-h[c], 0.f);
+      const float e2 = 2.f * (z[c] - pos);
 #pragma unroll
       for (int j = 0; j < kCand; ++j) {
-        const float df = relu_drop(h[c], d[c] * inv[j]);
-        part[j] = fmaf(df, fmaf(2.f, e0, df), part[j]);   // e1^2 - e0^2 = (e1 - e0)(e1 + e0), e1 - e0 = df
+        const float df = relu_drop(d[c], inv[j], neg, pos);
+        part[j] = fmaf(df, e2 + df, part[j]);   // e1^2 - e0^2 = (e1 - e0)(e1 + e0), e1 - e0 = df
       }
     }
 #pragma unroll
@@ -945,19 +948,20 @@ __device__ __forceinline__ void score_segment(const float4 (&k)[V], float di, co
   } else {
     float inv[kCand], part[kCand];
 #pragma unroll
-    for (int j = 0; j < kCand; ++j) { inv[j] = ctl[cur].inv_cand[j]; part[j] = 0.f; }
+    for (int j = 0; j < kCand; ++j) { inv[j] = di * ctl[cur].inv_cand[j]; part[j] = 0.f; }   // K_m[i] = di * k
 #pragma unroll
     for (int v = 0; v < V; ++v) {
-      const float kk[4] = {di * k[v].x, di * k[v].y, di * k[v].z, di * k[v].w};
+      const float kk[4] = {k[v].x, k[v].y, k[v].z, k[v].w};
       const float hh[4] = {a[v].x, a[v].y, a[v].z, a[v].w};
       const float zz[4] = {b[v].x, b[v].y, b[v].z, b[v].w};
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
-        const float e0 = zz[c] - relu(hh[c]);
+        const float pos = fmaxf(hh[c], 0.f), neg = fmaxf(-hh[c], 0.f);
+        const float e2 = 2.f * (zz[c] - pos);
 #pragma unroll
         for (int j = 0; j < kCand; ++j) {
-          const float df = relu_drop(hh[c], kk[c] * inv[j]);
-          part[j] = fmaf(df, fmaf(2.f, e0, df), part[j]);
+          const float df = relu_drop(kk[c], inv[j], neg, pos);
+          part[j] = fmaf(df, e2 + df, part[j]);
         }
       }
     }
@@ -971,7 +975,7 @@ __device__ __forceinline__ void score_segment(const float4 (&k)[V], float di, co
 }
 
 template <int V, bool OUT, int UN>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, (V <= 2 ? 3 : 1))
 k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
           const unsigned short* __restrict__ col_comm, const float* __restrict__ dinv,
           const float4* __restrict__ T, const float4* __restrict__ Hn, const float4* __restrict__ Zn,
