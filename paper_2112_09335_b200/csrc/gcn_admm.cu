@@ -325,14 +325,20 @@ struct gcn_admm {
   }
 
   // out[Ka x ldp] = A^T B over `rows` rows, through split partial sums reduced in a fixed order.
+  // Whether P^T R runs on the tensor cores (that form can also build a hidden layer's R itself).
+  bool tn_on_tensor_cores(long long rows) const { return (p.tensor_cores == 1 || p.tensor_cores == 3) && rows >= 4096; }
+
+  // With `zres` (tensor-core form only) B holds pre-activations H and the operand is
+  // h > 0 ? nu (h - z) : 0, formed while staging: the residual matrix is never stored.
   void gemm_tn(const float* A, int lda, const float* B, int ldb, float* out, int ldp, long long rows, int Ka,
-               int Nb) {
+               int Nb, const float* zres = nullptr, float nu = 0.f) {
     int splits = 1;
     long long rps = rows;
     char name[48];
-    if ((p.tensor_cores == 1 || p.tensor_cores == 3) && rows >= 4096) {
-      std::snprintf(name, sizeof name, "gemm_tn_tc@%dx%d", Ka, Nb);
-      Scope sc(this, name, 2, 4.0 * ((double)rows * (lda + ldb) + (double)Ka * ldp), 2.0 * (double)rows * Ka * Nb);
+    if (zres && !tn_on_tensor_cores(rows)) throw Fail{GCN_ADMM_ERR_ARG, "fused residual needs the tensor-core product"};
+    if (tn_on_tensor_cores(rows)) {
+      std::snprintf(name, sizeof name, zres ? "gemm_tn_tc.resid@%dx%d" : "gemm_tn_tc@%dx%d", Ka, Nb);
+      Scope sc(this, name, 2, 4.0 * ((double)rows * (lda + (zres ? 2 : 1) * ldb) + (double)Ka * ldp), 2.0 * (double)rows * Ka * Nb);
       const int nt_tn = Nb <= 16 ? 16 : Nb <= 32 ? 32 : Nb <= 48 ? 48 : Nb <= 64 ? 64 : Nb <= 128 ? 128 : 256;
       const int nb_groups = (int)cdiv(Nb, nt_tn);
       const int groups = (int)cdiv(Ka, gtc::kBlockM);
@@ -346,9 +352,14 @@ struct gcn_admm {
 #define TN_TC(NT)                                                                                              \
   {                                                                                                            \
     const size_t smem = gtc::TnCfg<NT>::kSmem;                                                                 \
-    CU(cudaFuncSetAttribute(gtc::k_gemm_tn_tc<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));   \
     dim3 grid((unsigned)splits, (unsigned)groups, (unsigned)nb_groups);                                        \
-    gtc::k_gemm_tn_tc<NT><<<grid, gtc::kTnThreads, smem, stream>>>(A, lda, B, ldb, part, ldp, rows, rps, Ka, Nb, tc_error); \
+    if (zres) {                                                                                                \
+      CU(cudaFuncSetAttribute(gtc::k_gemm_tn_tc<NT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+      gtc::k_gemm_tn_tc<NT, true><<<grid, gtc::kTnThreads, smem, stream>>>(A, lda, B, ldb, part, ldp, rows, rps, Ka, Nb, tc_error, zres, nu); \
+    } else {                                                                                                   \
+      CU(cudaFuncSetAttribute(gtc::k_gemm_tn_tc<NT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+      gtc::k_gemm_tn_tc<NT, false><<<grid, gtc::kTnThreads, smem, stream>>>(A, lda, B, ldb, part, ldp, rows, rps, Ka, Nb, tc_error, nullptr, 0.f); \
+    }                                                                                                          \
   }
       if (Nb <= 16) TN_TC(16)
       else if (Nb <= 32) TN_TC(32)
@@ -420,8 +431,12 @@ struct gcn_admm {
     const int Kp = C[l - 1], Cn = C[l], ldc = ld[l];
     const long long n4 = n * ldc / 4;
     SearchCtl* ctl = ctl_w + l;
-    resid(l, B0);                                                       // R_l
-    gemm_tn(P[l], ld[l - 1], B0, ldc, grad, ldc, n, Kp, Cn);            // grad = P_l^T R_l
+    if (l < L && tn_on_tensor_cores(n)) {                               // grad = P_l^T R_l, R_l formed inside the product
+      gemm_tn(P[l], ld[l - 1], H[l], ldc, grad, ldc, n, Kp, Cn, Z[l], p.nu);
+    } else {
+      resid(l, B0);                                                     // R_l
+      gemm_tn(P[l], ld[l - 1], B0, ldc, grad, ldc, n, Kp, Cn);          // grad = P_l^T R_l
+    }
     {
       Scope sc(this, "small", 3, 0.0, 0.0);
       gk::k_transpose_small<<<(unsigned)cdiv((long long)Kp * Cn, 256), 256, 0, stream>>>(grad, ldc, grad_t, ld[l - 1], Kp, Cn);

@@ -812,10 +812,15 @@ struct TnCfg {
   static constexpr size_t kSmem = (size_t)kStagesTn * kStage + 1024;
 };
 
-template <int NT>
+// RESID: B is not stored.  The operand is the derivative of a hidden layer's penalty with respect to
+// its pre-activation, formed while staging from the pre-activation H (passed as B) and the layer's
+// Z (Zres, same leading dimension):  b = h > 0 ? nu (h - z) : 0.  Both rows are fetched one chunk
+// ahead (A stays two chunks ahead), so the second matrix costs no further registers.
+template <int NT, bool RESID>
 __global__ void __launch_bounds__(kTnThreads, 1)
 k_gemm_tn_tc(const float* __restrict__ A, int lda, const float* __restrict__ B, int ldb, float* __restrict__ part, int ldp,
-             long long rows, long long rows_per_split, int Ka, int Nb, int* __restrict__ error_flag) {
+             long long rows, long long rows_per_split, int Ka, int Nb, int* __restrict__ error_flag,
+             const float* __restrict__ Zres, float nu) {
   using Cfg = TnCfg<NT>;
   constexpr int S = Cfg::kStagesTn;
   constexpr int A_PASSES = 4;                              // 1024 float4 / 256 threads
@@ -859,7 +864,7 @@ k_gemm_tn_tc(const float* __restrict__ A, int lda, const float* __restrict__ B, 
   if (warp < 8) {
     // ---------------- producers ----------------
     float4 ra[2][A_PASSES], rb[2][B_PASSES];
-    auto load_chunk = [&](int j, float4* pa, float4* pb) {
+    auto load_a = [&](int j, float4* pa) {
       if (j >= total) return;
       const long long r0 = r_begin + (long long)j * kTnRows;
 #pragma unroll
@@ -871,17 +876,21 @@ k_gemm_tn_tc(const float* __restrict__ A, int lda, const float* __restrict__ B, 
         if (r < r_end && col < Ka) v = *reinterpret_cast<const float4*>(A + r * lda + col);   // zero padding beyond Ka
         pa[i] = v;
       }
+    };
+    auto load_b = [&](int j, const float* __restrict__ src, float4* pb) {
+      if (j >= total) return;
+      const long long r0 = r_begin + (long long)j * kTnRows;
 #pragma unroll
       for (int i = 0; i < B_PASSES; ++i) {
         const int f = tid + 256 * i;
         const int rr = f / (NT / 4), c4 = f % (NT / 4);
         const long long r = r0 + rr;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (f < B_F4 && r < r_end && nb0 + 4 * c4 < Nb) v = *reinterpret_cast<const float4*>(B + r * ldb + nb0 + 4 * c4);
+        if (f < B_F4 && r < r_end && nb0 + 4 * c4 < Nb) v = *reinterpret_cast<const float4*>(src + r * ldb + nb0 + 4 * c4);
         pb[i] = v;
       }
     };
-    auto store_chunk = [&](int stage, const float4* pa, const float4* pb) {
+    auto store_chunk = [&](int stage, const float4* pa, const float4* pb, const float4* pz) {
       uint8_t* st = smem + (size_t)stage * Cfg::kStage;
 #pragma unroll
       for (int i = 0; i < A_PASSES; ++i) {
@@ -898,22 +907,44 @@ k_gemm_tn_tc(const float* __restrict__ A, int lda, const float* __restrict__ B, 
         const int f = tid + 256 * i;
         if (f < B_F4) {
           const int rr = f / (NT / 4), c4 = f % (NT / 4);
+          float4 b = pb[i];
+          if (RESID) {
+            const float4 z = pz[i];
+            b.x = b.x > 0.f ? nu * (b.x - z.x) : 0.f;
+            b.y = b.y > 0.f ? nu * (b.y - z.y) : 0.f;
+            b.z = b.z > 0.f ? nu * (b.z - z.z) : 0.f;
+            b.w = b.w > 0.f ? nu * (b.w - z.w) : 0.f;
+          }
           float4 h, l;
-          split_tf32(pb[i].x, h.x, l.x); split_tf32(pb[i].y, h.y, l.y);
-          split_tf32(pb[i].z, h.z, l.z); split_tf32(pb[i].w, h.w, l.w);
+          split_tf32(b.x, h.x, l.x); split_tf32(b.y, h.y, l.y);
+          split_tf32(b.z, h.z, l.z); split_tf32(b.w, h.w, l.w);
           const uint32_t off = swz_mn(rr, c4);
           *reinterpret_cast<float4*>(st + 2 * Cfg::kATile + off) = h;
           *reinterpret_cast<float4*>(st + 2 * Cfg::kATile + Cfg::kBTile + off) = l;
         }
       }
     };
-    load_chunk(0, ra[0], rb[0]);
-    load_chunk(1, ra[1], rb[1]);
+    load_a(0, ra[0]);
+    load_a(1, ra[1]);
+    if (RESID) {   // rb[0] = rows of H, rb[1] = rows of Z, both of the next chunk
+      load_b(0, B, rb[0]);
+      load_b(0, Zres, rb[1]);
+    } else {
+      load_b(0, B, rb[0]);
+      load_b(1, B, rb[1]);
+    }
     for (int j = 0; j < total; ++j) {
       const int stage = j % S;
       if (j >= S && !mbar_wait_abortable(bar_empty + 8 * stage, ((j / S) - 1) & 1, abortp)) break;
-      if (j & 1) { store_chunk(stage, ra[1], rb[1]); load_chunk(j + 2, ra[1], rb[1]); }
-      else       { store_chunk(stage, ra[0], rb[0]); load_chunk(j + 2, ra[0], rb[0]); }
+      if (RESID) {
+        if (j & 1) { store_chunk(stage, ra[1], rb[0], rb[1]); load_a(j + 2, ra[1]); }
+        else       { store_chunk(stage, ra[0], rb[0], rb[1]); load_a(j + 2, ra[0]); }
+        load_b(j + 1, B, rb[0]);
+        load_b(j + 1, Zres, rb[1]);
+      } else {
+        if (j & 1) { store_chunk(stage, ra[1], rb[1], nullptr); load_a(j + 2, ra[1]); load_b(j + 2, B, rb[1]); }
+        else       { store_chunk(stage, ra[0], rb[0], nullptr); load_a(j + 2, ra[0]); load_b(j + 2, B, rb[0]); }
+      }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       mbar_arrive(bar_full + 8 * stage);
     }
