@@ -158,6 +158,23 @@ def test_single_block_updates_from_identical_state(case):
     print("\n" + "\n".join(f"  {n}: rel {a:.2e}  step-rel {b:.2e}" for n, a, b in report))
 
 
+@pytest.mark.parametrize("tensor_cores", [1, 3])
+def test_single_block_updates_at_tensor_core_sizes(tensor_cores):
+    """The cases above have fewer than 4096 rows, where the weight gradient P^T R runs on the fp32 FMA
+    kernel.  With 8,467 rows every dense product of a block update, the transposed one with the
+    residual operand formed inside it included, runs on the tensor cores (3: weights pre-split):
+    same single-block check, every W block and every hidden Z block of every community."""
+    wl = inputs.make_workload(3, scale=0.05)
+    assert wl.n >= 4096
+    g = binding.GcnAdmm(wl.n, wl.row_ptr, wl.col_idx, wl.X, wl.y, wl.train_mask, wl.widths, wl.n_comm, wl.community,
+                        wl.w_init, nu=wl.nu, rho=wl.rho, tensor_cores=tensor_cores)
+    o = make_oracle(wl)
+    try:
+        test_single_block_updates_from_identical_state((wl, g, o))
+    finally:
+        g.destroy()
+
+
 @pytest.mark.parametrize("dual_mode", [0, 1])
 def test_ten_iterations(case, dual_mode):
     wl, g0, o0 = case
