@@ -345,6 +345,10 @@ struct gcn_admm {
       // at most 2048 rows (256 MMAs) per accumulator: the tensor core rounds the running sum toward zero at
       // every MMA, so long sums are cut into splits whose partial results are added in fp64
       splits = (int)std::max<long long>(std::max(1, kSmCount / (groups * nb_groups)), cdiv(rows, 2048));
+      {   // whole waves: with more CTAs than SMs (one CTA per SM), round the count up to a multiple of the SM count
+        const long long per = (long long)groups * nb_groups;
+        if (splits * per > kSmCount) splits = (int)(cdiv(splits * per, kSmCount) * kSmCount / per);
+      }
       splits = (int)std::min<long long>(splits, cdiv(rows, 256));
       splits = (int)std::min<long long>(splits, (long long)(part_elems / ((size_t)Ka * ldp)));
       rps = cdiv(rows, splits);
@@ -352,7 +356,7 @@ struct gcn_admm {
 #define TN_TC(NT)                                                                                              \
   {                                                                                                            \
     const size_t smem = gtc::TnCfg<NT>::kSmem;                                                                 \
-    dim3 grid((unsigned)splits, (unsigned)groups, (unsigned)nb_groups);                                        \
+    dim3 grid((unsigned)groups, (unsigned)splits, (unsigned)nb_groups);                                        \
     if (zres) {                                                                                                \
       CU(cudaFuncSetAttribute(gtc::k_gemm_tn_tc<NT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
       gtc::k_gemm_tn_tc<NT, true><<<grid, gtc::kTnThreads, smem, stream>>>(A, lda, B, ldb, part, ldp, rows, rps, Ka, Nb, tc_error, zres, nu); \
@@ -864,7 +868,7 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
     h->part_elems = std::max(h->part_elems, ge * 4 * kSmCount);
   }
   for (int l = 1; l <= L; ++l)   // room for one split per 2048 rows (tensor-core form of the transposed product)
-    h->part_elems = std::max(h->part_elems, (size_t)h->C[l - 1] * h->ld[l] * (size_t)cdiv(n, 2048));
+    h->part_elems = std::max(h->part_elems, (size_t)h->C[l - 1] * h->ld[l] * (size_t)(cdiv(n, 2048) + kSmCount));
   h->part_elems = std::min<size_t>(h->part_elems, (size_t)256 << 20);   // at most 1 GB of partial sums
   h->part_elems = std::max(h->part_elems, grad_elems);
   h->U = h->alloc<float>(rows * h->ld[L]);

@@ -780,8 +780,10 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
 // unit u of row r sits at unit u ^ (r mod 4); successive column groups are 4096 bytes apart (the
 // descriptor's leading byte offset), successive groups of 4 rows 512 bytes apart (its stride byte
 // offset).  One MMA consumes 8 rows (K = 8), i.e. two atoms.  Same hi/lo split, same separate correction accumulator, same roles as
-// above (8 producer warps, one MMA warp); a CTA owns 128 columns of A (blockIdx.y), NT columns of B
-// (blockIdx.z) and one row split (blockIdx.x) and writes its 128 x NT partial sum once, at the end.
+// above (8 producer warps, one MMA warp); a CTA owns 128 columns of A (blockIdx.x), NT columns of B
+// (blockIdx.z) and one row split (blockIdx.y) and writes its 128 x NT partial sum once, at the end.
+// The column groups of A are the fastest grid index: the CTAs that read the same rows of B start
+// together, and the second one finds them in L2.
 // ------------------------------------------------------------------------------------------------
 constexpr int kTnThreads = 9 * 32;
 constexpr int kTnRows = 32;                       // rows (reduction steps) per chunk
@@ -855,10 +857,10 @@ k_gemm_tn_tc(const float* __restrict__ A, int lda, const float* __restrict__ B, 
   const uint32_t tmem_base = tmem_base_slot;
   volatile int* abortp = &abort_flag;
 
-  const long long r_begin = (long long)blockIdx.x * rows_per_split;
+  const long long r_begin = (long long)blockIdx.y * rows_per_split;
   const long long r_end = min(rows, r_begin + rows_per_split);
   const int total = r_end > r_begin ? (int)((r_end - r_begin + kTnRows - 1) / kTnRows) : 0;
-  const int ka0 = blockIdx.y * kBlockM;
+  const int ka0 = blockIdx.x * kBlockM;
   const int nb0 = blockIdx.z * NT;                 // first column of B (and of the partial sum) of this CTA
 
   if (warp < 8) {
@@ -976,7 +978,7 @@ k_gemm_tn_tc(const float* __restrict__ A, int lda, const float* __restrict__ B, 
     if (total > 0) ok = mbar_wait_abortable(bar_acc, 0, abortp);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const int ka = ka0 + warp * 32 + lane;
-    float* dst = part + ((long long)blockIdx.x * Ka + ka) * ldp;
+    float* dst = part + ((long long)blockIdx.y * Ka + ka) * ldp;
 #pragma unroll 1
     for (int cchunk = 0; cchunk < NT / 16; ++cchunk) {
       uint32_t v[16], w[16];
