@@ -524,13 +524,14 @@ struct gcn_admm {
     const size_t dyn = use_smem ? smem : 0;
 #define SCORE_Z_U(V, OUT, UNZ)                                                                                 \
   {                                                                                                       \
-    if (dyn > 48 * 1024)                                                                                  \
-      CU(cudaFuncSetAttribute(gk::k_score_z<V, OUT, UNZ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn)); \
+    const size_t dynv = dyn + (size_t)warps * 2 * (V) * 32 * sizeof(float4);   /* per-warp copy of the row's a, b */ \
+    if (dynv > 48 * 1024)                                                                                 \
+      CU(cudaFuncSetAttribute(gk::k_score_z<V, OUT, UNZ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dynv)); \
     CU(cudaMemsetAsync(row_counter, 0, sizeof(int), stream));                                             \
     int occ = 1;                                                                                          \
-    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gk::k_score_z<V, OUT, UNZ>, warps * 32, dyn));      \
+    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gk::k_score_z<V, OUT, UNZ>, warps * 32, dynv));     \
     const unsigned grid = (unsigned)std::min<long long>(cdiv(n + n_items, warps), (long long)kSmCount * std::max(occ, 1)); \
-    gk::k_score_z<V, OUT, UNZ><<<grid, warps * 32, dyn, stream>>>(d_row_ptr, d_col, d_col_comm, d_dinv,        \
+    gk::k_score_z<V, OUT, UNZ><<<grid, warps * 32, dynv, stream>>>(d_row_ptr, d_col, d_col_comm, d_dinv,       \
         (const float4*)B1, (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0, ld4, (int)n, ctl, M, \
         acc_z, n_active, use_smem, row_counter, d_items, n_items, long_len, reinterpret_cast<float4*>(item_sums)); \
     if (n_split > 0) {                                                                                    \
@@ -543,7 +544,7 @@ struct gcn_admm {
 #define SCORE_Z(V, OUT)                                     \
   {                                                         \
     if (OUT) SCORE_Z_U(V, OUT, 4)                           \
-    else SCORE_Z_U(V, OUT, 2)                               \
+    else SCORE_Z_U(V, OUT, 4)                               \
   }
 #define SCORE_Z_ANY(OUT)                    \
   {                                         \

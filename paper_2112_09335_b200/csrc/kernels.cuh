@@ -927,7 +927,13 @@ __device__ __forceinline__ float warp_sum2(float v0, float v1, int lane) {
 // item that is one piece of a segment too long for one warp only leaves its part of K_m[i],
 // unscaled, in `scratch` (one padded row per item), and k_score_z_split scores the sum of the pieces.
 
-// Scores one finished K_m[i] (k, still without the factor di) against the row's a, b.
+// 2 (z - f(h)): twice the row's current error, formed once per row and reused by every segment.
+__device__ __forceinline__ float4 twice_error(const float4& h, const float4& z) {
+  return make_float4(2.f * (z.x - relu(h.x)), 2.f * (z.y - relu(h.y)), 2.f * (z.z - relu(h.z)), 2.f * (z.w - relu(h.w)));
+}
+
+// Scores one finished K_m[i] (k, still without the factor di) against the row's a, b:
+// OUT: a = R'; else a = h and b = twice_error(h, z).
 template <int V, bool OUT>
 __device__ __forceinline__ void score_segment(const float4 (&k)[V], float di, const float4 (&a)[V],
                                               const float4 (&b)[V], const SearchCtl* __restrict__ ctl,
@@ -953,15 +959,14 @@ __device__ __forceinline__ void score_segment(const float4 (&k)[V], float di, co
     for (int v = 0; v < V; ++v) {
       const float kk[4] = {k[v].x, k[v].y, k[v].z, k[v].w};
       const float hh[4] = {a[v].x, a[v].y, a[v].z, a[v].w};
-      const float zz[4] = {b[v].x, b[v].y, b[v].z, b[v].w};
+      const float ee[4] = {b[v].x, b[v].y, b[v].z, b[v].w};   // 2 (z - f(h)), see twice_error
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         const float pos = fmaxf(hh[c], 0.f), neg = fmaxf(-hh[c], 0.f);
-        const float e2 = 2.f * (zz[c] - pos);
 #pragma unroll
         for (int j = 0; j < kCand; ++j) {
           const float df = relu_drop(kk[c], inv[j], neg, pos);
-          part[j] = fmaf(df, e2 + df, part[j]);
+          part[j] = fmaf(df, ee[c] + df, part[j]);   // e1^2 - e0^2 = df (2 e0 + df)
         }
       }
     }
@@ -975,7 +980,7 @@ __device__ __forceinline__ void score_segment(const float4 (&k)[V], float di, co
 }
 
 template <int V, bool OUT, int UN>
-__global__ void __launch_bounds__(256, (V <= 2 ? 3 : 1))
+__global__ void __launch_bounds__(256, (V <= 1 ? 4 : V <= 2 ? 3 : 1))
 k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
           const unsigned short* __restrict__ col_comm, const float* __restrict__ dinv,
           const float4* __restrict__ T, const float4* __restrict__ Hn, const float4* __restrict__ Zn,
@@ -984,9 +989,13 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
           const int4* __restrict__ items, int n_items, int long_len, float4* __restrict__ scratch) {
   if (*n_active <= 0) return;
   constexpr int PER = OUT ? 2 : kCand;
-  extern __shared__ double s_acc[];
+  // dynamic shared memory: per warp the row's a, b (2 V float4 per lane; parked there during the
+  // walk so that the registers hold gathered rows instead), then the per-warp sums
+  extern __shared__ float4 s_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int warps_per_block = blockDim.x >> 5;
+  float4* row_ab = s_raw + (size_t)warp * (2 * V * 32) + lane;
+  double* s_acc = reinterpret_cast<double*>(s_raw + (size_t)warps_per_block * (2 * V * 32));
   double* mine = acc;
   if (use_smem) {
     for (int i = threadIdx.x; i < warps_per_block * n_comm * PER; i += blockDim.x) s_acc[i] = 0.0;
@@ -1015,15 +1024,17 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
       rs = row_ptr[row]; re = row_ptr[row + 1];
       if (re - rs > long_len) continue;
     }
-    float4 a[V], b[V];   // OUT: a = R' ; else a = h, b = z
+    __syncwarp();          // the previous unit's last segment has been scored
 #pragma unroll
-    for (int v = 0; v < V; ++v) {
+    for (int v = 0; v < V; ++v) {   // OUT: a = R' ; else a = h, b = 2 (z - f(h))
       const int f = lane + 32 * v;
-      a[v] = b[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+      float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
       if (f < ld4 && !piece) {
-        if (OUT) a[v] = Rn[(long long)row * ld4 + f];
-        else { a[v] = Hn[(long long)row * ld4 + f]; b[v] = Zn[(long long)row * ld4 + f]; }
+        if (OUT) a = Rn[(long long)row * ld4 + f];
+        else { a = Hn[(long long)row * ld4 + f]; b = twice_error(a, Zn[(long long)row * ld4 + f]); }
       }
+      row_ab[32 * v] = a;
+      if (!OUT) row_ab[32 * (V + v)] = b;
     }
     const float di = dinv[row];
     float4 k[V];
@@ -1042,55 +1053,64 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
         }
         return;
       }
+      float4 a[V], b[V];   // each lane reads back what it stored itself
+#pragma unroll
+      for (int v = 0; v < V; ++v) {
+        a[v] = row_ab[32 * v];
+        b[v] = OUT ? a[v] : row_ab[32 * (V + v)];
+      }
       score_segment<V, OUT>(k, di, a, b, ctl, cur, lane, mine, plain_add);
     };
 
     for (int base = rs; base < re; base += 32) {
       const int idx = base + lane;
-      int c = 0, m = -1;
+      const bool valid = idx < re;
+      int c = 0, m = -1;      // lanes past the row's end hold (column 0, weight 0)
       float w = 0.f;
-      if (idx < re) {
+      bool live = false;      // the entry's community is still searching: its row of T is gathered
+      if (valid) {
         c = col[idx];
         m = col_comm[idx];
-        if (ctl[m].done) m |= 0x10000;     // finished search: keep the community, skip the work
-        else w = dinv[c];
+        live = !ctl[m].done;
+        if (live) w = dinv[c];
       }
+      // entries of one community are contiguous: bit t of `chg` says that entry t opens a new
+      // segment, bit t of `on` that its row is gathered; both are the same in every lane, so the
+      // walk below needs the community of an entry only where a segment starts
+      int mprev = __shfl_up_sync(0xffffffffu, m, 1);
+      if (lane == 0) mprev = cur;
+      unsigned chg = __ballot_sync(0xffffffffu, valid && m != mprev);
+      unsigned on = __ballot_sync(0xffffffffu, live);
       const int cnt = min(32, re - base);
-      for (int t = 0; t < cnt; t += UN) {
-        int cj[UN], mj[UN];
+      for (int t = 0; t < cnt; t += UN, chg >>= UN, on >>= UN) {
+        int cj[UN];
         float wj[UN];
 #pragma unroll
         for (int u = 0; u < UN; ++u) {
-          cj[u] = __shfl_sync(0xffffffffu, c, (t + u) & 31);
-          mj[u] = __shfl_sync(0xffffffffu, m, (t + u) & 31);
-          wj[u] = __shfl_sync(0xffffffffu, w, (t + u) & 31);
-          if (t + u >= cnt) mj[u] = -1;
+          cj[u] = __shfl_sync(0xffffffffu, c, t + u);
+          wj[u] = __shfl_sync(0xffffffffu, w, t + u);
         }
-        float4 xv[UN][V];
+        float4 xv[UN][V];   // set and read under the same condition (entry gathered, column inside the row)
 #pragma unroll
         for (int u = 0; u < UN; ++u)
 #pragma unroll
-          for (int v = 0; v < V; ++v) {
-            const int f = lane + 32 * v;
-            xv[u][v] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (mj[u] >= 0 && mj[u] < 0x10000 && f < ld4) xv[u][v] = __ldg(T + (long long)cj[u] * ld4 + f);
-          }
+          for (int v = 0; v < V; ++v)
+            if (((on >> u) & 1u) && lane + 32 * v < ld4) xv[u][v] = __ldg(T + (long long)cj[u] * ld4 + (lane + 32 * v));
 #pragma unroll
         for (int u = 0; u < UN; ++u) {
-          if (mj[u] < 0) continue;                       // past the end of the row (warp-uniform)
-          const int mm = mj[u] & 0xffff;
-          if (mm != cur) {
+          if ((chg >> u) & 1u) {                          // warp-uniform
             finish_segment();
-            cur = mm;
-            cur_on = mj[u] < 0x10000;
+            cur = __shfl_sync(0xffffffffu, m, t + u);
+            cur_on = (on >> u) & 1u;
 #pragma unroll
             for (int v = 0; v < V; ++v) k[v] = make_float4(0.f, 0.f, 0.f, 0.f);
           }
 #pragma unroll
-          for (int v = 0; v < V; ++v) {
-            k[v].x = fmaf(wj[u], xv[u][v].x, k[v].x); k[v].y = fmaf(wj[u], xv[u][v].y, k[v].y);
-            k[v].z = fmaf(wj[u], xv[u][v].z, k[v].z); k[v].w = fmaf(wj[u], xv[u][v].w, k[v].w);
-          }
+          for (int v = 0; v < V; ++v)
+            if (((on >> u) & 1u) && lane + 32 * v < ld4) {
+              k[v].x = fmaf(wj[u], xv[u][v].x, k[v].x); k[v].y = fmaf(wj[u], xv[u][v].y, k[v].y);
+              k[v].z = fmaf(wj[u], xv[u][v].z, k[v].z); k[v].w = fmaf(wj[u], xv[u][v].w, k[v].w);
+            }
         }
       }
     }
@@ -1128,7 +1148,7 @@ k_score_z_split(const int4* __restrict__ split, int n_split, const float* __rest
     a[v] = b[v] = k[v] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (f < ld4) {
       if (OUT) a[v] = Rn[(long long)sp.x * ld4 + f];
-      else { a[v] = Hn[(long long)sp.x * ld4 + f]; b[v] = Zn[(long long)sp.x * ld4 + f]; }
+      else { a[v] = Hn[(long long)sp.x * ld4 + f]; b[v] = twice_error(a[v], Zn[(long long)sp.x * ld4 + f]); }
       for (int q = 0; q < sp.w; ++q) {
         const float4 t = scratch[(long long)(sp.z + q) * ld4 + f];
         k[v].x += t.x; k[v].y += t.y; k[v].z += t.z; k[v].w += t.w;
