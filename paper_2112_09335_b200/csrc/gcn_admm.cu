@@ -786,6 +786,9 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
     throw Fail{GCN_ADMM_ERR_WIDTHS, "more than 128 classes are not supported"};
   for (int l = 2; l <= n_layers; ++l)
     if (h->ld[l] / 4 > 256) throw Fail{GCN_ADMM_ERR_WIDTHS, "layer widths above 1024 are supported for C_0 only"};
+  for (int l = 1; l <= n_layers; ++l)   // the Z scoring addresses rows of an N x C_l matrix by 32-bit float4 offsets
+    if (n * (long long)(h->ld[l] / 4) >= (1LL << 32))
+      throw Fail{GCN_ADMM_ERR_WIDTHS, "n x layer width exceeds 2^34 elements"};
 
   // host copies of the graph-side inputs, then the index tables
   HostView<long long> rp(row_ptr, (size_t)n + 1);

@@ -1003,6 +1003,10 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
     mine = s_acc + (size_t)warp * n_comm * PER;
   }
   const bool plain_add = use_smem != 0;
+  const float4* __restrict__ T_lane = T + lane;   // rows of T are addressed by 32-bit float4 offsets (n * ld4 < 2^32)
+  bool in_row[V];
+#pragma unroll
+  for (int v = 0; v < V; ++v) in_row[v] = lane + 32 * v < ld4;
   const int n_units = n + n_items;
   // units (items first, then rows) are handed out four at a time from a global counter: row lengths
   // follow a power law, a static deal leaves most warps waiting at the closing barrier for the unlucky ones
@@ -1065,14 +1069,15 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
     for (int base = rs; base < re; base += 32) {
       const int idx = base + lane;
       const bool valid = idx < re;
-      int c = 0, m = -1;      // lanes past the row's end hold (column 0, weight 0)
+      unsigned off = 0u;      // first float4 of the entry's row of T; lanes past the row's end hold (row 0, weight 0)
+      int m = -1;
       float w = 0.f;
       bool live = false;      // the entry's community is still searching: its row of T is gathered
       if (valid) {
-        c = col[idx];
+        const int c = col[idx];
         m = col_comm[idx];
         live = !ctl[m].done;
-        if (live) w = dinv[c];
+        if (live) { w = dinv[c]; off = (unsigned)c * (unsigned)ld4; }
       }
       // entries of one community are contiguous: bit t of `chg` says that entry t opens a new
       // segment, bit t of `on` that its row is gathered; both are the same in every lane, so the
@@ -1083,11 +1088,11 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
       unsigned on = __ballot_sync(0xffffffffu, live);
       const int cnt = min(32, re - base);
       for (int t = 0; t < cnt; t += UN, chg >>= UN, on >>= UN) {
-        int cj[UN];
+        unsigned oj[UN];
         float wj[UN];
 #pragma unroll
         for (int u = 0; u < UN; ++u) {
-          cj[u] = __shfl_sync(0xffffffffu, c, t + u);
+          oj[u] = __shfl_sync(0xffffffffu, off, t + u);
           wj[u] = __shfl_sync(0xffffffffu, w, t + u);
         }
         float4 xv[UN][V];   // set and read under the same condition (entry gathered, column inside the row)
@@ -1095,7 +1100,7 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
         for (int u = 0; u < UN; ++u)
 #pragma unroll
           for (int v = 0; v < V; ++v)
-            if (((on >> u) & 1u) && lane + 32 * v < ld4) xv[u][v] = __ldg(T + (long long)cj[u] * ld4 + (lane + 32 * v));
+            if (((on >> u) & 1u) && in_row[v]) xv[u][v] = __ldg(T_lane + oj[u] + 32 * v);
 #pragma unroll
         for (int u = 0; u < UN; ++u) {
           if ((chg >> u) & 1u) {                          // warp-uniform
@@ -1107,7 +1112,7 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
           }
 #pragma unroll
           for (int v = 0; v < V; ++v)
-            if (((on >> u) & 1u) && lane + 32 * v < ld4) {
+            if (((on >> u) & 1u) && in_row[v]) {
               k[v].x = fmaf(wj[u], xv[u][v].x, k[v].x); k[v].y = fmaf(wj[u], xv[u][v].y, k[v].y);
               k[v].z = fmaf(wj[u], xv[u][v].z, k[v].z); k[v].w = fmaf(wj[u], xv[u][v].w, k[v].w);
             }
