@@ -38,7 +38,7 @@ SM_COUNT = 148
 # DRAM bytes (read + write) per launch from the committed ncu capture of k_spmm at leading dimension 256 on the
 # workload's recipe at scale 0.1 (profiles/k_spmm_powerlaw_xlarge_scale0.1.md); a full-size launch is estimated by
 # the ratio of stored entries, since the excess traffic is neighbour rows that miss L2 (one per such entry).
-NCU_SPMM256 = dict(dram_bytes=1.548e9 + 0.2536e9, nnz=2 * 5653426 + 244903)
+NCU_SPMM256 = dict(dram_bytes=1.461740e9 + 0.271949e9, nnz=2 * 5653426 + 244903)
 
 
 def measured_peaks():
