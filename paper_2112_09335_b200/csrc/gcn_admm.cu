@@ -3,6 +3,7 @@
 #include "../../include/gcn_admm.h"
 
 #include <climits>
+#include <cmath>
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -141,6 +142,7 @@ struct gcn_admm {
   size_t item_sums_elems = 0;
   unsigned char* d_train = nullptr;
   int* d_train_rows = nullptr;            // new ids of the training rows, ascending
+  float* d_fista_momentum = nullptr;      // (t_j - 1) / t_{j+1}, j = 1..fista_iters
 
   std::vector<float*> W, Wt, Z, P, H;   // 1..L
   float* U = nullptr;
@@ -608,9 +610,15 @@ struct gcn_admm {
                                                                       update_z ? 1 : 0);
     CU(cudaGetLastError());
     if (n_train > 0) {
-      gk::k_output_rows<<<(unsigned)cdiv(n_train, warps), warps * 32, 0, stream>>>(
-          Z[L], U, H[L], ld[L], C[L], n_train, d_y, d_train, p.rho, p.loss_scale, p.fista_iters, dual_now ? 1 : 0,
-          update_z ? 1 : 0, d_train_rows);
+#define OUTPUT_ROWS(CPL)                                                                                          \
+  gk::k_output_rows<CPL><<<(unsigned)cdiv(n_train, warps), warps * 32, 0, stream>>>(                              \
+      Z[L], U, H[L], ld[L], C[L], n_train, d_y, d_train, p.rho, p.loss_scale, p.fista_iters, dual_now ? 1 : 0,    \
+      update_z ? 1 : 0, d_train_rows, d_fista_momentum);
+      if (C[L] <= 32) OUTPUT_ROWS(1)
+      else if (C[L] <= 64) OUTPUT_ROWS(2)
+      else if (C[L] <= 96) OUTPUT_ROWS(3)
+      else OUTPUT_ROWS(4)
+#undef OUTPUT_ROWS
       CU(cudaGetLastError());
       ++launches;
     }
@@ -840,6 +848,16 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
     for (long long i = 0; i < n; ++i)
       if (t_new[i]) tr.push_back((int)i);
     h->d_train_rows = upload(h, tr);
+  }
+  {
+    std::vector<float> mom((size_t)std::max(p.fista_iters, 1), 0.f);
+    double t = 1.0;
+    for (int j = 0; j < p.fista_iters; ++j) {
+      const double tn = 0.5 * (1.0 + std::sqrt(1.0 + 4.0 * t * t));
+      mom[(size_t)j] = (float)((t - 1.0) / tn);
+      t = tn;
+    }
+    h->d_fista_momentum = upload(h, mom);
   }
   {
     h->long_len = p.long_row > 0 ? p.long_row : kDefaultLongRow;

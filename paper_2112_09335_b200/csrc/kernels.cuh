@@ -1207,27 +1207,31 @@ __global__ void k_apply_z(float4* __restrict__ Z, const float4* __restrict__ G, 
 //   loss_scale * CE(z, y) + <u, z - q> + (rho/2)||z - q||^2 ;  other rows: z = q - u / rho.
 //   dual_now != 0: U <- u + rho (z_old - q) in the same sweep (Eq. 3 as printed).
 // `rows` (may be NULL = every row) lists the rows to visit: the training rows, when the rest is
-// left to k_output_plain.
+// left to k_output_plain.  CPL = classes per lane (C <= 32 CPL).  momentum[j] = (t_j - 1) / t_{j+1}
+// of FISTA's sequence t_1 = 1, t_{j+1} = (1 + sqrt(1 + 4 t_j^2)) / 2: the same for every row, so it
+// is tabulated once (in fp64) instead of being recomputed by every lane in every iteration.
 // ------------------------------------------------------------------------------------------
+template <int CPL>
 __global__ void __launch_bounds__(256)
 k_output_rows(float* __restrict__ ZL, float* __restrict__ U, const float* __restrict__ HL, int ld, int C,
               int n, const int* __restrict__ y, const unsigned char* __restrict__ train, float rho,
-              float loss_scale, int iters, int dual_now, int update_z, const int* __restrict__ rows) {
+              float loss_scale, int iters, int dual_now, int update_z, const int* __restrict__ rows,
+              const float* __restrict__ momentum) {
   const int lane = threadIdx.x & 31;
   const int slot = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (slot >= n) return;
   const int row = rows != nullptr ? rows[slot] : slot;
-  float q[kMaxClassesPerLane], u[kMaxClassesPerLane], z[kMaxClassesPerLane];
+  float q[CPL], u[CPL], z[CPL];
   const long long base = (long long)row * ld;
 #pragma unroll
-  for (int t = 0; t < kMaxClassesPerLane; ++t) {
+  for (int t = 0; t < CPL; ++t) {
     const int c = lane + 32 * t;
     q[t] = u[t] = z[t] = 0.f;
     if (c < C) { q[t] = HL[base + c]; u[t] = U[base + c]; z[t] = ZL[base + c]; }
   }
   if (dual_now) {
 #pragma unroll
-    for (int t = 0; t < kMaxClassesPerLane; ++t) {
+    for (int t = 0; t < CPL; ++t) {
       const int c = lane + 32 * t;
       if (c < C) U[base + c] = fmaf(rho, z[t] - q[t], u[t]);
     }
@@ -1236,7 +1240,7 @@ k_output_rows(float* __restrict__ ZL, float* __restrict__ U, const float* __rest
   if (!train[row]) {
     const float inv_rho = 1.f / rho;
 #pragma unroll
-    for (int t = 0; t < kMaxClassesPerLane; ++t) {
+    for (int t = 0; t < CPL; ++t) {
       const int c = lane + 32 * t;
       if (c < C) ZL[base + c] = fmaf(-u[t], inv_rho, q[t]);
     }
@@ -1244,28 +1248,26 @@ k_output_rows(float* __restrict__ ZL, float* __restrict__ U, const float* __rest
   }
   const int yi = y[row];
   const float step = 1.f / (0.5f * loss_scale + rho);
-  float xp[kMaxClassesPerLane], v[kMaxClassesPerLane];
+  float xp[CPL], v[CPL];
 #pragma unroll
-  for (int t = 0; t < kMaxClassesPerLane; ++t) { xp[t] = z[t]; v[t] = z[t]; }
-  double tm = 1.0;
+  for (int t = 0; t < CPL; ++t) { xp[t] = z[t]; v[t] = z[t]; }
   for (int it = 0; it < iters; ++it) {
     float mx = -3.0e38f;
 #pragma unroll
-    for (int t = 0; t < kMaxClassesPerLane; ++t)
+    for (int t = 0; t < CPL; ++t)
       if (lane + 32 * t < C) mx = fmaxf(mx, v[t]);
     mx = warp_max(mx);
-    float ex[kMaxClassesPerLane], se = 0.f;
+    float ex[CPL], se = 0.f;
 #pragma unroll
-    for (int t = 0; t < kMaxClassesPerLane; ++t) {
+    for (int t = 0; t < CPL; ++t) {
       ex[t] = (lane + 32 * t < C) ? expf(v[t] - mx) : 0.f;
       se += ex[t];
     }
     se = warp_sum(se);
     const float inv_se = 1.f / se;
-    const double tn = 0.5 * (1.0 + sqrt(1.0 + 4.0 * tm * tm));
-    const float mom = (float)((tm - 1.0) / tn);
+    const float mom = momentum[it];
 #pragma unroll
-    for (int t = 0; t < kMaxClassesPerLane; ++t) {
+    for (int t = 0; t < CPL; ++t) {
       const int c = lane + 32 * t;
       const float p = ex[t] * inv_se - (c == yi ? 1.f : 0.f);
       const float g = loss_scale * p + u[t] + rho * (v[t] - q[t]);
@@ -1273,10 +1275,9 @@ k_output_rows(float* __restrict__ ZL, float* __restrict__ U, const float* __rest
       v[t] = fmaf(mom, x - xp[t], x);
       xp[t] = x;
     }
-    tm = tn;
   }
 #pragma unroll
-  for (int t = 0; t < kMaxClassesPerLane; ++t) {
+  for (int t = 0; t < CPL; ++t) {
     const int c = lane + 32 * t;
     if (c < C) ZL[base + c] = xp[t];
   }
