@@ -175,6 +175,37 @@ def test_single_block_updates_at_tensor_core_sizes(tensor_cores):
         g.destroy()
 
 
+def test_w_block_updates_on_full_powerlaw_large():
+    """Every W block on the whole powerlaw-large workload (169,343 rows): here the transposed product
+    runs in more CTAs than there are SMs (row splits rounded to whole waves, two column groups per
+    split) and the hidden layers' residual operand is formed inside it.  The oracle's W update needs
+    only a handful of full products, so it is affordable at this size; the Z blocks are not."""
+    wl = inputs.make_workload(3)
+    g, o = make_pair(wl)
+    try:
+        o.forced_tol = 1e-4
+        L = o.L
+        Z0, U0 = perturbed(wl, o, seed=11)
+        W0 = [None] + [w.copy() for w in o.W[1:]]
+        tau = [None] + [0.37] * L
+        for l in range(1, L + 1):
+            push_state(g, o, Z=Z0, U=U0, W=W0, tau=tau)
+            Wn, t, rec = o.update_W(l)
+            g.step_block(binding.PHASE_W, l)
+            dec = g.decisions()
+            rec, redo = check_trial(f"W{l}", rec, int(dec["trial_w"][0, l - 1]), lambda f: o.update_W(l, forced=f))
+            if redo:
+                Wn, t = redo[0], redo[1]
+            got = g.get_state(binding.ST_W, l)
+            e, estep = relerr(got, Wn), relerr(got - o.W[l], Wn - o.W[l])
+            print(f"\n  W{l}: rel {e:.2e}  step-rel {estep:.2e}  trial {rec['trial']}")
+            assert e <= BLOCK_TOL, (l, e)
+            assert estep <= 2e-3, (l, estep)
+            assert abs(g.get_state(binding.ST_TAU, l)[0] - t) <= 1e-12 * t
+    finally:
+        g.destroy()
+
+
 @pytest.mark.parametrize("dual_mode", [0, 1])
 def test_ten_iterations(case, dual_mode):
     wl, g0, o0 = case
