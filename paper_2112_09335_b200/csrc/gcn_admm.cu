@@ -563,7 +563,28 @@ struct gcn_admm {
     if (out) {
       {
         Scope sc(this, zname, 1, zbytes, 2.0 * (double)gi.nnz * ldn);
-        SCORE_Z_ANY(true)
+        if (ld4 <= 16) {   // narrow output layer: two rows per warp (see k_score_z_out_half)
+          const size_t smem_h = (size_t)2 * warps * M * 2 * sizeof(double);
+          const int use_smem_h = smem_h <= 96 * 1024;
+          const size_t dyn_h = use_smem_h ? smem_h : 0;
+          if (dyn_h > 48 * 1024)
+            CU(cudaFuncSetAttribute(gk::k_score_z_out_half<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_h));
+          CU(cudaMemsetAsync(row_counter, 0, sizeof(int), stream));
+          int occ = 1;
+          CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gk::k_score_z_out_half<4>, warps * 32, dyn_h));
+          const unsigned grid = (unsigned)std::min<long long>(cdiv(n + n_items, 2 * warps), (long long)kSmCount * std::max(occ, 1));
+          gk::k_score_z_out_half<4><<<grid, warps * 32, dyn_h, stream>>>(d_row_ptr, d_col, d_col_comm, d_dinv,
+              (const float4*)B1, (const float4*)B0, ld4, (int)n, ctl, M, acc_z, n_active, use_smem_h, row_counter, d_items,
+              n_items, long_len, reinterpret_cast<float4*>(item_sums));
+          if (n_split > 0) {
+            gk::k_score_z_split<1, true><<<(unsigned)cdiv(n_split, warps), warps * 32, 0, stream>>>(d_split, n_split, d_dinv,
+                reinterpret_cast<const float4*>(item_sums), (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0,
+                ld4, ctl, acc_z, n_active);
+            ++launches;
+          }
+        } else {
+          SCORE_Z_ANY(true)
+        }
       }
       a.mode = 1;
       a.quad_coef = 0.5 * p.rho;

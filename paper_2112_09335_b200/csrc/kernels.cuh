@@ -1132,6 +1132,147 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
   }
 }
 
+// The output-layer form of k_score_z (OUT = true) for rows of at most 16 float4 (C_L <= 64), two
+// units per warp: each half-warp walks its own row or item, 16 stored entries per chunk.  With 12 of
+// 32 lanes carrying columns (47 classes) the full-warp form spends most of its issue slots on lanes
+// that hold nothing; here every instruction of the walk serves two rows.  Control flow is kept the
+// same for both halves (loop bounds are the larger of the two, a half that has run out holds weight 0
+// and no segment start), shuffles use width 16, and only the closing of a segment is a divergent
+// branch, inside which nothing is exchanged beyond the half's own 16 lanes.  Sums go to one array
+// per half-warp (the halves may close segments of the same community at the same time).
+// Dynamic shared memory: 2 x warps x n_comm x 2 doubles when use_smem != 0.
+template <int UN>
+__global__ void __launch_bounds__(256, 4)
+k_score_z_out_half(const int* __restrict__ row_ptr, const int* __restrict__ col,
+                   const unsigned short* __restrict__ col_comm, const float* __restrict__ dinv,
+                   const float4* __restrict__ T, const float4* __restrict__ Rn, int ld4, int n,
+                   const SearchCtl* __restrict__ ctl, int n_comm, double* __restrict__ acc,
+                   const int* __restrict__ n_active, int use_smem, int* __restrict__ row_counter,
+                   const int4* __restrict__ items, int n_items, int long_len, float4* __restrict__ scratch) {
+  if (*n_active <= 0) return;
+  static_assert(16 % UN == 0, "UN divides the chunk");
+  extern __shared__ double s_half[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, half = lane >> 4, hl = lane & 15;
+  const int warps_per_block = blockDim.x >> 5;
+  const unsigned hmask = 0xffffu << (16 * half);
+  double* mine = acc;
+  if (use_smem) {
+    for (int i = threadIdx.x; i < 2 * warps_per_block * n_comm * 2; i += blockDim.x) s_half[i] = 0.0;
+    __syncthreads();
+    mine = s_half + (size_t)(2 * warp + half) * n_comm * 2;
+  }
+  const bool plain_add = use_smem != 0;
+  const bool in_row = hl < ld4;
+  const float4* __restrict__ T_lane = T + hl;
+  const int n_units = n + n_items;
+  for (;;) {
+    int unit_base = 0;
+    if (lane == 0) unit_base = atomicAdd(row_counter, 4);
+    unit_base = __shfl_sync(0xffffffffu, unit_base, 0);
+    if (unit_base >= n_units) break;
+    for (int pair = 0; pair < 2; ++pair) {
+      const int unit = unit_base + 2 * pair + half;
+      int row = 0, rs = 0, re = 0;
+      bool piece = false;
+      if (unit < n_units) {
+        if (unit < n_items) {
+          const int4 it = items[unit];
+          row = it.x; rs = it.y; re = it.z;
+          piece = it.w >= 0;
+        } else {
+          row = unit - n_items;
+          rs = row_ptr[row]; re = row_ptr[row + 1];
+          if (re - rs > long_len) re = rs;          // walked as items
+        }
+      }
+      float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (in_row && !piece && re > rs) a = Rn[(long long)row * ld4 + hl];
+      const float di = dinv[row];
+      float4 k = make_float4(0.f, 0.f, 0.f, 0.f);
+      int cur = -1;
+      bool cur_on = false;
+
+      auto finish_segment = [&]() {   // called by one half at a time: exchanges stay inside hmask
+        if (!cur_on) return;
+        if (piece) {
+          if (in_row) scratch[(long long)unit * ld4 + hl] = k;
+          return;
+        }
+        const float kx = di * k.x, ky = di * k.y, kz = di * k.z, kw = di * k.w;
+        const float p1 = kx * a.x + ky * a.y + kz * a.z + kw * a.w;
+        const float p2 = kx * kx + ky * ky + kz * kz + kw * kw;
+        const bool up8 = hl & 8;
+        float c = (up8 ? p2 : p1) + __shfl_xor_sync(hmask, up8 ? p1 : p2, 8, 16);
+        c += __shfl_xor_sync(hmask, c, 4, 16);
+        c += __shfl_xor_sync(hmask, c, 2, 16);
+        c += __shfl_xor_sync(hmask, c, 1, 16);
+        if ((hl & 7) == 0) {
+          double* dst = mine + cur * 2 + (hl >> 3);
+          if (plain_add) *dst += (double)c; else atomicAdd(dst, (double)c);
+        }
+      };
+
+      const int len = re - rs;
+      const int len_max = max(len, __shfl_xor_sync(0xffffffffu, len, 16));
+      for (int o = 0; o < len_max; o += 16) {
+        const int idx = rs + o + hl;
+        const bool valid = idx < re;
+        unsigned off = 0u;
+        int m = -1;
+        float w = 0.f;
+        bool live = false;
+        if (valid) {
+          const int c = col[idx];
+          m = col_comm[idx];
+          live = !ctl[m].done;
+          if (live) { w = dinv[c]; off = (unsigned)c * (unsigned)ld4; }
+        }
+        int mprev = __shfl_up_sync(0xffffffffu, m, 1, 16);
+        if (hl == 0) mprev = cur;
+        unsigned chg = (__ballot_sync(0xffffffffu, valid && m != mprev) >> (16 * half)) & 0xffffu;
+        unsigned on = (__ballot_sync(0xffffffffu, live) >> (16 * half)) & 0xffffu;
+        const int cnt_max = min(16, len_max - o);
+        for (int t = 0; t < cnt_max; t += UN, chg >>= UN, on >>= UN) {
+          unsigned oj[UN];
+          float wj[UN];
+#pragma unroll
+          for (int u = 0; u < UN; ++u) {
+            oj[u] = __shfl_sync(0xffffffffu, off, t + u, 16);
+            wj[u] = __shfl_sync(0xffffffffu, w, t + u, 16);
+          }
+          float4 xv[UN];   // set and read under the same condition
+#pragma unroll
+          for (int u = 0; u < UN; ++u)
+            if (((on >> u) & 1u) && in_row) xv[u] = __ldg(T_lane + oj[u]);
+#pragma unroll
+          for (int u = 0; u < UN; ++u) {
+            if ((chg >> u) & 1u) {                        // uniform within the half
+              finish_segment();
+              cur = col_comm[rs + o + t + u];
+              cur_on = (on >> u) & 1u;
+              k = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            if (((on >> u) & 1u) && in_row) {
+              k.x = fmaf(wj[u], xv[u].x, k.x); k.y = fmaf(wj[u], xv[u].y, k.y);
+              k.z = fmaf(wj[u], xv[u].z, k.z); k.w = fmaf(wj[u], xv[u].w, k.w);
+            }
+          }
+        }
+      }
+      finish_segment();
+      __syncwarp();
+    }
+  }
+  if (use_smem) {
+    __syncthreads();
+    for (int i = threadIdx.x; i < n_comm * 2; i += blockDim.x) {
+      double t = 0.0;
+      for (int q = 0; q < 2 * warps_per_block; ++q) t += s_half[(size_t)q * n_comm * 2 + i];
+      if (t != 0.0) atomicAdd(acc + i, t);
+    }
+  }
+}
+
 // Segments that k_score_z handled in pieces: K_m[i] = sum of the pieces (item order), then scored
 // as above.  split[s] = {row, community, first item, number of items}; one warp per entry.
 template <int V, bool OUT>
