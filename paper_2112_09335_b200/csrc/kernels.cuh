@@ -1066,18 +1066,23 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
       score_segment<V, OUT>(k, di, a, b, ctl, cur, lane, mine, plain_add);
     };
 
+    // column and community of a chunk are fetched while the chunk before it is walked; the two
+    // loads that depend on them (weight, search state) are issued together, not one after the other
+    int c_next = 0, m_next = -1;
+    if (rs + lane < re) { c_next = col[rs + lane]; m_next = col_comm[rs + lane]; }
     for (int base = rs; base < re; base += 32) {
       const int idx = base + lane;
       const bool valid = idx < re;
+      const int c = c_next, m = m_next;
+      if (idx + 32 < re) { c_next = col[idx + 32]; m_next = col_comm[idx + 32]; }
+      else m_next = -1;
       unsigned off = 0u;      // first float4 of the entry's row of T; lanes past the row's end hold (row 0, weight 0)
-      int m = -1;
       float w = 0.f;
       bool live = false;      // the entry's community is still searching: its row of T is gathered
       if (valid) {
-        const int c = col[idx];
-        m = col_comm[idx];
+        const float wc = dinv[c];
         live = !ctl[m].done;
-        if (live) { w = dinv[c]; off = (unsigned)c * (unsigned)ld4; }
+        if (live) { w = wc; off = (unsigned)c * (unsigned)ld4; }
       }
       // entries of one community are contiguous: bit t of `chg` says that entry t opens a new
       // segment, bit t of `on` that its row is gathered; both are the same in every lane, so the
@@ -1214,18 +1219,21 @@ k_score_z_out_half(const int* __restrict__ row_ptr, const int* __restrict__ col,
 
       const int len = re - rs;
       const int len_max = max(len, __shfl_xor_sync(0xffffffffu, len, 16));
+      int c_next = 0, m_next = -1;   // fetched one chunk ahead, as in k_score_z
+      if (rs + hl < re) { c_next = col[rs + hl]; m_next = col_comm[rs + hl]; }
       for (int o = 0; o < len_max; o += 16) {
         const int idx = rs + o + hl;
         const bool valid = idx < re;
+        const int c = c_next, m = m_next;
+        if (idx + 16 < re) { c_next = col[idx + 16]; m_next = col_comm[idx + 16]; }
+        else m_next = -1;
         unsigned off = 0u;
-        int m = -1;
         float w = 0.f;
         bool live = false;
         if (valid) {
-          const int c = col[idx];
-          m = col_comm[idx];
+          const float wc = dinv[c];
           live = !ctl[m].done;
-          if (live) { w = dinv[c]; off = (unsigned)c * (unsigned)ld4; }
+          if (live) { w = wc; off = (unsigned)c * (unsigned)ld4; }
         }
         int mprev = __shfl_up_sync(0xffffffffu, m, 1, 16);
         if (hl == 0) mprev = cur;
