@@ -1016,18 +1016,35 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
     unit_base = __shfl_sync(0xffffffffu, unit_base, 0);
     if (unit_base >= n_units) break;
     const int unit_end = min(n_units, unit_base + 4);
-  for (int unit = unit_base; unit < unit_end; ++unit) {
-    int row, rs, re;
-    bool piece = false;
-    if (unit < n_items) {
-      const int4 it = items[unit];
-      row = it.x; rs = it.y; re = it.z;
-      piece = it.w >= 0;
-    } else {
-      row = unit - n_items;
-      rs = row_ptr[row]; re = row_ptr[row + 1];
-      if (re - rs > long_len) continue;
+    // lanes 0..3 fetch the descriptions of the four units together (one load latency, not four)
+    int4 my_unit = make_int4(0, 0, 0, -1);   // row, first entry, one past the last, split (>= 0: a piece)
+    if (lane < 4 && unit_base + lane < unit_end) {
+      const int u = unit_base + lane;
+      if (u < n_items) my_unit = items[u];
+      else {
+        const int r = u - n_items;
+        my_unit = make_int4(r, row_ptr[r], row_ptr[r + 1], -1);
+        if (my_unit.z - my_unit.y > long_len) my_unit.z = my_unit.y;   // walked as items
+      }
     }
+    // column and community of a unit's first chunk are fetched while the unit before it is walked
+    int c_first = 0, m_first = -1;
+    {
+      const int s0 = __shfl_sync(0xffffffffu, my_unit.y, 0), e0 = __shfl_sync(0xffffffffu, my_unit.z, 0);
+      if (s0 + lane < e0) { c_first = col[s0 + lane]; m_first = col_comm[s0 + lane]; }
+    }
+  for (int unit = unit_base; unit < unit_end; ++unit) {
+    const int q = unit - unit_base;
+    const int row = __shfl_sync(0xffffffffu, my_unit.x, q);
+    const int rs = __shfl_sync(0xffffffffu, my_unit.y, q), re = __shfl_sync(0xffffffffu, my_unit.z, q);
+    const bool piece = __shfl_sync(0xffffffffu, my_unit.w, q) >= 0;
+    int c_next = c_first, m_next = m_first;
+    {
+      const int s1 = __shfl_sync(0xffffffffu, my_unit.y, (q + 1) & 3), e1 = __shfl_sync(0xffffffffu, my_unit.z, (q + 1) & 3);
+      m_first = -1;
+      if (q + 1 < unit_end - unit_base && s1 + lane < e1) { c_first = col[s1 + lane]; m_first = col_comm[s1 + lane]; }
+    }
+    if (rs >= re) continue;
     __syncwarp();          // the previous unit's last segment has been scored
 #pragma unroll
     for (int v = 0; v < V; ++v) {   // OUT: a = R' ; else a = h, b = 2 (z - f(h))
@@ -1068,8 +1085,6 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
 
     // column and community of a chunk are fetched while the chunk before it is walked; the two
     // loads that depend on them (weight, search state) are issued together, not one after the other
-    int c_next = 0, m_next = -1;
-    if (rs + lane < re) { c_next = col[rs + lane]; m_next = col_comm[rs + lane]; }
     for (int base = rs; base < re; base += 32) {
       const int idx = base + lane;
       const bool valid = idx < re;
