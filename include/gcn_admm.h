@@ -66,7 +66,7 @@ enum {
  *                  forms run at the same ~10 TB/s of gathered bytes on B200, the ring is kept for comparison)
  *  use_graph       1: gcn_admm_step records one pass as a CUDA graph on first use and replays it (only when
  *                  the handle's stream is not the default stream and profiling is off); 2: the same, but
- *                  only for problems small enough to be launch-bound (N x widest layer < 2^25);
+ *                  only for problems small enough for launch gaps to show (N x widest layer < 2^27);
  *                  0: plain launches
  *  schedule        0: Algorithm 1 (every W_l, then every Z_{l,m}, then U; Jacobi inside a pass);
  *                  1: the serial schedule of Section 4.1 (W_1, Z_1, .., W_L, Z_L, U one after the other,

@@ -1092,7 +1092,7 @@ int gcn_admm_step(gcn_admm* h, int n_iters) {
     // A pass is a fixed sequence of launches (every decision is taken on the device), so on a stream
     // that can be captured it is recorded once and replayed: the small workloads are launch-bound.
     // use_graph 1: always; 2: only where a pass is short enough for launch overhead to matter
-    const bool wanted = h->p.use_graph == 1 || (h->p.use_graph == 2 && h->n * (long long)h->max_ld < (1LL << 25));
+    const bool wanted = h->p.use_graph == 1 || (h->p.use_graph == 2 && h->n * (long long)h->max_ld < (1LL << 27));
     const bool replay = wanted && h->stream != nullptr && !h->profiling && n_iters >= 2;
     if (!replay) {
       for (int k = 0; k < n_iters; ++k) h->iterate();
