@@ -37,7 +37,8 @@ enum {
   GCN_ADMM_ERR_GRAPH = -2,     /* CSR not monotone / column out of range / unsorted or duplicate
                                   columns / not symmetric / more than 2^31-1 stored entries */
   GCN_ADMM_ERR_COMMUNITY = -3, /* community id outside 0..M-1, or an empty community */
-  GCN_ADMM_ERR_WIDTHS = -4,    /* a width < 1, fewer than 1 layer, C_L > 128, label >= C_L */
+  GCN_ADMM_ERR_WIDTHS = -4,    /* a width < 1, fewer than 1 layer, C_L > 128, label >= C_L, a hidden width above 1024,
+                                  or n x (C_l rounded up to 4) of 2^34 elements or more for some layer l >= 1 */
   GCN_ADMM_ERR_ALLOC = -5,     /* host or device allocation failed */
   GCN_ADMM_ERR_CUDA = -6,      /* any CUDA runtime failure, including "no device" */
   GCN_ADMM_ERR_NONFINITE = -7  /* a NaN or infinity reached a step-size decision */
