@@ -256,10 +256,10 @@ struct gcn_admm {
       gtc::k_split_b<<<(unsigned)std::min<long long>(cdiv(work, 256), 4 * kSmCount), 256, 0, stream>>>(Bk, ldbk, N, K, NT, b_image); \
       ++launches;                                                                                              \
       CU(cudaFuncSetAttribute(gtc::k_gemm_tc_ws<NT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-      gtc::k_gemm_tc_ws<NT, true><<<grid, gtc::kWsThreads, smem, stream>>>(A, lda, Bk, ldbk, Cm, ldc, (int)Mr, N, K, skip, tc_error, b_image); \
+      gtc::k_gemm_tc_ws<NT, true><<<grid, gtc::WsCfg<NT>::kThreads, smem, stream>>>(A, lda, Bk, ldbk, Cm, ldc, (int)Mr, N, K, skip, tc_error, b_image); \
     } else {                                                                                                   \
       CU(cudaFuncSetAttribute(gtc::k_gemm_tc_ws<NT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-      gtc::k_gemm_tc_ws<NT, false><<<grid, gtc::kWsThreads, smem, stream>>>(A, lda, Bk, ldbk, Cm, ldc, (int)Mr, N, K, skip, tc_error, nullptr); \
+      gtc::k_gemm_tc_ws<NT, false><<<grid, gtc::WsCfg<NT>::kThreads, smem, stream>>>(A, lda, Bk, ldbk, Cm, ldc, (int)Mr, N, K, skip, tc_error, nullptr); \
     }                                                                                                          \
   }
         if (N <= 16) TC_WS(16)
