@@ -308,6 +308,14 @@ def run_ours(args):
         roofline["note"] = ("gather kernel: every stored entry pulls a full operand row through L2 (nnz x ld x 4 B, about "
                             "23x the algorithmic bytes at mean degree 50), so it runs at the L2-to-SM rate, not at the HBM "
                             "rate; algorithmic bytes = 4 nnz + 8 N + 8 N ld")
+    if dominant["kernel"].startswith("spmm@"):
+        # what the kernel pulls through L2: one operand row per stored entry of A + I
+        ldw = int(dominant["kernel"].split("@")[1])
+        gathered = float(2 * wl.n_edges + wl.n) * ldw * 4.0
+        per_launch_s = dominant["ms_per_iter"] / max(dominant["launches_per_iter"], 1e-9) * 1e-3
+        roofline["l2_gather"] = dict(bytes_per_launch=gathered, gbs=gathered / per_launch_s / 1e9,
+                                     ncu_l2_sector_rate_of_peak=0.79,
+                                     source="profiles/k_spmm_powerlaw_xlarge_scale0.1.md (lts__t_sectors_srcunit_tex)")
     roofline.update(kernel=dominant["kernel"], ms_per_launch=dominant["ms_per_iter"] / max(dominant["launches_per_iter"], 1e-9),
                     share_of_kernel_time=dominant["share"])
 
