@@ -653,9 +653,17 @@ struct gcn_admm {
   }
 
   // P_l = A~ Z_{l-1} (l >= 2; P_1 is constant) and H_l = P_l W_l from the stored W, Z.
-  void refresh() {
+  // keep_h1: the caller knows that H_1 already is P_1 W_1.  After a pass it is: P_1 never changes and
+  // the W_1 step left H_1 - D/tau = P_1 (W_1 - grad/tau) behind, so the product is skipped; to keep
+  // rounding from piling up over many passes it is still formed afresh every kH1RefreshEvery passes.
+  static constexpr int kH1RefreshEvery = 16;
+  int h1_age = 0;
+  bool capturing = false;
+  void refresh(bool keep_h1 = false) {
     for (int l = 2; l <= L; ++l) spmm(Z[l - 1], P[l], ld[l - 1]);
-    for (int l = 1; l <= L; ++l)
+    const bool skip_h1 = keep_h1 && !capturing && h1_age + 1 < kH1RefreshEvery;
+    h1_age = skip_h1 ? h1_age + 1 : 0;
+    for (int l = skip_h1 ? 2 : 1; l <= L; ++l)
       gemm_nn(P[l], ld[l - 1], W[l], ld[l], Wt[l], ld[l - 1], H[l], ld[l], n, C[l], C[l - 1]);
     fresh = true;
   }
@@ -674,7 +682,7 @@ struct gcn_admm {
       if (l < L) update_Z_hidden(l);
       else update_output(false, true);
     }
-    refresh();
+    refresh(true);
     dual_from_stored();
     end_log_pass();
   }
@@ -686,7 +694,7 @@ struct gcn_admm {
     for (int l = 1; l <= L; ++l) update_W(l);
     for (int l = 1; l < L; ++l) update_Z_hidden(l);
     update_output(p.dual_mode == 0, true);
-    refresh();
+    refresh(true);
     if (p.dual_mode != 0) dual_from_stored();
     end_log_pass();
   }
@@ -1103,9 +1111,12 @@ int gcn_admm_step(gcn_admm* h, int n_iters) {
       cudaGraph_t graph = nullptr;
       CU(cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
       const long long launches_before = h->launches, log_before = h->log_count;
+      h->capturing = true;          // the recorded pass is replayed many times: it forms every product
       try {
         h->iterate();
+        h->capturing = false;
       } catch (...) {
+        h->capturing = false;
         cudaStreamEndCapture(h->stream, &graph);
         if (graph) cudaGraphDestroy(graph);
         throw;
