@@ -38,3 +38,31 @@ def test_graph_replay_matches_plain_launches(index, scale):
         finally:
             a.destroy()
             b.destroy()
+
+
+def test_kept_first_layer_product_over_many_passes():
+    """Plain launches keep H_1 = P_1 W_1 from the W_1 step and form it afresh only every 16th pass; a
+    recorded graph forms it in every pass.  Over 36 passes (two refresh points) both must give the same
+    iterates up to rounding."""
+    import torch
+    wl = inputs.make_workload(0)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        def make(use_graph):
+            return binding.GcnAdmm(wl.n, wl.row_ptr, wl.col_idx, wl.X, wl.y, wl.train_mask, wl.widths, wl.n_comm,
+                                   wl.community, wl.w_init, nu=wl.nu, rho=wl.rho, stream=side.cuda_stream,
+                                   use_graph=use_graph)
+        a, b = make(1), make(0)
+        try:
+            a.step(36)
+            b.step(36)
+            side.synchronize()
+            da, db = a.decisions(), b.decisions()
+            assert np.array_equal(da["trial_w"], db["trial_w"]) and np.array_equal(da["trial_z"], db["trial_z"])
+            for l in range(1, len(wl.widths)):
+                assert relerr(a.get_state(binding.ST_W, l), b.get_state(binding.ST_W, l)) < 1e-5
+                assert relerr(a.get_state(binding.ST_Z, l), b.get_state(binding.ST_Z, l)) < 1e-5
+            assert a.launches() - b.launches() == 36 - 2      # passes 16 and 32 formed the product again
+        finally:
+            a.destroy()
+            b.destroy()
