@@ -438,3 +438,102 @@ def test_sequential_schedule_uses_latest_values():
     np.testing.assert_array_equal(o.W[1], W1)
     np.testing.assert_array_equal(o.Z[1], Z1)
     np.testing.assert_array_equal(o.W[2], W2)
+
+
+# ---- time indices of Algorithm 1 (Appendix A, first display; Eq. 3) -------------------------
+
+def dense_hidden_gradient(At, nu, rho, L, l, W, Z, U):
+    """Full-graph gradient of the Z_l objective (Eq. 5 / Eq. 6) from dense matrices, with the
+    weights, states and dual handed in, so the caller chooses the time index of each."""
+    H = At @ Z[l - 1] @ W[l]
+    Hn = At @ Z[l] @ W[l + 1]
+    if l + 1 < L:
+        back = nu * (np.maximum(Hn, 0) - Z[l + 1]) * (Hn > 0)
+    else:
+        back = -(U + rho * (Z[L] - Hn))
+    return nu * (Z[l] - np.maximum(H, 0)) + At.T @ back @ W[l + 1].T
+
+
+@pytest.mark.parametrize("seed,dual_mode", [(51, 0), (52, 1), (53, 0)])
+def test_one_pass_reads_the_iterates_algorithm_1_names(seed, dual_mode):
+    """Algorithm 1 with Appendix A's first display: every W_l from (W^k, Z^k, U^k); every Z_{l,m} and Z_L
+    from (W^{k+1}, Z^k, U^k), layers and communities in parallel; U by Eq. 3.  Checked two ways:
+    against dense-matrix formulas evaluated at those iterates (the step times its parameter must be
+    the gradient there), and against a pass assembled by hand from single block updates of a twin."""
+    pr, o = make(seed, n=26, widths=(5, 6, 4, 4, 3))
+    pr, ref = make(seed, n=26, widths=(5, 6, 4, 4, 3))
+    o.p.dual_mode = ref.p.dual_mode = dual_mode
+    for x in (o, ref):                       # low starting parameters: every search runs a few trials
+        x.tau = [None] + [1e-2] * x.L
+        x.theta = [None] + [[1e-2] * x.M for _ in range(1, x.L)]
+    At = dense_At(pr)
+    L, M, nu, rho = o.L, o.M, o.p.nu, o.p.rho
+    Wk = [None] + [w.copy() for w in o.W[1:]]
+    Zk = [z.copy() for z in o.Z]
+    Uk = o.U.copy()
+    rec = o.iterate()
+    assert all(r["trial"] >= 0 for r in rec["W"].values()) and all(r["trial"] >= 0 for r in rec["Z"].values())
+
+    # (a) dense formulas at the iterates the paper names
+    for l in range(1, L + 1):
+        P = At @ Zk[l - 1]
+        H = P @ Wk[l]
+        if l < L:
+            g = nu * P.T @ ((np.maximum(H, 0) - Zk[l]) * (H > 0))
+        else:
+            g = -P.T @ (Uk + rho * (Zk[L] - H))
+        np.testing.assert_allclose((Wk[l] - o.W[l]) * o.tau[l], g, rtol=1e-9, atol=1e-12)
+    for l in range(1, L):
+        G = dense_hidden_gradient(At, nu, rho, L, l, o.W, Zk, Uk)        # W^{k+1}, Z^k, U^k
+        for m in range(M):
+            Vm = o.V[m]
+            np.testing.assert_allclose((Zk[l][Vm] - o.Z[l][Vm]) * o.theta[l][m], G[Vm], rtol=1e-9, atol=1e-12)
+        # the neighbouring readings (W^k; layers below l already at k+1) give a different matrix
+        assert np.abs(dense_hidden_gradient(At, nu, rho, L, l, Wk, Zk, Uk) - G).max() > 1e-6
+        if l > 1:
+            Zgs = [o.Z[j] if 1 <= j < l else Zk[j] for j in range(L + 1)]
+            assert np.abs(dense_hidden_gradient(At, nu, rho, L, l, o.W, Zgs, Uk) - G).max() > 1e-6
+    off = ~o.train
+    q = At @ Zk[L - 1] @ o.W[L]                                           # Z_{L-1}^k with W_L^{k+1}
+    np.testing.assert_allclose(o.Z[L][off], q[off] - Uk[off] / rho, atol=1e-11)
+    assert np.abs(q - At @ Zk[L - 1] @ Wk[L]).max() > 1e-6 and np.abs(q - At @ o.Z[L - 1] @ o.W[L]).max() > 1e-6
+    Zd = Zk if dual_mode == 0 else o.Z
+    np.testing.assert_allclose(o.U, Uk + rho * (Zd[L] - At @ Zd[L - 1] @ o.W[L]), atol=1e-12)
+
+    # (b) the same pass assembled from single block updates of the twin
+    Wn, taun = list(ref.W), list(ref.tau)
+    for l in range(1, L + 1):
+        Wn[l], taun[l], _ = ref.update_W(l)
+    Zn = [z.copy() for z in ref.Z]
+    thetan = [None] + [list(t) for t in ref.theta[1:]]
+    for l in range(1, L):
+        for m in range(M):
+            Zn[l][ref.V[m]], thetan[l][m], _ = ref.update_Z(l, m, Wn)      # ref.Z, ref.U still at k
+    Zn[L] = ref.update_ZL(Wn)
+    Un = ref.update_U(Wn, ref.Z if dual_mode == 0 else Zn)
+    for l in range(1, L + 1):
+        np.testing.assert_array_equal(o.W[l], Wn[l])
+        np.testing.assert_array_equal(o.Z[l], Zn[l])
+        assert o.tau[l] == taun[l]
+    for l in range(1, L):
+        assert o.theta[l] == thetan[l]
+    np.testing.assert_array_equal(o.U, Un)
+
+
+def test_train_accuracy_is_that_of_the_forward_pass():
+    """Entry 5 of objective() is the accuracy of predict() (Problem 1's network with the current W), not
+    of the auxiliary Z_L: away from the forward-consistent start the two differ."""
+    pr, o = make(57, n=40, n_train=30, perturb=0)
+    rng = np.random.default_rng(5)
+    o.Z[o.L] = rng.standard_normal(o.Z[o.L].shape) * 3.0       # Z_L no longer the network's output
+    At = dense_At(pr)
+    Z = pr["X"]
+    for l in range(1, o.L + 1):
+        Z = At @ Z @ o.W[l]
+        if l < o.L:
+            Z = np.maximum(Z, 0)
+    tr = np.flatnonzero(o.train)
+    acc_net = np.mean(np.argmax(Z[tr], 1) == o.y[tr])
+    acc_aux = np.mean(np.argmax(o.Z[o.L][tr], 1) == o.y[tr])
+    assert acc_net != acc_aux
+    assert o.objective()[5] == acc_net
