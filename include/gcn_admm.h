@@ -37,7 +37,7 @@ enum {
   GCN_ADMM_ERR_GRAPH = -2,     /* CSR not monotone / column out of range / unsorted or duplicate
                                   columns / not symmetric / more than 2^31-1 stored entries */
   GCN_ADMM_ERR_COMMUNITY = -3, /* community id outside 0..M-1, or an empty community */
-  GCN_ADMM_ERR_WIDTHS = -4,    /* a width < 1, fewer than 1 layer, C_L > 128, label >= C_L, a hidden width above 1024,
+  GCN_ADMM_ERR_WIDTHS = -4,    /* a width < 1, fewer than 1 layer, C_L > 128, label >= C_L, a width C_l above 1024 for some l >= 2,
                                   or n x (C_l rounded up to 4) of 2^34 elements or more for some layer l >= 1 */
   GCN_ADMM_ERR_ALLOC = -5,     /* host or device allocation failed */
   GCN_ADMM_ERR_CUDA = -6,      /* any CUDA runtime failure, including "no device" */
@@ -55,16 +55,12 @@ enum {
  *                  1/(loss_scale/2 + rho), t_1 = 1, warm start, no early exit)
  *  loss_scale      R = loss_scale * sum over training rows of the softmax cross-entropy
  *  dual_mode       0: Eq. 3 as printed (Z_L^k, Z_{L-1}^k, W_L^{k+1}); 1: the k+1 iterates
- *  tensor_cores    1: dense products with at most 256 output columns and K <= 512 run on the tensor
- *                  cores as an error-compensated TF32 product (three passes, fp32 accumulation,
- *                  relative error of a few 1e-7 of sum |a||b|); 2: the same product with its earlier, unsplit
- *                  scheduling (kept for comparison); 0: fp32 FMA kernels everywhere.  With 1, products of
- *                  16384 rows or more first split the weight operand once into the staged layout and
- *                  fetch it with bulk copies (smaller ones re-split it per row tile, which is cheaper
- *                  than another launch); 3: the same kernels, pre-split at every size
- *  spmm_ring       0: propagation gathers neighbour rows into registers; 1: rows of 68..256 floats are
- *                  kept in flight in a shared-memory ring filled with cp.async instead (same result; both
- *                  forms run at the same ~10 TB/s of gathered bytes on B200, the ring is kept for comparison)
+ *  tensor_cores    1: dense products with 8 <= K <= 2048 and at least 512 rows run on the tensor cores as an
+ *                  error-compensated TF32 product (three passes, fp32 accumulation, relative error of a few
+ *                  1e-7 of sum |a||b|); products of 16384 rows or more first split the weight operand once
+ *                  into the staged layout and fetch it with bulk copies (smaller ones re-split it per row
+ *                  tile, which is cheaper than another launch); 2: the same kernels, pre-split at every
+ *                  size; 0: fp32 FMA kernels everywhere
  *  use_graph       1: gcn_admm_step records one pass as a CUDA graph on first use and replays it (only when
  *                  the handle's stream is not the default stream and profiling is off); 2: the same, but
  *                  only for problems small enough for launch gaps to show (N x widest layer < 2^27);
@@ -77,7 +73,12 @@ enum {
  *                  in a fixed order afterwards (the paper's graphs have power-law degrees; a hub row
  *                  walked by one warp would outlast the rest of the launch).  Same sums up to fp32
  *                  rounding order.  0: the default, 256; a value above the longest row switches it off
- *  w_init          L host pointers to row-major C_{l-1} x C_l matrices (required)
+ *  w_init          L host pointers to row-major C_{l-1} x C_l matrices, or NULL: then every W_l is drawn
+ *                  Glorot-uniform, entry (i, j) of W_l = a (2 u - 1) with a = sqrt(6 / (C_{l-1} + C_l)) and
+ *                  u = (top 24 bits of splitmix64(seed + 2^32 l + i C_l + j)) / 2^24, where splitmix64(x) is
+ *                  the output function of that generator applied to the state x + 0x9E3779B97F4A7C15 (the
+ *                  paper does not say how W starts)
+ *  seed            seed of that draw; ignored when w_init is given
  *  device          CUDA device ordinal;  stream: a cudaStream_t owned by the caller (NULL = the
  *                  default stream) */
 typedef struct {
@@ -89,19 +90,18 @@ typedef struct {
   float loss_scale;
   int dual_mode;
   int tensor_cores;
-  int spmm_ring;
   int use_graph;
   int schedule;
   int long_row;
+  unsigned long long seed;
   const float* const* w_init;
   int device;
   void* stream;
 } gcn_admm_params;
 
 /* Fills *p with the defaults: nu = rho = 1e-3, tau0 = theta0 = 1, growth 2, shrink 0.5,
- * 40 trials, 30 FISTA iterations, loss_scale 1, dual_mode 0, tensor_cores 1, spmm_ring 0, use_graph 2, schedule 0, long_row 0, device 0,
- * stream NULL,
- * w_init NULL. */
+ * 40 trials, 30 FISTA iterations, loss_scale 1, dual_mode 0, tensor_cores 1, use_graph 2, schedule 0, long_row 0, seed 0, w_init NULL,
+ * device 0, stream NULL. */
 void gcn_admm_default_params(gcn_admm_params* p);
 
 /* Builds the problem of Algorithm 1 (its REQUIRE line) on the device.
@@ -149,7 +149,7 @@ const char* gcn_admm_last_error(const gcn_admm* h);
 
 /* ---- propagation alone (the product A~ X of Problem 1) ---------------------------------------
  * out = A~ x for an n x width matrix x in the original node order (host or device, both the same
- * kind; out may not alias x).  Uses the handle's graph only; the ADMM state is untouched. */
+ * kind; out may not alias x; width at most 2^24).  Uses the handle's graph only; the ADMM state is untouched. */
 int gcn_admm_propagate(gcn_admm* h, const float* x, int width, float* out);
 
 /* ---- the dense product alone (the contraction with W_l in Problem 1 and in every block update) ----
@@ -174,6 +174,8 @@ int gcn_admm_dense_product_tn(gcn_admm* h, const float* A, const float* B, float
  * (32 MiB of device memory on every GPU that loads the library, held until the process ends), and
  * calls neither cudaMalloc nor cudaFree nor any allocating routine.
  *  - x and out are DEVICE pointers to n x width floats, original node order; out may not alias x.
+ *  - its launches are counted by gcn_admm_launches but never timed by gcn_admm_profile (event
+ *    creation reserves memory), whether profiling is on or off.
  *  - limit: n * (width rounded up to a multiple of 4) <= 4,194,304; larger sizes are refused with
  *    GCN_ADMM_ERR_ARG and a message naming the limit.
  *  - the first call on a device looks up the device address of the array (one runtime query, no
@@ -211,8 +213,12 @@ int gcn_admm_index(gcn_admm* h, int which, int comm, const int** data, long long
  *  GCN_ADMM_ST_Z      layer 1..L   float  n x C_l
  *  GCN_ADMM_ST_U      layer ignored float n x C_L
  *  GCN_ADMM_ST_TAU    layer 1..L   double [1]
- *  GCN_ADMM_ST_THETA  layer 1..L-1 double [M] */
-enum { GCN_ADMM_ST_W = 0, GCN_ADMM_ST_Z, GCN_ADMM_ST_U, GCN_ADMM_ST_TAU, GCN_ADMM_ST_THETA };
+ *  GCN_ADMM_ST_THETA  layer 1..L-1 double [M]
+ *  GCN_ADMM_ST_PIPELINE_FLAG  layer ignored, int [1]: non-zero once a tensor-core product has given up one of
+ *                     its bounded waits.  The next call that synchronises (objective, decisions, dense
+ *                     products) then returns GCN_ADMM_ERR_CUDA once and clears the flag; the handle stays
+ *                     usable.  Writable so that this path can be exercised without a failing kernel. */
+enum { GCN_ADMM_ST_W = 0, GCN_ADMM_ST_Z, GCN_ADMM_ST_U, GCN_ADMM_ST_TAU, GCN_ADMM_ST_THETA, GCN_ADMM_ST_PIPELINE_FLAG };
 int gcn_admm_get_state(gcn_admm* h, int which, int layer, void* out);
 int gcn_admm_set_state(gcn_admm* h, int which, int layer, const void* in);
 

@@ -23,15 +23,15 @@ EXPORTS = [
 
 IX = dict(perm=0, inv_perm=1, comm_ptr=2, nbr=3, halo1=4, halo2=5, csr_row_ptr=6, csr_col=7,
           seg_row_ptr=8, seg_comm=9, seg_begin=10)
-ST_W, ST_Z, ST_U, ST_TAU, ST_THETA = range(5)
+ST_W, ST_Z, ST_U, ST_TAU, ST_THETA, ST_PIPELINE_FLAG = range(6)
 PHASE_W, PHASE_Z, PHASE_U = range(3)
 
 
 class Params(C.Structure):
     _fields_ = [("nu", C.c_float), ("rho", C.c_float), ("tau0", C.c_float), ("theta0", C.c_float),
                 ("bt_growth", C.c_float), ("bt_shrink", C.c_float), ("bt_max_trials", C.c_int),
-                ("fista_iters", C.c_int), ("loss_scale", C.c_float), ("dual_mode", C.c_int), ("tensor_cores", C.c_int), ("spmm_ring", C.c_int), ("use_graph", C.c_int), ("schedule", C.c_int), ("long_row", C.c_int),
-                ("w_init", C.POINTER(C.POINTER(C.c_float))), ("device", C.c_int), ("stream", C.c_void_p)]
+                ("fista_iters", C.c_int), ("loss_scale", C.c_float), ("dual_mode", C.c_int), ("tensor_cores", C.c_int), ("use_graph", C.c_int), ("schedule", C.c_int), ("long_row", C.c_int),
+                ("seed", C.c_ulonglong), ("w_init", C.POINTER(C.POINTER(C.c_float))), ("device", C.c_int), ("stream", C.c_void_p)]
 
 
 class GcnAdmmError(RuntimeError):
@@ -101,7 +101,7 @@ class GcnAdmm:
 
     def __init__(self, n, row_ptr, col_idx, X, y, train_mask, widths, n_comm, community, w_init, nu=1e-3, rho=1e-3,
                  tau0=1.0, theta0=1.0, bt_growth=2.0, bt_shrink=0.5, bt_max_trials=40, fista_iters=30,
-                 loss_scale=1.0, dual_mode=0, tensor_cores=1, spmm_ring=0, use_graph=2, schedule=0, long_row=0, device=0, stream=0):
+                 loss_scale=1.0, dual_mode=0, tensor_cores=1, use_graph=2, schedule=0, long_row=0, seed=0, device=0, stream=0):
         lib = load()
         self._lib = lib
         self._h = C.c_void_p()
@@ -112,14 +112,15 @@ class GcnAdmm:
         p.bt_growth, p.bt_shrink, p.bt_max_trials = bt_growth, bt_shrink, bt_max_trials
         p.fista_iters, p.loss_scale, p.dual_mode = fista_iters, loss_scale, dual_mode
         p.tensor_cores = int(tensor_cores)
-        p.spmm_ring = int(spmm_ring)
         p.use_graph = int(use_graph)
         p.schedule = int(schedule)
         p.long_row = int(long_row)
+        p.seed = int(seed)
         p.device, p.stream = device, stream or None
-        ws = [np.ascontiguousarray(w, dtype=np.float32) for w in w_init]
-        arr = (C.POINTER(C.c_float) * len(ws))(*[w.ctypes.data_as(C.POINTER(C.c_float)) for w in ws])
-        p.w_init = C.cast(arr, C.POINTER(C.POINTER(C.c_float)))
+        if w_init is not None:
+            ws = [np.ascontiguousarray(w, dtype=np.float32) for w in w_init]
+            arr = (C.POINTER(C.c_float) * len(ws))(*[w.ctypes.data_as(C.POINTER(C.c_float)) for w in ws])
+            p.w_init = C.cast(arr, C.POINTER(C.POINTER(C.c_float)))
         keep = []
 
         def host(a, dt):
@@ -214,6 +215,8 @@ class GcnAdmm:
             return (self.n, self.widths[-1]), np.float32
         if which == ST_TAU:
             return (1,), np.float64
+        if which == ST_PIPELINE_FLAG:
+            return (1,), np.int32
         return (self.n_comm,), np.float64
 
     def get_state(self, which, layer=0):

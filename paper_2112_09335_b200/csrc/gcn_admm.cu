@@ -28,11 +28,22 @@ namespace {
 constexpr int kLogPasses = 256;
 constexpr int kSmCount = 148;
 constexpr long long kImageMinRows = 16384;   // row count from which the weight operand is pre-split
+constexpr int kZBlockRows = 32;      // rows per block of the hidden-layer gradient's closing sweep
+constexpr int kCandZ = 2;           // theta candidates scored per sweep (tau: gk::kCand)
 constexpr int kDefaultLongRow = 256;   // stored entries one warp walks before a row is cut into items
 
 thread_local std::string g_create_error;
 
 inline int ldpad(int c) { return (c + 3) & ~3; }
+constexpr int kMaxWidth = 1 << 24;   // widest matrix an entry point accepts (keeps the padded width inside int)
+
+// Output function of the splitmix64 generator applied to the state x + 0x9E3779B97F4A7C15.
+inline unsigned long long splitmix64(unsigned long long x) {
+  unsigned long long z = x + 0x9E3779B97F4A7C15ULL;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+  return z ^ (z >> 31);
+}
 inline long long cdiv(long long a, long long b) { return (a + b - 1) / b; }
 
 struct Fail {
@@ -155,7 +166,11 @@ struct gcn_admm {
   float* part = nullptr;     // split partial sums of the transposed product
   size_t part_elems = 0;
   SearchCtl *ctl_w = nullptr, *ctl_z = nullptr;   // [L+1], [(L+1) * M]
-  double *sums_w = nullptr, *sums_z = nullptr, *acc_w = nullptr, *acc_z = nullptr, *obj = nullptr;
+  double *sums_w = nullptr, *sums_z = nullptr, *acc_z = nullptr, *obj = nullptr;
+  double* red_part = nullptr;               // per-block partial sums awaiting their fixed-order reduction
+  int2* d_zblocks = nullptr;                // row blocks of at most kZBlockRows rows, none crossing a community
+  int* d_comm_block_ptr = nullptr;          // [M+1] first row block of every community
+  int n_zblocks = 0;
   int *n_active = nullptr, *status = nullptr, *row_counter = nullptr, *d_pass = nullptr;
   cudaGraphExec_t pass_graph = nullptr;   // one pass of Algorithm 1, recorded once and replayed
   int *log_trial_w = nullptr, *log_trial_z = nullptr;
@@ -185,25 +200,6 @@ struct gcn_admm {
     char name[48];
     std::snprintf(name, sizeof name, "spmm@%d", ldx);
     Scope sc(this, name, 1, 4.0 * gi.nnz + 8.0 * n + 8.0 * (double)n * ldx, 2.0 * (double)gi.nnz * ldx);
-    if (p.spmm_ring && ld4 > 16 && ld4 <= 64) {
-      // rows of 17..64 float4: gathered rows in flight in a shared-memory ring (see k_spmm_ring)
-      CU(cudaMemsetAsync(row_counter, 0, sizeof(int), stream));
-      constexpr int kRingDepth = 16, kRingWarps = 4;
-#define RING_CASE(V)                                                                                          \
-  {                                                                                                           \
-    const size_t smem = (size_t)kRingWarps * kRingDepth * (V) * 32 * sizeof(float4);                          \
-    CU(cudaFuncSetAttribute(gk::k_spmm_ring<V, kRingDepth>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-    int occ = 1;                                                                                              \
-    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gk::k_spmm_ring<V, kRingDepth>, kRingWarps * 32, smem)); \
-    const unsigned grid = (unsigned)std::min<long long>(cdiv(n, (long long)gk::kGrab * kRingWarps), (long long)kSmCount * std::max(occ, 1)); \
-    gk::k_spmm_ring<V, kRingDepth><<<grid, kRingWarps * 32, smem, stream>>>(d_row_ptr, d_col, d_dinv, x4, o4, nn, ld4, row_counter); \
-  }
-      if (ld4 <= 32) RING_CASE(1)
-      else RING_CASE(2)
-#undef RING_CASE
-      CU(cudaGetLastError());
-      return;
-    }
     // 64-thread blocks: rows differ widely in length, small blocks keep the SMs evenly loaded.
     // Long rows go as items unless the operand is wider than the item buffer was sized for (a
     // caller's matrix wider than every layer): then they are walked whole, slower but the same sums.
@@ -237,21 +233,20 @@ struct gcn_admm {
   void gemm_nn(const float* A, int lda, const float* B, int ldb, const float* Bk, int ldbk, float* Cm, int ldc,
                long long Mr, int N, int K, const int* skip = nullptr) {
     char name[48];
-    if (p.tensor_cores && Bk != nullptr && K >= 8 && K <= 2048 && Mr >= 512 && (p.tensor_cores == 1 || p.tensor_cores == 3 || (N <= 256 && K <= 512))) {
+    if (p.tensor_cores && Bk != nullptr && K >= 8 && K <= 2048 && Mr >= 512) {
       std::snprintf(name, sizeof name, "gemm_tc@%dx%d", K, N);
       Scope sc(this, name, 1, 4.0 * ((double)Mr * (lda + ldc) + (double)K * ldb), 2.0 * (double)Mr * N * K);
       const int tiles = (int)cdiv(Mr, gtc::kBlockM);
-      if (p.tensor_cores == 1 || p.tensor_cores == 3) {   // role-split kernel: producers / MMA issue / epilogue overlap
       // With many row tiles the weight operand is split once into an image of the staged layout and
       // fetched by bulk copies; with few (launch-bound problems) the extra launch costs more than the
-      // producers' repeated work.  tensor_cores = 3 takes the image at every size.
+      // producers' repeated work.  tensor_cores = 2 takes the image at every size.
 #define TC_WS(NT)                                                                                              \
   {                                                                                                            \
     const size_t smem = gtc::WsCfg<NT>::kSmem;                                                                 \
     const int groups = (int)cdiv(N, NT);                                                                       \
     const size_t image_bytes = (size_t)groups * cdiv(K, gtc::kChunkK) * 2 * (NT) * gtc::kChunkK * 4;            \
     dim3 grid((unsigned)std::max(1, std::min(tiles, kSmCount / groups)), (unsigned)groups);                    \
-    if ((p.tensor_cores == 3 || Mr >= kImageMinRows) && image_bytes <= b_image_bytes) {                        \
+    if ((p.tensor_cores == 2 || Mr >= kImageMinRows) && image_bytes <= b_image_bytes) {                        \
       const long long work = (long long)groups * cdiv(K, gtc::kChunkK) * (NT) * 8;                             \
       gtc::k_split_b<<<(unsigned)std::min<long long>(cdiv(work, 256), 4 * kSmCount), 256, 0, stream>>>(Bk, ldbk, N, K, NT, b_image); \
       ++launches;                                                                                              \
@@ -262,53 +257,13 @@ struct gcn_admm {
       gtc::k_gemm_tc_ws<NT, false><<<grid, gtc::WsCfg<NT>::kThreads, smem, stream>>>(A, lda, Bk, ldbk, Cm, ldc, (int)Mr, N, K, skip, tc_error, nullptr); \
     }                                                                                                          \
   }
-        if (N <= 16) TC_WS(16)
-        else if (N <= 32) TC_WS(32)
-        else if (N <= 48) TC_WS(48)
-        else if (N <= 64) TC_WS(64)
-        else if (N <= 128) TC_WS(128)
-        else TC_WS(256)
+      if (N <= 16) TC_WS(16)
+      else if (N <= 32) TC_WS(32)
+      else if (N <= 48) TC_WS(48)
+      else if (N <= 64) TC_WS(64)
+      else if (N <= 128) TC_WS(128)
+      else TC_WS(256)
 #undef TC_WS
-        CU(cudaGetLastError());
-        return;
-      }
-      const size_t smem_cap = 227 * 1024;
-      // preferred form when one or two column groups suffice: the split weight operand stays in shared
-      // memory; with more groups the re-reads of A cost more than re-staging B (measured), so B is streamed
-#define TC_RES(NT)                                                                                             \
-  if (!launched && (N + (NT) - 1) / (NT) <= 2 && gtc::resident_smem_bytes<NT>(K) <= smem_cap) {                \
-    const size_t smem = gtc::resident_smem_bytes<NT>(K);                                                       \
-    const int groups = (int)cdiv(N, NT);                                                                       \
-    CU(cudaFuncSetAttribute(gtc::k_gemm_tc_resident<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-    dim3 grid((unsigned)std::max(1, std::min(tiles, kSmCount / groups)), (unsigned)groups);                    \
-    gtc::k_gemm_tc_resident<NT><<<grid, gtc::kThreads, smem, stream>>>(A, lda, Bk, ldbk, Cm, ldc, (int)Mr, N, K, skip, tc_error); \
-    launched = true;                                                                                           \
-  }
-      bool launched = false;
-      const int want = N <= 16 ? 16 : N <= 32 ? 32 : N <= 48 ? 48 : N <= 64 ? 64 : N <= 128 ? 128 : 256;
-      if (want >= 256) TC_RES(256)
-      if (want >= 128) TC_RES(128)
-      if (want >= 64) TC_RES(64)
-      if (want == 48) TC_RES(48)
-      if (want >= 32) TC_RES(32)
-      TC_RES(16)
-#undef TC_RES
-      if (launched) { CU(cudaGetLastError()); return; }
-#define TC_CASE(NT)                                                                                          \
-  {                                                                                                          \
-    const size_t smem = gtc::smem_bytes<NT>();                                                               \
-    CU(cudaFuncSetAttribute(gtc::k_gemm_tc<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));    \
-    const int per_sm = std::max(1, std::min(2, (int)((220 * 1024) / smem)));                                 \
-    const int grid = std::min(tiles, kSmCount * per_sm);                                                     \
-    gtc::k_gemm_tc<NT><<<grid, gtc::kThreads, smem, stream>>>(A, lda, Bk, ldbk, Cm, ldc, (int)Mr, N, K, skip, tc_error); \
-  }
-      if (N <= 16) TC_CASE(16)
-      else if (N <= 32) TC_CASE(32)
-      else if (N <= 48) TC_CASE(48)
-      else if (N <= 64) TC_CASE(64)
-      else if (N <= 128) TC_CASE(128)
-      else TC_CASE(256)
-#undef TC_CASE
       CU(cudaGetLastError());
       return;
     }
@@ -328,7 +283,7 @@ struct gcn_admm {
 
   // out[Ka x ldp] = A^T B over `rows` rows, through split partial sums reduced in a fixed order.
   // Whether P^T R runs on the tensor cores (that form can also build a hidden layer's R itself).
-  bool tn_on_tensor_cores(long long rows) const { return (p.tensor_cores == 1 || p.tensor_cores == 3) && rows >= 4096; }
+  bool tn_on_tensor_cores(long long rows) const { return p.tensor_cores != 0 && rows >= 4096; }
 
   // With `zres` (tensor-core form only) B holds pre-activations H and the operand is
   // h > 0 ? nu (h - z) : 0, formed while staging: the residual matrix is never stored.
@@ -414,7 +369,7 @@ struct gcn_admm {
     CU(cudaGetLastError());
   }
 
-  int n_passes() const { return (p.bt_max_trials + gk::kCand - 1) / gk::kCand; }
+  int n_passes(int cand) const { return (p.bt_max_trials + cand - 1) / cand; }
 
   long long z_per_pass() const { return (long long)std::max(L - 1, 0) * M; }
 
@@ -447,36 +402,38 @@ struct gcn_admm {
       Scope sc(this, "small", 3, 0.0, 0.0);
       gk::k_transpose_small<<<(unsigned)cdiv((long long)Kp * Cn, 256), 256, 0, stream>>>(grad, ldc, grad_t, ld[l - 1], Kp, Cn);
       gk::k_two_sumsq<<<1, 1024, 0, stream>>>(grad, W[l], (long long)Kp * ldc, sums_w);
-      gk::k_search_begin<<<1, 32, 0, stream>>>(ctl, 1, sums_w, 2, p.bt_shrink, p.bt_growth, acc_w, gk::kCand, nullptr, status);
+      gk::k_search_begin<<<1, 32, 0, stream>>>(ctl, sums_w, p.bt_shrink, p.bt_growth, status);
       CU(cudaGetLastError());
     }
     gemm_nn(P[l], ld[l - 1], grad, ldc, grad_t, ld[l - 1], B1, ldc, n, Cn, Kp, &ctl->done);   // D = P_l grad
     gk::DecideArgs a{};
     a.growth = p.bt_growth;
     a.max_trials = p.bt_max_trials;
+    a.cand = gk::kCand;
+    const int score_grid = grid_for(n4);   // every block of a scoring sweep leaves its sums in red_part
     if (l == L) {
       {
         Scope sc(this, "score_w_out", 1, 32.0 * n4, 0.0);
-        gk::k_score_w_out<<<grid_for(n4), 256, 0, stream>>>((const float4*)B1, (const float4*)B0, n4, ctl, acc_w);
+        gk::k_score_w_out<<<score_grid, 256, 0, stream>>>((const float4*)B1, (const float4*)B0, n4, ctl, red_part);
       }
       a.mode = 1;
       a.quad_coef = 0.5 * p.rho;
       a.last_pass = 1;
       Scope sc(this, "small", 1, 0.0, 0.0);
-      gk::k_search_decide<<<1, 32, 0, stream>>>(ctl, 1, acc_w, gk::kCand, nullptr, 0, a, nullptr, status);
+      gk::k_search_decide_w<<<1, 256, 0, stream>>>(ctl, red_part, score_grid, 2, a, status);
     } else {
       a.mode = 0;
       a.scale = 0.5 * p.nu;
-      const int passes = n_passes();
+      const int passes = n_passes(gk::kCand);
       for (int ps = 0; ps < passes; ++ps) {
         {   // passes after the first almost always find the search finished and return at once
           Scope sc(this, ps == 0 ? "score_w_hidden" : "score_w_hidden.retry", 1, ps == 0 ? 48.0 * n4 : 0.0, 0.0);
-          gk::k_score_w_hidden<<<grid_for(n4), 256, 0, stream>>>((const float4*)H[l], (const float4*)B1,
-                                                                 (const float4*)Z[l], n4, ctl, acc_w);
+          gk::k_score_w_hidden<<<score_grid, 256, 0, stream>>>((const float4*)H[l], (const float4*)B1,
+                                                               (const float4*)Z[l], n4, ctl, red_part);
         }
         a.last_pass = (ps == passes - 1);
         Scope sc(this, "small", 1, 0.0, 0.0);
-        gk::k_search_decide<<<1, 32, 0, stream>>>(ctl, 1, acc_w, gk::kCand, nullptr, 0, a, nullptr, status);
+        gk::k_search_decide_w<<<1, 256, 0, stream>>>(ctl, red_part, score_grid, gk::kCand, a, status);
       }
     }
     CU(cudaGetLastError());
@@ -498,26 +455,25 @@ struct gcn_admm {
     resid(l + 1, B0);                                                    // R'_{l+1}
     spmm(B0, B1, ldn);                                                   // S = A~ R'
     gemm_nn(B1, ldn, Wt[l + 1], ldl, W[l + 1], ldn, B2, ldl, n, C[l], C[l + 1]);        // S W_{l+1}^T
-    CU(cudaMemsetAsync(sums_z, 0, sizeof(double) * 3 * M, stream));
     CU(cudaMemsetAsync(n_active, 0, sizeof(int), stream));
-    const int rows_per_block = 32;
     {
-    Scope sc(this, "zgrad_finish", 1, 16.0 * 4.0 * (double)n * (ldl / 4), 0.0);
-    gk::k_zgrad_finish<<<(unsigned)cdiv(n, rows_per_block), 256, 0, stream>>>(
-        (float4*)B2, (const float4*)Z[l], (const float4*)H[l], ldl / 4, n, rows_per_block, d_row_comm, p.nu, sums_z);
+      Scope sc(this, "zgrad_finish", 1, 16.0 * 4.0 * (double)n * (ldl / 4), 0.0);
+      gk::k_zgrad_finish<<<(unsigned)n_zblocks, 256, 0, stream>>>((float4*)B2, (const float4*)Z[l], (const float4*)H[l],
+                                                                 ldl / 4, d_zblocks, p.nu, red_part);
     }
     const bool out = (l + 1 == L);
-    const int per = out ? 2 : gk::kCand;
+    const int per = out ? 2 : kCandZ;
     {
       Scope sc(this, "small", 1, 0.0, 0.0);
-      gk::k_search_begin<<<(unsigned)cdiv(M, 128), 128, 0, stream>>>(ctl, M, sums_z, 3, p.bt_shrink, p.bt_growth, acc_z,
-                                                                     per, n_active, status);
+      gk::k_search_begin_z<<<(unsigned)cdiv((long long)M * 32, 128), 128, 0, stream>>>(
+          ctl, M, red_part, d_comm_block_ptr, sums_z, p.bt_shrink, p.bt_growth, acc_z, per, n_active, status);
       CU(cudaGetLastError());
     }
     gemm_nn(B2, ldl, W[l + 1], ldn, Wt[l + 1], ldl, B1, ldn, n, C[l + 1], C[l]);         // T = G W_{l+1}
     gk::DecideArgs a{};
     a.growth = p.bt_growth;
     a.max_trials = p.bt_max_trials;
+    a.cand = kCandZ;
     a.own_nu = p.nu;
     const int ld4 = ldn / 4;
     const int warps = 8;
@@ -528,16 +484,16 @@ struct gcn_admm {
   {                                                                                                       \
     const size_t dynv = dyn + (size_t)warps * 2 * (V) * 32 * sizeof(float4);   /* per-warp copy of the row's a, b */ \
     if (dynv > 48 * 1024)                                                                                 \
-      CU(cudaFuncSetAttribute(gk::k_score_z<V, OUT, UNZ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dynv)); \
+      CU(cudaFuncSetAttribute(gk::k_score_z<V, OUT, UNZ, kCandZ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dynv)); \
     CU(cudaMemsetAsync(row_counter, 0, sizeof(int), stream));                                             \
     int occ = 1;                                                                                          \
-    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gk::k_score_z<V, OUT, UNZ>, warps * 32, dynv));     \
+    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gk::k_score_z<V, OUT, UNZ, kCandZ>, warps * 32, dynv));     \
     const unsigned grid = (unsigned)std::min<long long>(cdiv(n + n_items, warps), (long long)kSmCount * std::max(occ, 1)); \
-    gk::k_score_z<V, OUT, UNZ><<<grid, warps * 32, dynv, stream>>>(d_row_ptr, d_col, d_col_comm, d_dinv,       \
+    gk::k_score_z<V, OUT, UNZ, kCandZ><<<grid, warps * 32, dynv, stream>>>(d_row_ptr, d_col, d_col_comm, d_dinv,       \
         (const float4*)B1, (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0, ld4, (int)n, ctl, M, \
         acc_z, n_active, use_smem, row_counter, d_items, n_items, long_len, reinterpret_cast<float4*>(item_sums)); \
     if (n_split > 0) {                                                                                    \
-      gk::k_score_z_split<V, OUT><<<(unsigned)cdiv(n_split, warps), warps * 32, 0, stream>>>(d_split, n_split, d_dinv, \
+      gk::k_score_z_split<V, OUT, kCandZ><<<(unsigned)cdiv(n_split, warps), warps * 32, 0, stream>>>(d_split, n_split, d_dinv, \
           reinterpret_cast<const float4*>(item_sums), (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0, \
           ld4, ctl, acc_z, n_active);                                                                     \
       ++launches;                                                                                         \
@@ -577,7 +533,7 @@ struct gcn_admm {
               (const float4*)B1, (const float4*)B0, ld4, (int)n, ctl, M, acc_z, n_active, use_smem_h, row_counter, d_items,
               n_items, long_len, reinterpret_cast<float4*>(item_sums));
           if (n_split > 0) {
-            gk::k_score_z_split<1, true><<<(unsigned)cdiv(n_split, warps), warps * 32, 0, stream>>>(d_split, n_split, d_dinv,
+            gk::k_score_z_split<1, true, kCandZ><<<(unsigned)cdiv(n_split, warps), warps * 32, 0, stream>>>(d_split, n_split, d_dinv,
                 reinterpret_cast<const float4*>(item_sums), (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0,
                 ld4, ctl, acc_z, n_active);
             ++launches;
@@ -594,7 +550,7 @@ struct gcn_admm {
     } else {
       a.mode = 0;
       a.scale = 0.5 * p.nu;
-      const int passes = n_passes();
+      const int passes = n_passes(kCandZ);
       for (int ps = 0; ps < passes; ++ps) {
         {   // later passes touch only the segments of communities still searching
           Scope sc(this, ps == 0 ? zname : zretry.c_str(), 1, ps == 0 ? zbytes : 0.0,
@@ -822,7 +778,7 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
   if (h->C[n_layers] > 32 * gk::kMaxClassesPerLane)
     throw Fail{GCN_ADMM_ERR_WIDTHS, "more than 128 classes are not supported"};
   for (int l = 2; l <= n_layers; ++l)
-    if (h->ld[l] / 4 > 256) throw Fail{GCN_ADMM_ERR_WIDTHS, "layer widths above 1024 are supported for C_0 only"};
+    if (h->ld[l] / 4 > 256) throw Fail{GCN_ADMM_ERR_WIDTHS, "layer widths above 1024 are supported for C_0 and C_1 only"};
   for (int l = 1; l <= n_layers; ++l)   // the Z scoring addresses rows of an N x C_l matrix by 32-bit float4 offsets
     if (n * (long long)(h->ld[l] / 4) >= (1LL << 32))
       throw Fail{GCN_ADMM_ERR_WIDTHS, "n x layer width exceeds 2^34 elements"};
@@ -940,9 +896,23 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
   h->ctl_z = h->alloc<SearchCtl>((size_t)(L + 1) * n_comm);
   h->sums_w = h->alloc<double>(2);
   h->sums_z = h->alloc<double>((size_t)3 * n_comm);
-  h->acc_w = h->alloc<double>(gk::kCand);
   h->acc_z = h->alloc<double>((size_t)gk::kCand * n_comm);
   h->obj = h->alloc<double>(8);
+  {   // row blocks of the hidden-layer gradient's closing sweep, cut at community boundaries
+    std::vector<int2> zb;
+    std::vector<int> cbp((size_t)n_comm + 1, 0);
+    for (int m = 0; m < n_comm; ++m) {
+      cbp[m] = (int)zb.size();
+      for (int r = g.comm_ptr[m]; r < g.comm_ptr[m + 1]; r += kZBlockRows)
+        zb.push_back(make_int2(r, std::min(r + kZBlockRows, g.comm_ptr[m + 1])));
+    }
+    cbp[n_comm] = (int)zb.size();
+    h->n_zblocks = (int)zb.size();
+    h->d_zblocks = upload(h, zb);
+    h->d_comm_block_ptr = upload(h, cbp);
+  }
+  h->red_part = h->alloc<double>(std::max<size_t>({(size_t)kSmCount * 8 * gk::kCand, (size_t)h->n_zblocks * 3,
+                                                   (size_t)cdiv(n, 8) * 2}));
   h->n_active = h->alloc<int>(1);
   h->status = h->alloc<int>(1);
   h->row_counter = h->alloc<int>(1);
@@ -993,7 +963,18 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
     cudaFree(x_pad);
   }
 
-  for (int l = 1; l <= L; ++l) h->upload_weight(l, p.w_init[l - 1]);
+  for (int l = 1; l <= L; ++l) {
+    if (p.w_init != nullptr) { h->upload_weight(l, p.w_init[l - 1]); continue; }
+    // no weights given: Glorot-uniform from a counter-based generator (see the header for the definition)
+    const int r = h->C[l - 1], c = h->C[l];
+    std::vector<float> w((size_t)r * c);
+    const double a = std::sqrt(6.0 / ((double)r + (double)c));
+    for (size_t e = 0; e < w.size(); ++e) {
+      const double u = (double)(splitmix64(p.seed + ((unsigned long long)l << 32) + e) >> 40) / 16777216.0;
+      w[e] = (float)(a * (2.0 * u - 1.0));
+    }
+    h->upload_weight(l, w.data());
+  }
   // forward pass of Problem 1 with the same kernels that later recompute H_l, so that the
   // initial residuals are exactly zero
   for (int l = 1; l <= L; ++l) {
@@ -1027,10 +1008,10 @@ void gcn_admm_default_params(gcn_admm_params* p) {
   p->loss_scale = 1.f;
   p->dual_mode = 0;
   p->tensor_cores = 1;
-  p->spmm_ring = 0;
   p->use_graph = 2;
   p->schedule = 0;
   p->long_row = 0;
+  p->seed = 0;
   p->w_init = nullptr;
   p->device = 0;
   p->stream = nullptr;
@@ -1047,8 +1028,7 @@ int gcn_admm_create(gcn_admm** out, long long n, const long long* row_ptr, const
   if (n < 1 || n > 2147483647LL / 2 || n_comm < 1) { g_create_error = "n and n_comm must be positive"; return GCN_ADMM_ERR_ARG; }
   if (n_comm > 65535) { g_create_error = "more than 65535 communities are not supported"; return GCN_ADMM_ERR_COMMUNITY; }
   if (n_layers < 1 || n_layers > 64) { g_create_error = "n_layers must be 1..64"; return GCN_ADMM_ERR_WIDTHS; }
-  if (!p->w_init) { g_create_error = "w_init is required"; return GCN_ADMM_ERR_ARG; }
-  for (int l = 0; l < n_layers; ++l)
+  for (int l = 0; p->w_init && l < n_layers; ++l)
     if (!p->w_init[l]) { g_create_error = "w_init holds a NULL pointer"; return GCN_ADMM_ERR_ARG; }
   if (!(p->nu > 0.f) || !(p->rho > 0.f) || !(p->bt_growth > 1.f) || !(p->bt_shrink > 0.f) || p->bt_max_trials < 1 ||
       p->bt_max_trials > 64 || p->fista_iters < 0 || p->schedule < 0 || p->schedule > 1 || p->long_row < 0 || !(p->tau0 > 0.f) || !(p->theta0 > 0.f) || !(p->loss_scale > 0.f)) {
@@ -1168,23 +1148,36 @@ int gcn_admm_objective(gcn_admm* h, double out[6]) {
     const int L = h->L;
     cudaStream_t s = h->stream;
     CU(cudaMemsetAsync(h->obj, 0, 8 * sizeof(double), s));
+    // every sum: per-block partials, then one block adds them in a fixed order
     for (int l = 1; l < L; ++l) {
       const long long n4 = h->n * h->ld[l] / 4;
-      gcn_admm::Scope sc(h, "objective_sums", 1, 32.0 * n4, 0.0);
-      gk::k_sum_hidden_penalty<<<h->grid_for(n4), 256, 0, s>>>((const float4*)h->Z[l], (const float4*)h->H[l], n4, h->obj + 2);
+      gcn_admm::Scope sc(h, "objective_sums", 2, 32.0 * n4, 0.0);
+      const int grid = h->grid_for(n4);
+      gk::k_sum_hidden_penalty<<<grid, 256, 0, s>>>((const float4*)h->Z[l], (const float4*)h->H[l], n4, h->red_part);
+      gk::k_add_partials<<<1, 256, 0, s>>>(h->red_part, grid, 1, h->obj + 2);
     }
     const long long n4 = h->n * h->ld[L] / 4;
-    gcn_admm::Scope sc_obj(h, "objective_sums", 3, 48.0 * n4, 0.0);
-    gk::k_sum_constraint<<<h->grid_for(n4), 256, 0, s>>>((const float4*)h->Z[L], (const float4*)h->H[L],
-                                                        (const float4*)h->U, n4, h->obj + 3);
     const int warps = 8;
-    gk::k_row_loss_argmax<<<(unsigned)cdiv(h->n, warps), warps * 32, 0, s>>>(h->Z[L], nullptr, h->ld[L], h->C[L], (int)h->n,
-                                                                             h->d_y, h->d_train, nullptr, h->obj);
-    CU(cudaGetLastError());
+    const int row_blocks = (int)cdiv(h->n, warps);
+    {
+      gcn_admm::Scope sc_obj(h, "objective_sums", 4, 48.0 * n4, 0.0);
+      const int grid = h->grid_for(n4);
+      gk::k_sum_constraint<<<grid, 256, 0, s>>>((const float4*)h->Z[L], (const float4*)h->H[L], (const float4*)h->U, n4,
+                                                h->red_part);
+      gk::k_add_partials<<<1, 256, 0, s>>>(h->red_part, grid, 2, h->obj + 3);
+      gk::k_row_loss_argmax<<<row_blocks, warps * 32, 0, s>>>(h->Z[L], nullptr, h->ld[L], h->C[L], (int)h->n, h->d_y,
+                                                              h->d_train, nullptr, h->red_part);
+      gk::k_add_partials<<<1, 256, 0, s>>>(h->red_part, row_blocks, 2, h->obj);      // obj[0] = cross-entropy sum
+      CU(cudaGetLastError());
+    }
     h->forward_logits();
-    gk::k_row_loss_argmax<<<(unsigned)cdiv(h->n, warps), warps * 32, 0, s>>>(nullptr, h->B0, h->ld[L], h->C[L], (int)h->n,
-                                                                             h->d_y, h->d_train, nullptr, h->obj);
-    CU(cudaGetLastError());
+    {
+      gcn_admm::Scope sc_obj(h, "objective_sums", 2, 4.0 * (double)h->n * h->ld[L], 0.0);
+      gk::k_row_loss_argmax<<<row_blocks, warps * 32, 0, s>>>(nullptr, h->B0, h->ld[L], h->C[L], (int)h->n, h->d_y,
+                                                              h->d_train, nullptr, h->red_part);
+      gk::k_add_partials<<<1, 256, 0, s>>>(h->red_part, row_blocks, 2, h->obj + 5);  // obj[6] = correct training rows
+      CU(cudaGetLastError());
+    }
     double v[8];
     CU(cudaMemcpyAsync(v, h->obj, 8 * sizeof(double), cudaMemcpyDeviceToHost, s));
     CU(cudaStreamSynchronize(s));
@@ -1194,7 +1187,7 @@ int gcn_admm_objective(gcn_admm* h, double out[6]) {
     const double rr = 0.5 * h->p.rho * v[4];
     out[0] = R + pen + ur + rr;
     out[1] = R; out[2] = pen; out[3] = ur; out[4] = rr;
-    out[5] = h->n_train > 0 ? v[1] / h->n_train : 0.0;
+    out[5] = h->n_train > 0 ? v[6] / h->n_train : 0.0;
     h->check_status();
   });
 }
@@ -1210,10 +1203,9 @@ int gcn_admm_predict(gcn_admm* h, float* logits, int* labels) {
     if (labels) {
       const int warps = 8;
       int* d_lab = reinterpret_cast<int*>(h->B1);
-      CU(cudaMemsetAsync(h->obj, 0, 8 * sizeof(double), h->stream));
       gcn_admm::Scope sc(h, "row_argmax", 1, 4.0 * (double)h->n * h->ld[L], 0.0);
       gk::k_row_loss_argmax<<<(unsigned)cdiv(h->n, warps), warps * 32, 0, h->stream>>>(
-          nullptr, h->B0, h->ld[L], h->C[L], (int)h->n, h->d_y, h->d_train, d_lab, h->obj);
+          nullptr, h->B0, h->ld[L], h->C[L], (int)h->n, h->d_y, h->d_train, d_lab, h->red_part);
       CU(cudaGetLastError());
       std::vector<int> lab(h->n);
       CU(cudaMemcpyAsync(lab.data(), d_lab, sizeof(int) * h->n, cudaMemcpyDeviceToHost, h->stream));
@@ -1227,7 +1219,7 @@ int gcn_admm_predict(gcn_admm* h, float* logits, int* labels) {
 
 int gcn_admm_propagate(gcn_admm* h, const float* x, int width, float* out) {
   return guarded(h, [&] {
-    if (!x || !out || width < 1) throw Fail{GCN_ADMM_ERR_ARG, "bad argument"};
+    if (!x || !out || width < 1 || width > kMaxWidth) throw Fail{GCN_ADMM_ERR_ARG, "bad argument"};
     const int ldw = ldpad(width);
     const size_t rows = (size_t)h->n;
     const bool dev_in = is_device_pointer(x), dev_out = is_device_pointer(out);
@@ -1351,7 +1343,7 @@ float* static_scratch(int device) {
 
 int gcn_admm_propagate_static(gcn_admm* h, const float* x, int width, float* out) {
   return guarded(h, [&] {
-    if (!x || !out || width < 1) throw Fail{GCN_ADMM_ERR_ARG, "bad argument"};
+    if (!x || !out || width < 1 || width > kMaxWidth) throw Fail{GCN_ADMM_ERR_ARG, "bad argument"};
     const int ldw = ldpad(width);
     if ((long long)h->n * ldw > kStaticHalf)
       throw Fail{GCN_ADMM_ERR_ARG, "n * padded width exceeds the static scratch of 4194304 floats per staging matrix"};
@@ -1359,6 +1351,11 @@ int gcn_admm_propagate_static(gcn_admm* h, const float* x, int width, float* out
       throw Fail{GCN_ADMM_ERR_ARG, "x and out must be device pointers"};
     float* a = static_scratch(h->p.device);
     float* b = a + kStaticHalf;
+    struct Untimed {   // event creation reserves memory: launches here are counted, never timed
+      gcn_admm* h; bool saved;
+      explicit Untimed(gcn_admm* h_) : h(h_), saved(h_->profiling) { h->profiling = false; }
+      ~Untimed() { h->profiling = saved; }
+    } untimed(h);
     {
       gcn_admm::Scope sc(h, "permute_rows", 1, 8.0 * (double)h->n * width, 0.0);
       gk::k_permute_rows<<<h->grid_for(h->n * ldw), 256, 0, h->stream>>>(x, a, h->d_perm, h->n, width, ldw, 1);
@@ -1432,6 +1429,9 @@ int gcn_admm_get_state(gcn_admm* h, int which, int layer, void* out) {
                          h->stream));
       CU(cudaStreamSynchronize(h->stream));
       for (int m = 0; m < h->M; ++m) static_cast<double*>(out)[m] = c[m].t_prev;
+    } else if (which == GCN_ADMM_ST_PIPELINE_FLAG) {
+      CU(cudaMemcpyAsync(out, h->tc_error, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+      CU(cudaStreamSynchronize(h->stream));
     } else {
       throw Fail{GCN_ADMM_ERR_ARG, "unknown state selector"};
     }
@@ -1469,6 +1469,9 @@ int gcn_admm_set_state(gcn_admm* h, int which, int layer, const void* in) {
         CU(cudaMemcpyAsync(&h->ctl_z[(size_t)layer * h->M + m].t_prev, t + m, sizeof(double), cudaMemcpyHostToDevice,
                            h->stream));
       }
+      CU(cudaStreamSynchronize(h->stream));
+    } else if (which == GCN_ADMM_ST_PIPELINE_FLAG) {
+      CU(cudaMemcpyAsync(h->tc_error, in, sizeof(int), cudaMemcpyHostToDevice, h->stream));
       CU(cudaStreamSynchronize(h->stream));
     } else {
       throw Fail{GCN_ADMM_ERR_ARG, "unknown state selector"};

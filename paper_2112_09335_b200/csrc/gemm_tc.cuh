@@ -20,12 +20,11 @@
 // row-major (the library keeps W_l and its transpose, so one of them always has this form).
 // One CTA owns 128 rows of A and all N <= 256 columns; the accumulators (128 lanes x 2 NT columns of
 // fp32) live in tensor memory.  K is walked in chunks of 32 floats = one 128-byte swizzle row.
-// All 256 threads stage the chunk: 128-bit loads from global memory, split into hi/lo, stores into
-// shared memory in the canonical K-major 128-byte-swizzled operand layout; then one thread issues
-// the twelve MMAs (3 products x 4 steps of K = 8) and commits them to the mbarrier that frees the
-// stage.  Loads of the next chunk are in flight while the current MMAs run.  Every wait on an
-// mbarrier is bounded; a wait that runs out raises `*error_flag` and the CTA leaves through the
-// normal exit (tensor memory released).
+// Producer warps stage each chunk (128-bit loads from global memory, split into hi/lo, stores into shared
+// memory in the canonical K-major 128-byte-swizzled operand layout); one thread issues the twelve MMAs
+// (3 products x 4 steps of K = 8) and commits them to the mbarrier that frees the stage; epilogue warps
+// drain finished accumulators (see k_gemm_tc_ws).  Every wait on an mbarrier is bounded; a wait that runs
+// out raises `*error_flag` and the CTA leaves through the normal exit (tensor memory released).
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -34,8 +33,6 @@ namespace gtc {
 
 constexpr int kBlockM = 128;
 constexpr int kChunkK = 32;                 // floats per K chunk (128 bytes)
-constexpr int kThreads = 256;
-constexpr int kStages = 2;
 constexpr int kATileBytes = kBlockM * kChunkK * 4;     // 16 KiB, one of hi / lo
 constexpr uint32_t kSpinLimit = 4u << 20;
 
@@ -44,22 +41,6 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-// Bounded wait for the phase with the given parity; false when the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    if (ok) return true;
-  }
-  return false;
-}
-
 // Shared-memory operand descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t operand_desc(uint32_t smem_addr) {
   const uint32_t lo = ((smem_addr >> 4) & 0x3fffu) | (1u << 16);          // start address, LBO field = 1
@@ -103,388 +84,8 @@ __device__ __forceinline__ void split_tf32(float x, float& hi, float& lo) {
 // Swizzled byte offset of the 16-byte unit `c16` (0..7) of row `r` inside a K-major operand tile.
 __device__ __forceinline__ uint32_t swz(int r, int c16) { return (uint32_t)r * 128u + (uint32_t)((c16 ^ (r & 7)) << 4); }
 
-// Dynamic shared memory: [stage][A_hi | A_lo | B_hi | B_lo], each tile 1024-byte aligned.
-template <int NT>   // NT: accumulator columns = N rounded up to 16 (16..256)
-__global__ void __launch_bounds__(kThreads, 1)
-k_gemm_tc(const float* __restrict__ A, int lda, const float* __restrict__ Bk, int ldbk, float* __restrict__ C, int ldc,
-          int M, int N, int K, const int* __restrict__ skip, int* __restrict__ error_flag) {
-  constexpr int kBTileBytes = NT * kChunkK * 4;
-  constexpr int kStageBytes = 2 * kATileBytes + 2 * kBTileBytes;
-  constexpr int ROWS_PER_PASS = kThreads / 8;                      // 32 rows per pass of the loaders
-  constexpr int B_PASSES = (NT + ROWS_PER_PASS - 1) / ROWS_PER_PASS;
-  constexpr int A_PASSES = kBlockM / ROWS_PER_PASS;                // 4
-  constexpr uint32_t TMEM_COLS = 2 * NT <= 32 ? 32 : 2 * NT <= 64 ? 64 : 2 * NT <= 128 ? 128 : 2 * NT <= 256 ? 256 : 512;
-  if (skip != nullptr && *skip) return;
-
-  extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[kStages + 1];
-  __shared__ uint32_t tmem_base_slot;
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const uint32_t smem_base = smem_u32(smem);
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const uint32_t bar_empty0 = smem_u32(&bars[0]);
-  const uint32_t bar_acc = smem_u32(&bars[kStages]);
-
-  if (tid == 0) {
-    for (int s = 0; s <= kStages; ++s) mbar_init(smem_u32(&bars[s]), 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem_base = tmem_base_slot;
-  const uint32_t idesc = instr_desc(NT);
-
-  const int kc_count = (K + kChunkK - 1) / kChunkK;
-  const int n_tiles = (M + kBlockM - 1) / kBlockM;
-  const int ld_c16 = tid & 7;          // which 16-byte unit of the 128-byte row this thread stages
-  const int ld_row = tid >> 3;         // 0..31, plus 32 per pass
-
-  float4 ra[A_PASSES], rb[B_PASSES];
-  auto load_chunk = [&](int tile, int kc) {
-    const int k0 = kc * kChunkK + ld_c16 * 4;
-    const long long row0 = (long long)tile * kBlockM;
-#pragma unroll
-    for (int i = 0; i < A_PASSES; ++i) {
-      const long long r = row0 + ld_row + 32 * i;
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (r < M && k0 < K) {
-        v = *reinterpret_cast<const float4*>(A + r * lda + k0);   // lda % 4 == 0 and k0 % 4 == 0
-      }
-      ra[i] = v;
-    }
-#pragma unroll
-    for (int i = 0; i < B_PASSES; ++i) {
-      const int nrow = ld_row + 32 * i;
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (nrow < N && k0 < K) {
-        v = *reinterpret_cast<const float4*>(Bk + (long long)nrow * ldbk + k0);
-      }
-      rb[i] = v;
-    }
-  };
-  auto store_chunk = [&](int stage) {
-    uint8_t* st = smem + (size_t)stage * kStageBytes;
-#pragma unroll
-    for (int i = 0; i < A_PASSES; ++i) {
-      float4 h, l;
-      split_tf32(ra[i].x, h.x, l.x); split_tf32(ra[i].y, h.y, l.y);
-      split_tf32(ra[i].z, h.z, l.z); split_tf32(ra[i].w, h.w, l.w);
-      const uint32_t off = swz(ld_row + 32 * i, ld_c16);
-      *reinterpret_cast<float4*>(st + off) = h;
-      *reinterpret_cast<float4*>(st + kATileBytes + off) = l;
-    }
-#pragma unroll
-    for (int i = 0; i < B_PASSES; ++i) {
-      const int nrow = ld_row + 32 * i;
-      if (nrow < NT) {
-        float4 h, l;
-        split_tf32(rb[i].x, h.x, l.x); split_tf32(rb[i].y, h.y, l.y);
-        split_tf32(rb[i].z, h.z, l.z); split_tf32(rb[i].w, h.w, l.w);
-        const uint32_t off = swz(nrow, ld_c16);
-        *reinterpret_cast<float4*>(st + 2 * kATileBytes + off) = h;
-        *reinterpret_cast<float4*>(st + 2 * kATileBytes + kBTileBytes + off) = l;
-      }
-    }
-  };
-
-  uint32_t stage_uses[kStages];
-#pragma unroll
-  for (int s = 0; s < kStages; ++s) stage_uses[s] = 0;
-  uint32_t it = 0, tiles_done = 0;
-  bool failed = false;
-
-  int tile = blockIdx.x;
-  if (tile < n_tiles) load_chunk(tile, 0);
-  for (; tile < n_tiles && !failed; tile += gridDim.x) {
-    for (int kc = 0; kc < kc_count; ++kc, ++it) {
-      const int stage = it % kStages;
-      // the MMAs that last read this stage must have completed before it is overwritten
-      bool ok = true;
-      if (stage_uses[stage] > 0) ok = mbar_wait(bar_empty0 + 8 * stage, (stage_uses[stage] - 1) & 1);
-      if (__syncthreads_or(!ok)) { failed = true; break; }
-      store_chunk(stage);
-      ++stage_uses[stage];
-      // next chunk (of this tile or of the CTA's next tile) on its way while the MMAs run
-      if (kc + 1 < kc_count) load_chunk(tile, kc + 1);
-      else if (tile + (int)gridDim.x < n_tiles) load_chunk(tile + gridDim.x, 0);
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> async-proxy reads
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      __syncthreads();
-      if (tid == 0) {
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t a_hi = smem_base + stage * kStageBytes, a_lo = a_hi + kATileBytes;
-        const uint32_t b_hi = a_hi + 2 * kATileBytes, b_lo = b_hi + kBTileBytes;
-#pragma unroll
-        for (int ks = 0; ks < kChunkK / 8; ++ks) {
-          const uint32_t o = ks * 32;    // 8 floats further along K inside the swizzled row
-          const uint32_t first = (kc > 0 || ks > 0) ? 1u : 0u;
-          mma_tf32(tmem_base + NT, operand_desc(a_lo + o), operand_desc(b_hi + o), idesc, first);   // corrections
-          mma_tf32(tmem_base + NT, operand_desc(a_hi + o), operand_desc(b_lo + o), idesc, 1u);
-          mma_tf32(tmem_base, operand_desc(a_hi + o), operand_desc(b_hi + o), idesc, first);        // main product
-        }
-        mma_commit(bar_empty0 + 8 * stage);
-        if (kc + 1 == kc_count) mma_commit(bar_acc);
-      }
-    }
-    if (failed) break;
-    // epilogue: accumulators (tensor memory) -> registers -> C
-    {
-      const bool ok = mbar_wait(bar_acc, tiles_done & 1);
-      if (__syncthreads_or(!ok)) { failed = true; break; }
-      ++tiles_done;
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int quarter = warp & 3;                       // tensor-memory lanes 32*quarter .. +31
-      const long long row = (long long)tile * kBlockM + quarter * 32 + lane;
-      for (int cchunk = (warp >> 2); cchunk < NT / 16; cchunk += 2) {
-        uint32_t v[16], w[16];
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(cchunk * 16);
-        GTC_TMEM_LD16(v, taddr);
-        GTC_TMEM_LD16(w, taddr + (uint32_t)NT);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (row < M) {
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const int col = cchunk * 16 + q * 4;
-            if (col < ldc)   // ldc % 4 == 0; columns N..ldc-1 receive the zeros of B's padding rows
-              *reinterpret_cast<float4*>(C + row * ldc + col) =
-                  make_float4(__uint_as_float(v[q * 4]) + __uint_as_float(w[q * 4]),
-                              __uint_as_float(v[q * 4 + 1]) + __uint_as_float(w[q * 4 + 1]),
-                              __uint_as_float(v[q * 4 + 2]) + __uint_as_float(w[q * 4 + 2]),
-                              __uint_as_float(v[q * 4 + 3]) + __uint_as_float(w[q * 4 + 3]));
-          }
-        }
-      }
-      // the next tile's first MMA overwrites the accumulators: every warp must be done reading them
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      __syncthreads();
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    }
-  }
-  if (failed && tid == 0) atomicExch(error_flag, 1);
-  // drain: the last commits must have landed before tensor memory is released
-  if (!failed) {
-    for (int s = 0; s < kStages; ++s)
-      if (stage_uses[s] > 0) mbar_wait(bar_empty0 + 8 * s, (stage_uses[s] - 1) & 1);
-  }
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
-  if (warp == 0) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
-  }
-}
-
 // ------------------------------------------------------------------------------------------------
-// Second form, used whenever the split weight operand fits in shared memory next to the pipeline:
-// B stays resident.  The grid is (row workers) x (column groups of NT columns); a CTA splits its
-// NT x K slice of B into hi/lo once, keeps it for all of its row tiles, and streams only A:
-// three stages, each filled two chunks ahead with 16-byte cp.async copies (zero-filled past the
-// matrix edge), split in place by the thread that copied them (raw -> hi in the same slot, lo in
-// the neighbouring one), then consumed by the twelve MMAs of the chunk.
-// ------------------------------------------------------------------------------------------------
-constexpr int kAStages = 3;
-
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_all_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
-
-template <int NT>
-__global__ void __launch_bounds__(kThreads, 1)
-k_gemm_tc_resident(const float* __restrict__ A, int lda, const float* __restrict__ Bk, int ldbk, float* __restrict__ C,
-                   int ldc, int M, int N, int K, const int* __restrict__ skip, int* __restrict__ error_flag) {
-  constexpr int kBTileBytes = NT * kChunkK * 4;          // one of hi / lo, one chunk
-  constexpr int kAStageBytes = 2 * kATileBytes;
-  constexpr int ROWS_PER_PASS = kThreads / 8;
-  constexpr int B_PASSES = (NT + ROWS_PER_PASS - 1) / ROWS_PER_PASS;
-  constexpr int A_PASSES = kBlockM / ROWS_PER_PASS;
-  constexpr uint32_t TMEM_COLS = 2 * NT <= 32 ? 32 : 2 * NT <= 64 ? 64 : 2 * NT <= 128 ? 128 : 2 * NT <= 256 ? 256 : 512;
-  if (skip != nullptr && *skip) return;
-
-  extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[kAStages + 1];
-  __shared__ uint32_t tmem_base_slot;
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int kc_count = (K + kChunkK - 1) / kChunkK;
-  uint8_t* a_stages = smem;                                        // kAStages x [A_hi | A_lo]
-  uint8_t* b_res = smem + (size_t)kAStages * kAStageBytes;         // kc_count x [B_hi | B_lo]
-  const uint32_t a_base = smem_u32(a_stages), b_base = smem_u32(b_res);
-  const uint32_t bar_empty0 = smem_u32(&bars[0]);
-  const uint32_t bar_acc = smem_u32(&bars[kAStages]);
-
-  if (tid == 0) {
-    for (int s = 0; s <= kAStages; ++s) mbar_init(smem_u32(&bars[s]), 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-
-  const int ld_c16 = tid & 7, ld_row = tid >> 3;
-  const int n0 = blockIdx.y * NT;                 // first output column of this CTA
-  const int n_loc = min(NT, N - n0);
-  // resident B: rows n0 .. n0+n_loc-1 of Bk, all K, split into hi / lo
-  for (int kc = 0; kc < kc_count; ++kc) {
-    const int k0 = kc * kChunkK + ld_c16 * 4;
-#pragma unroll
-    for (int i = 0; i < B_PASSES; ++i) {
-      const int nrow = ld_row + 32 * i;
-      if (nrow < NT) {
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (nrow < n_loc && k0 < K) {
-          v = *reinterpret_cast<const float4*>(Bk + (long long)(n0 + nrow) * ldbk + k0);
-        }
-        float4 h, l;
-        split_tf32(v.x, h.x, l.x); split_tf32(v.y, h.y, l.y); split_tf32(v.z, h.z, l.z); split_tf32(v.w, h.w, l.w);
-        uint8_t* dst = b_res + (size_t)kc * 2 * kBTileBytes + swz(nrow, ld_c16);
-        *reinterpret_cast<float4*>(dst) = h;
-        *reinterpret_cast<float4*>(dst + kBTileBytes) = l;
-      }
-    }
-  }
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem_base = tmem_base_slot;
-  const uint32_t idesc = instr_desc(NT);
-
-  const int n_tiles = (M + kBlockM - 1) / kBlockM;
-  const int my_tiles = (n_tiles > (int)blockIdx.x) ? (n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
-  const int total = my_tiles * kc_count;
-
-  // copies of chunk j = (tile, kc) into the hi slot of stage j % kAStages, raw fp32
-  auto issue_load = [&](int j) {
-    if (j < total) {
-      const int tile = blockIdx.x + (j / kc_count) * gridDim.x, kc = j % kc_count;
-      const int k0 = kc * kChunkK + ld_c16 * 4;
-      const int kbytes = max(0, min(16, 4 * (K - k0)));
-      const uint32_t st = a_base + (j % kAStages) * kAStageBytes;
-#pragma unroll
-      for (int i = 0; i < A_PASSES; ++i) {
-        const int rr = ld_row + 32 * i;
-        const long long r = (long long)tile * kBlockM + rr;
-        const bool in = r < M && kbytes > 0;
-        cp_async16(st + swz(rr, ld_c16), in ? (const void*)(A + r * lda + k0) : (const void*)A, in ? kbytes : 0);
-      }
-    }
-    cp_async_commit();
-  };
-
-  uint32_t stage_uses[kAStages];
-#pragma unroll
-  for (int s = 0; s < kAStages; ++s) stage_uses[s] = 0;
-  uint32_t tiles_done = 0;
-  bool failed = false, bad = false;   // bad: this thread saw a wait run out; failed: the whole CTA agreed to stop
-  issue_load(0);
-  issue_load(1);
-  for (int j = 0; j < total; ++j) {
-    const int stage = j % kAStages;
-    const int kc = j % kc_count;
-    const int tile = blockIdx.x + (j / kc_count) * gridDim.x;
-    cp_async_wait_all_but_one();                   // this thread's copies of chunk j have landed
-    {
-      uint8_t* st = a_stages + (size_t)stage * kAStageBytes;
-#pragma unroll
-      for (int i = 0; i < A_PASSES; ++i) {
-        const uint32_t off = swz(ld_row + 32 * i, ld_c16);
-        const float4 v = *reinterpret_cast<const float4*>(st + off);
-        float4 h, l;
-        split_tf32(v.x, h.x, l.x); split_tf32(v.y, h.y, l.y); split_tf32(v.z, h.z, l.z); split_tf32(v.w, h.w, l.w);
-        *reinterpret_cast<float4*>(st + off) = h;
-        *reinterpret_cast<float4*>(st + kATileBytes + off) = l;
-      }
-    }
-    ++stage_uses[stage];
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    if (__syncthreads_or(bad)) { failed = true; break; }
-    if (tid == 0) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t a_hi = a_base + stage * kAStageBytes, a_lo = a_hi + kATileBytes;
-      const uint32_t b_hi = b_base + kc * 2 * kBTileBytes, b_lo = b_hi + kBTileBytes;
-#pragma unroll
-      for (int ks = 0; ks < kChunkK / 8; ++ks) {
-        const uint32_t o = ks * 32;
-        const uint32_t first = (kc > 0 || ks > 0) ? 1u : 0u;
-        mma_tf32(tmem_base + NT, operand_desc(a_lo + o), operand_desc(b_hi + o), idesc, first);   // corrections
-        mma_tf32(tmem_base + NT, operand_desc(a_hi + o), operand_desc(b_lo + o), idesc, 1u);
-        mma_tf32(tmem_base, operand_desc(a_hi + o), operand_desc(b_hi + o), idesc, first);        // main product
-      }
-      mma_commit(bar_empty0 + 8 * stage);
-      if (kc + 1 == kc_count) mma_commit(bar_acc);
-    }
-    // refill the stage that chunk j-1 used (its MMAs were issued one iteration ago) with chunk j+2
-    {
-      const int prev = (j + 2) % kAStages;
-      if (j + 2 < total && stage_uses[prev] > 0 && !mbar_wait(bar_empty0 + 8 * prev, (stage_uses[prev] - 1) & 1))
-        bad = true;
-      issue_load(bad ? total : j + 2);
-    }
-    if (kc + 1 == kc_count) {
-      // epilogue: accumulators (tensor memory) -> registers -> C
-      const bool ok = mbar_wait(bar_acc, tiles_done & 1);
-      if (__syncthreads_or(!ok || bad)) { failed = true; break; }
-      ++tiles_done;
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int quarter = warp & 3;
-      const long long row = (long long)tile * kBlockM + quarter * 32 + lane;
-      for (int cchunk = (warp >> 2); cchunk < NT / 16; cchunk += 2) {
-        uint32_t v[16], w[16];
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(cchunk * 16);
-        GTC_TMEM_LD16(v, taddr);
-        GTC_TMEM_LD16(w, taddr + (uint32_t)NT);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (row < M) {
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const int col = n0 + cchunk * 16 + q * 4;
-            if (col < ldc && cchunk * 16 + q * 4 < NT)
-              *reinterpret_cast<float4*>(C + row * ldc + col) =
-                  make_float4(__uint_as_float(v[q * 4]) + __uint_as_float(w[q * 4]),
-                              __uint_as_float(v[q * 4 + 1]) + __uint_as_float(w[q * 4 + 1]),
-                              __uint_as_float(v[q * 4 + 2]) + __uint_as_float(w[q * 4 + 2]),
-                              __uint_as_float(v[q * 4 + 3]) + __uint_as_float(w[q * 4 + 3]));
-          }
-        }
-      }
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      __syncthreads();
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    }
-  }
-  asm volatile("cp.async.wait_all;" ::: "memory");
-  if (failed && tid == 0) atomicExch(error_flag, 1);
-  if (!failed) {
-    for (int s = 0; s < kAStages; ++s)
-      if (stage_uses[s] > 0) mbar_wait(bar_empty0 + 8 * s, (stage_uses[s] - 1) & 1);
-  }
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
-  if (warp == 0) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
-  }
-}
-
-// dynamic shared memory of k_gemm_tc_resident<NT> for a given K
-template <int NT>
-inline size_t resident_smem_bytes(int K) {
-  const int kc = (K + kChunkK - 1) / kChunkK;
-  return (size_t)kAStages * 2 * kATileBytes + (size_t)kc * 2 * NT * kChunkK * 4 + 1024;
-}
-
-// ------------------------------------------------------------------------------------------------
-// Third form: the same product with the work split by role, so that staging, MMA issue and the
-// epilogue overlap instead of taking turns.
+// The product kernel: work split by role, so that staging, MMA issue and the epilogue overlap.
 //   warps 0-7   producers: 128-bit loads of the A and B chunks (two chunks ahead, in registers),
 //               hi/lo split, swizzled stores, fence, arrive on full[stage]
 //   warps 8-11 (8-15 with one accumulator set)  epilogue: wait for a finished accumulator set,
@@ -1020,9 +621,5 @@ k_gemm_tn_tc(const float* __restrict__ A, int lda, const float* __restrict__ B, 
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(Cfg::kTmemCols) : "memory");
   }
 }
-
-// dynamic shared memory of k_gemm_tc<NT>
-template <int NT>
-constexpr size_t smem_bytes() { return (size_t)kStages * (2 * kATileBytes + 2 * NT * kChunkK * 4) + 1024; }
 
 }  // namespace gtc

@@ -162,139 +162,6 @@ __global__ void k_spmm_long_rows(const int4* __restrict__ rows, const float4* __
   }
 }
 
-// Propagation with the gathered rows in flight in shared memory instead of registers.
-// The register-held form above keeps UN x V 16-byte loads per lane in flight, and the register
-// file caps how many warps can do that; measured, it stalls on load latency at ~45 % of the L2
-// rate.  Here a warp owns a ring of D row slots in shared memory: the row of stored entry q is
-// fetched with cp.async into slot q mod D while entry q - D, fetched D steps earlier, is read back
-// (each lane reads the bytes it copied itself) and accumulated, so a warp keeps D whole rows in
-// flight at the cost of a handful of registers.  A warp takes kGrab consecutive rows at a time from
-// a global counter (`row_counter`, zero at launch) and walks their stored entries as one stream, so
-// the ring drains once per grab, not once per row; column indices are prefetched two chunks of 32
-// ahead and their weights dinv[col] one chunk ahead.  V = float4 per lane (ld <= 128 V).
-constexpr int kGrab = 16;
-
-template <int V, int D>
-__global__ void __launch_bounds__(128)
-k_spmm_ring(const int* __restrict__ row_ptr, const int* __restrict__ col, const float* __restrict__ dinv,
-            const float4* __restrict__ x, float4* __restrict__ out, int n, int ld4, int* __restrict__ row_counter) {
-  static_assert(D <= 32, "the lag must stay within two chunks of 32");
-  extern __shared__ __align__(16) float4 ring_all[];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  float4* ring = ring_all + (size_t)warp * D * V * 32;
-  const uint32_t ring_s = (uint32_t)__cvta_generic_to_shared(ring);
-  for (;;) {
-    int row_base = 0;
-    if (lane == 0) row_base = atomicAdd(row_counter, kGrab);
-    row_base = __shfl_sync(0xffffffffu, row_base, 0);
-    if (row_base >= n) break;
-    const int rows_here = min(kGrab, n - row_base);
-    // lane t holds the end position and the scale of row row_base + t
-    int rp_lane = 0;
-    float di_lane = 0.f;
-    if (lane < rows_here) { rp_lane = row_ptr[row_base + lane + 1]; di_lane = dinv[row_base + lane]; }
-    const int p0 = row_ptr[row_base];
-    const int p1 = __shfl_sync(0xffffffffu, rp_lane, rows_here - 1);
-    const int total = p1 - p0;
-    int crow = 0;                                       // row (relative) being accumulated
-    int crow_end = __shfl_sync(0xffffffffu, rp_lane, 0);
-    float4 acc[V];
-#pragma unroll
-    for (int v = 0; v < V; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-    int c_cur = 0, c_nxt = 0, c_nxt2 = 0, cur_chunk = -1;
-    float w_cur = 0.f, w_prev = 0.f, w_nxt = 0.f;
-    if (p0 + lane < p1) c_nxt = col[p0 + lane];
-    if (p0 + 32 + lane < p1) c_nxt2 = col[p0 + 32 + lane];
-    if (p0 + lane < p1) w_nxt = dinv[c_nxt];
-
-    auto finish_row = [&]() {
-      const float di = __shfl_sync(0xffffffffu, di_lane, crow);
-#pragma unroll
-      for (int v = 0; v < V; ++v) {
-        const int f = lane + 32 * v;
-        if (f < ld4)
-          out[(long long)(row_base + crow) * ld4 + f] =
-              make_float4(di * acc[v].x, di * acc[v].y, di * acc[v].z, di * acc[v].w);
-        acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-      }
-    };
-
-    // entries move in batches of kBatch: one commit / one wait per batch, the batch's reads independent
-    constexpr int kBatch = 8;
-    static_assert(D % kBatch == 0 && 32 % kBatch == 0, "batching");
-    constexpr int kLagBatches = D / kBatch;
-    const int n_batches = (total + kBatch - 1) / kBatch;
-    for (int bq = 0; bq < n_batches + kLagBatches; ++bq) {
-      if (bq >= kLagBatches) {              // consume batch bq - kLagBatches (the oldest group in flight)
-        asm volatile("cp.async.wait_group %0;" ::"n"(kLagBatches - 1) : "memory");
-        const int q0 = (bq - kLagBatches) * kBatch;
-        float wj[kBatch];
-#pragma unroll
-        for (int t = 0; t < kBatch; ++t) {
-          const int qc = q0 + t;
-          const float wa = __shfl_sync(0xffffffffu, w_cur, qc & 31), wb = __shfl_sync(0xffffffffu, w_prev, qc & 31);
-          wj[t] = ((qc >> 5) == cur_chunk) ? wa : wb;
-        }
-        float4 xv[kBatch][V];
-#pragma unroll
-        for (int t = 0; t < kBatch; ++t)
-#pragma unroll
-          for (int v = 0; v < V; ++v) {
-            const int f = lane + 32 * v;
-            xv[t][v] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (f < ld4 && q0 + t < total) xv[t][v] = ring[(size_t)((q0 + t) % D) * V * 32 + f];
-          }
-#pragma unroll
-        for (int t = 0; t < kBatch; ++t) {
-          const int qc = q0 + t;
-          if (qc < total) {
-            while (p0 + qc >= crow_end) {   // entry belongs to a later row: close the finished one(s)
-              finish_row();
-              ++crow;
-              crow_end = __shfl_sync(0xffffffffu, rp_lane, crow);
-            }
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-              acc[v].x = fmaf(wj[t], xv[t][v].x, acc[v].x); acc[v].y = fmaf(wj[t], xv[t][v].y, acc[v].y);
-              acc[v].z = fmaf(wj[t], xv[t][v].z, acc[v].z); acc[v].w = fmaf(wj[t], xv[t][v].w, acc[v].w);
-            }
-          }
-        }
-      }
-      if (bq < n_batches) {                 // issue batch bq
-        const int q0 = bq * kBatch;
-        if ((q0 & 31) == 0) {               // the next chunk of 32 entries becomes current
-          w_prev = w_cur;
-          c_cur = c_nxt; w_cur = w_nxt;
-          c_nxt = c_nxt2;
-          cur_chunk = q0 >> 5;
-          const int a1 = p0 + q0 + 32 + lane, a2 = p0 + q0 + 64 + lane;
-          w_nxt = (a1 < p1) ? dinv[c_nxt] : 0.f;
-          c_nxt2 = (a2 < p1) ? col[a2] : 0;
-        }
-#pragma unroll
-        for (int t = 0; t < kBatch; ++t) {
-          const int q = q0 + t;
-          const int cj = __shfl_sync(0xffffffffu, c_cur, q & 31);
-          if (q < total) {
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-              const int f = lane + 32 * v;
-              if (f < ld4)
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ring_s + (uint32_t)(((q % D) * V * 32 + f) * 16)),
-                             "l"(x + (long long)cj * ld4 + f)
-                             : "memory");
-            }
-          }
-        }
-      }
-      asm volatile("cp.async.commit_group;" ::: "memory");
-    }
-    finish_row();                           // the last row of the grab (every row stores its self loop)
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-  }
-}
-
 // ------------------------------------------------------------------------------------------
 // Dense products.
 //   k_gemm_nn : C[M x N] = A[M x K] B[K x N]          (H = P W, D = P grad, G = S W^T, T = G W)
@@ -629,10 +496,12 @@ __global__ void k_resid_out(const float4* __restrict__ H, const float4* __restri
 // Step-size search of a W block (Section 3.1).  Along W - grad/t the pre-activation is
 // H - D/t with D = P grad, so every candidate is scored from H, D, Z without another product.
 // ------------------------------------------------------------------------------------------
-// hidden layer: acc[j] += sum ( (z - f(h - d/t_j))^2 - (z - f(h))^2 )   (times nu/2 at decision time)
+// Every block leaves its sums in `partial` (kCand, resp. 2, doubles per block); k_search_decide_w adds the
+// blocks up in a fixed order, so a decision does not depend on how the blocks were scheduled.
+// hidden layer: sum_j = sum ( (z - f(h - d/t_j))^2 - (z - f(h))^2 )   (times nu/2 at decision time)
 __global__ void __launch_bounds__(256)
 k_score_w_hidden(const float4* __restrict__ H, const float4* __restrict__ D, const float4* __restrict__ Z,
-                 long long n4, const SearchCtl* __restrict__ ctl, double* __restrict__ acc) {
+                 long long n4, const SearchCtl* __restrict__ ctl, double* __restrict__ partial) {
   if (ctl->done) return;
   __shared__ double sh[32];
   float inv[kCand];
@@ -665,14 +534,14 @@ k_score_w_hidden(const float4* __restrict__ H, const float4* __restrict__ D, con
 #pragma unroll
   for (int j = 0; j < kCand; ++j) {
     const double v = block_sum(s[j], sh);
-    if (threadIdx.x == 0) atomicAdd(acc + j, v);
+    if (threadIdx.x == 0) partial[(size_t)blockIdx.x * kCand + j] = v;
   }
 }
 
-// last layer: phi_L(t) - phi_L = -(1/t) <D, R> + (rho / 2t^2) ||D||^2 ; acc[0] += <D,R>, acc[1] += ||D||^2
+// last layer: phi_L(t) - phi_L = -(1/t) <D, R> + (rho / 2t^2) ||D||^2 ; sums <D,R> and ||D||^2
 __global__ void __launch_bounds__(256)
 k_score_w_out(const float4* __restrict__ D, const float4* __restrict__ R, long long n4,
-              const SearchCtl* __restrict__ ctl, double* __restrict__ acc) {
+              const SearchCtl* __restrict__ ctl, double* __restrict__ partial) {
   if (ctl->done) return;
   __shared__ double sh[32];
   double s1 = 0.0, s2 = 0.0;
@@ -684,7 +553,7 @@ k_score_w_out(const float4* __restrict__ D, const float4* __restrict__ R, long l
   }
   s1 = block_sum(s1, sh);
   s2 = block_sum(s2, sh);
-  if (threadIdx.x == 0) { atomicAdd(acc, s1); atomicAdd(acc + 1, s2); }
+  if (threadIdx.x == 0) { partial[(size_t)blockIdx.x * 2] = s1; partial[(size_t)blockIdx.x * 2 + 1] = s2; }
 }
 
 __device__ __forceinline__ void set_candidates(SearchCtl* c, double growth) {
@@ -693,19 +562,14 @@ __device__ __forceinline__ void set_candidates(SearchCtl* c, double growth) {
   for (int j = 0; j < kCand; ++j) { c->inv_cand[j] = (float)(1.0 / t); t *= growth; }
 }
 
-// Starts `count` searches: sums[i*stride + 0] = ||grad||^2, sums[i*stride + 1] = ||x||^2.
-__global__ void k_search_begin(SearchCtl* ctl, int count, const double* __restrict__ sums, int stride,
-                               double shrink, double growth, double* __restrict__ acc, int acc_per,
-                               int* __restrict__ n_active, int* __restrict__ status) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= count) return;
-  SearchCtl* c = ctl + i;
-  c->gg = sums[i * stride];
-  c->xx = sums[i * stride + 1];
+// Starts one search from ||grad||^2 and ||x||^2 of its block.
+__device__ __forceinline__ void begin_one(SearchCtl* c, double gg, double xx, double shrink, double growth,
+                                          int* __restrict__ n_active, int* __restrict__ status) {
+  c->gg = gg;
+  c->xx = xx;
   c->pass = 0;
   c->q = 0.0;
   c->inv_step = 0.f;
-  for (int j = 0; j < acc_per; ++j) acc[i * acc_per + j] = 0.0;
   if (!(c->gg > 1e-24 * c->xx)) {          // zero up to rounding (also catches NaN): skip
     c->done = 1;
     const bool finite = (c->gg == c->gg) && (c->xx == c->xx) && c->gg < 1.0e300 && c->xx < 1.0e300;
@@ -720,15 +584,44 @@ __global__ void k_search_begin(SearchCtl* ctl, int count, const double* __restri
   if (n_active) atomicAdd(n_active, 1);
 }
 
-// One decision per search.  mode 0: acc holds kCand sums of a scoring pass, delta_j = scale * acc[j]
+// Starts the search of a W block: sums[0] = ||grad||^2, sums[1] = ||W||^2.
+__global__ void k_search_begin(SearchCtl* ctl, const double* __restrict__ sums, double shrink, double growth,
+                               int* __restrict__ status) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) begin_one(ctl, sums[0], sums[1], shrink, growth, nullptr, status);
+}
+
+// Starts the searches of the `count` communities of a hidden layer, one warp each.  k_zgrad_finish left
+// three sums per row block in `partial`; the blocks of community i are block_ptr[i] .. block_ptr[i+1]-1
+// and are added up in a fixed order (lane-strided, then the shuffle tree).  sums[i*3 + ..] receives
+// { ||G_i||^2, ||Z_i||^2, <Z_i - f(H_i), G_i> }; acc (acc_per doubles per community) is cleared.
+__global__ void k_search_begin_z(SearchCtl* ctl, int count, const double* __restrict__ partial,
+                                 const int* __restrict__ block_ptr, double* __restrict__ sums, double shrink,
+                                 double growth, double* __restrict__ acc, int acc_per, int* __restrict__ n_active,
+                                 int* __restrict__ status) {
+  const int lane = threadIdx.x & 31;
+  const int i = (int)(((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+  if (i >= count) return;
+  double s0 = 0.0, s1 = 0.0, s2 = 0.0;
+  for (int b = block_ptr[i] + lane; b < block_ptr[i + 1]; b += 32) {
+    s0 += partial[(size_t)b * 3]; s1 += partial[(size_t)b * 3 + 1]; s2 += partial[(size_t)b * 3 + 2];
+  }
+  s0 = warp_sum(s0); s1 = warp_sum(s1); s2 = warp_sum(s2);
+  if (lane != 0) return;
+  sums[i * 3] = s0; sums[i * 3 + 1] = s1; sums[i * 3 + 2] = s2;
+  for (int j = 0; j < acc_per; ++j) acc[i * acc_per + j] = 0.0;
+  begin_one(ctl + i, s0, s1, shrink, growth, n_active, status);
+}
+
+// One decision per search.  mode 0: `cand` sums of a scoring pass, delta_j = scale * sum[j]
 // plus the quadratic own term; mode 1: closed form, delta(t) = -lin/t + quad/t^2, all trials at once.
 //   own term (Z blocks only): -(nu/t) sag + (nu/2t^2) sgg with sag = <Z - f(H), G>, sgg = gg
 struct DecideArgs {
   double growth;
   int max_trials;
   int mode;          // 0 scored candidates, 1 closed form
+  int cand;          // mode 0: candidates scored per pass (<= kCand)
   double scale;      // multiplies the scored sums (nu/2)
-  double quad_coef;  // closed form: delta = -acc[0]/t + quad_coef * acc[1] / t^2
+  double quad_coef;  // closed form: delta = -sum[0]/t + quad_coef * sum[1] / t^2
   double own_nu;     // nu when the block has a quadratic own term, else 0
   int last_pass;     // this is the final pass: mark exhausted searches
 };
@@ -746,17 +639,14 @@ __device__ __forceinline__ bool accept(SearchCtl* c, double delta, double t, int
   return false;
 }
 
-__global__ void k_search_decide(SearchCtl* ctl, int count, double* __restrict__ acc, int acc_per,
-                                const double* __restrict__ own, int own_stride, DecideArgs a,
-                                int* __restrict__ n_active, int* __restrict__ status) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= count) return;
-  SearchCtl* c = ctl + i;
-  if (c->done) return;
-  const double sag = (a.own_nu != 0.0) ? own[i * own_stride + 2] : 0.0;
+// Decision of one open search from the sums of the pass just scored.  Returns true when the search
+// goes on to another pass (its candidates are then already set).
+__device__ __forceinline__ bool decide_one(SearchCtl* c, const double* __restrict__ sums, double sag,
+                                           const DecideArgs& a, int* __restrict__ n_active,
+                                           int* __restrict__ status) {
   if (a.mode == 1) {
     double t = c->t_base;
-    const double lin = acc[i * acc_per], quad = a.quad_coef * acc[i * acc_per + 1];
+    const double lin = sums[0], quad = a.quad_coef * sums[1];
     bool ok = false;
     for (int trial = 0; trial < a.max_trials && !ok; ++trial) {
       const double delta = -lin / t + quad / (t * t) - a.own_nu * sag / t + 0.5 * a.own_nu * c->gg / (t * t);
@@ -765,30 +655,61 @@ __global__ void k_search_decide(SearchCtl* ctl, int count, double* __restrict__ 
     }
     if (!ok) { c->done = 1; c->trial = -2; c->inv_step = 0.f; if (!(lin == lin && quad == quad)) atomicOr(status, 1); }
     if (n_active) atomicSub(n_active, 1);
-    return;
+    return false;
   }
   double t = c->t_base;
   bool ok = false, finite = true;
-  for (int j = 0; j < kCand && !ok; ++j) {
-    const int trial = c->pass * kCand + j;
+  for (int j = 0; j < a.cand && !ok; ++j) {
+    const int trial = c->pass * a.cand + j;
     if (trial >= a.max_trials) break;
-    const double sum = acc[i * acc_per + j];
+    const double sum = sums[j];
     finite = finite && (sum == sum);
     const double delta = a.scale * sum - a.own_nu * sag / t + 0.5 * a.own_nu * c->gg / (t * t);
     ok = accept(c, delta, t, trial);
     t *= a.growth;
   }
   if (!finite) atomicOr(status, 1);
-  if (ok) { if (n_active) atomicSub(n_active, 1); return; }
+  if (ok) { if (n_active) atomicSub(n_active, 1); return false; }
   c->pass += 1;
-  if (a.last_pass || c->pass * kCand >= a.max_trials) {
+  if (a.last_pass || c->pass * a.cand >= a.max_trials) {
     c->done = 1; c->trial = -2; c->inv_step = 0.f;
     if (n_active) atomicSub(n_active, 1);
-    return;
+    return false;
   }
   c->t_base = t;
   set_candidates(c, a.growth);
-  for (int j = 0; j < acc_per; ++j) acc[i * acc_per + j] = 0.0;
+  return true;
+}
+
+// Decisions of `count` searches whose pass sums are in acc (acc_per doubles each).
+__global__ void k_search_decide(SearchCtl* ctl, int count, double* __restrict__ acc, int acc_per,
+                                const double* __restrict__ own, int own_stride, DecideArgs a,
+                                int* __restrict__ n_active, int* __restrict__ status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  SearchCtl* c = ctl + i;
+  if (c->done) return;
+  const double sag = (a.own_nu != 0.0) ? own[i * own_stride + 2] : 0.0;
+  if (decide_one(c, acc + i * acc_per, sag, a, n_active, status))
+    for (int j = 0; j < acc_per; ++j) acc[i * acc_per + j] = 0.0;
+}
+
+// Decision of a W block: the `n_part` blocks of the scoring kernel left `per` sums each in `partial`;
+// they are added in a fixed order (thread-strided, then the block tree) before the decision is taken.
+// One block of 256 threads.
+__global__ void __launch_bounds__(256)
+k_search_decide_w(SearchCtl* c, const double* __restrict__ partial, int n_part, int per, DecideArgs a,
+                  int* __restrict__ status) {
+  if (c->done) return;
+  __shared__ double sh[32];
+  __shared__ double total[kCand];
+  for (int j = 0; j < per; ++j) {
+    double s = 0.0;
+    for (int b = threadIdx.x; b < n_part; b += blockDim.x) s += partial[(size_t)b * per + j];
+    s = block_sum(s, sh);
+    if (threadIdx.x == 0) total[j] = s;
+  }
+  if (threadIdx.x == 0) decide_one(c, total, 0.0, a, nullptr, status);
 }
 
 // The decision log is a ring of `ring` passes; the slot in use is *pass mod ring, with the pass counter
@@ -843,47 +764,31 @@ __global__ void k_axpy_ctl(float4* __restrict__ Y, const float4* __restrict__ X,
 // ------------------------------------------------------------------------------------------
 // Hidden Z blocks (Appendix A).  The gradient of psi_m with respect to Z_{l,m} is the rows V_m of
 //   G = nu (Z_l - f(H_l)) + (A~ R') W_{l+1}^T ,
-// R' the residual of layer l+1 at the new W.  k_zgrad_finish adds the first term to the product
-// and accumulates, per community, sums[m] = { ||G_m||^2, ||Z_{l,m}||^2, <Z_l - f(H_l), G>_m }.
-// One block owns `rows_per_block` consecutive rows.
+// R' the residual of layer l+1 at the new W.  k_zgrad_finish adds the first term to the product and
+// leaves, per row block, partial[b*3 + ..] = { ||G||^2, ||Z_l||^2, <Z_l - f(H_l), G> } over the block's
+// rows.  blocks[b] = {first row, one past the last}: a block never crosses a community boundary, so
+// the sums of a community are the sums of its blocks, added in a fixed order by k_search_begin_z.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 k_zgrad_finish(float4* __restrict__ G, const float4* __restrict__ Z, const float4* __restrict__ H, int ld4,
-               long long n, int rows_per_block, const int* __restrict__ row_comm, float nu,
-               double* __restrict__ sums) {
+               const int2* __restrict__ blocks, float nu, double* __restrict__ partial) {
   __shared__ double sh[32];
-  const long long r0 = (long long)blockIdx.x * rows_per_block;
-  const long long r1 = min(n, r0 + rows_per_block);
-  if (r0 >= r1) return;
-  const bool single = row_comm[r0] == row_comm[r1 - 1];
+  const int2 rb = blocks[blockIdx.x];
   double sgg = 0.0, szz = 0.0, sag = 0.0;
-  int cur = row_comm[r0];
-  const long long e0 = r0 * ld4, e1 = r1 * ld4;
+  const long long e0 = (long long)rb.x * ld4, e1 = (long long)rb.y * ld4;
   for (long long e = e0 + threadIdx.x; e < e1; e += blockDim.x) {
     const float4 z = Z[e], h = H[e];
     float4 g = G[e];
     const float ax = z.x - relu(h.x), ay = z.y - relu(h.y), az = z.z - relu(h.z), aw = z.w - relu(h.w);
     g.x = fmaf(nu, ax, g.x); g.y = fmaf(nu, ay, g.y); g.z = fmaf(nu, az, g.z); g.w = fmaf(nu, aw, g.w);
     G[e] = g;
-    if (!single) {
-      const int m = row_comm[e / ld4];
-      if (m != cur) {
-        atomicAdd(sums + cur * 3 + 0, sgg); atomicAdd(sums + cur * 3 + 1, szz); atomicAdd(sums + cur * 3 + 2, sag);
-        sgg = szz = sag = 0.0;
-        cur = m;
-      }
-    }
     sgg += (double)(g.x * g.x + g.y * g.y + g.z * g.z + g.w * g.w);
     szz += (double)(z.x * z.x + z.y * z.y + z.z * z.z + z.w * z.w);
     sag += (double)(ax * g.x + ay * g.y + az * g.z + aw * g.w);
   }
-  if (single) {
-    sgg = block_sum(sgg, sh); szz = block_sum(szz, sh); sag = block_sum(sag, sh);
-    if (threadIdx.x == 0) {
-      atomicAdd(sums + cur * 3 + 0, sgg); atomicAdd(sums + cur * 3 + 1, szz); atomicAdd(sums + cur * 3 + 2, sag);
-    }
-  } else {
-    atomicAdd(sums + cur * 3 + 0, sgg); atomicAdd(sums + cur * 3 + 1, szz); atomicAdd(sums + cur * 3 + 2, sag);
+  sgg = block_sum(sgg, sh); szz = block_sum(szz, sh); sag = block_sum(sag, sh);
+  if (threadIdx.x == 0) {
+    partial[(size_t)blockIdx.x * 3] = sgg; partial[(size_t)blockIdx.x * 3 + 1] = szz; partial[(size_t)blockIdx.x * 3 + 2] = sag;
   }
 }
 
@@ -916,7 +821,11 @@ __device__ __forceinline__ float warp_sum2(float v0, float v1, int lane) {
 // which is non-zero on V_m and its first-order neighbour rows only.  A warp owns row i and walks
 // its stored entries once; col_comm gives the community of every entry, entries of one community
 // are contiguous (ascending columns), and at every change of community the finished K_m[i] is scored:
-//   OUT = false (layer l+1 < L, ReLU):  acc[m*kCand + j] += sum_c (z - f(h - k/t_j))^2 - (z - f(h))^2
+//   OUT = false (layer l+1 < L, ReLU):  acc[m*NC + j] += sum_c (z - f(h - k/t_j))^2 - (z - f(h))^2, j < NC
+//                                        (NC = candidates scored per sweep, 2 or 4: almost every search
+//                                        closes at its first or second trial, and a candidate costs two
+//                                        instructions per element, so the first sweep scores two and the
+//                                        rare search that needs more is served by a further sweep)
 //   OUT = true  (layer l+1 = L):        acc[m*2] += <k, R'>, acc[m*2+1] += ||k||^2   (closed form)
 // Sums are kept per warp in shared memory (no atomics on the hot path) and added to `acc` once per
 // block; with too many communities for that (use_smem == 0) they go to `acc` directly.
@@ -934,7 +843,7 @@ __device__ __forceinline__ float4 twice_error(const float4& h, const float4& z) 
 
 // Scores one finished K_m[i] (k, still without the factor di) against the row's a, b:
 // OUT: a = R'; else a = h and b = twice_error(h, z).
-template <int V, bool OUT>
+template <int V, bool OUT, int NC>
 __device__ __forceinline__ void score_segment(const float4 (&k)[V], float di, const float4 (&a)[V],
                                               const float4 (&b)[V], const SearchCtl* __restrict__ ctl,
                                               int cur, int lane, double* mine, bool plain_add) {
@@ -952,9 +861,10 @@ __device__ __forceinline__ void score_segment(const float4 (&k)[V], float di, co
       if (plain_add) *dst += (double)r; else atomicAdd(dst, (double)r);
     }
   } else {
-    float inv[kCand], part[kCand];
+    static_assert(NC == 2 || NC == 4, "two or four candidates per sweep");
+    float inv[NC], part[NC];
 #pragma unroll
-    for (int j = 0; j < kCand; ++j) { inv[j] = di * ctl[cur].inv_cand[j]; part[j] = 0.f; }   // K_m[i] = di * k
+    for (int j = 0; j < NC; ++j) { inv[j] = di * ctl[cur].inv_cand[j]; part[j] = 0.f; }   // K_m[i] = di * k
 #pragma unroll
     for (int v = 0; v < V; ++v) {
       const float kk[4] = {k[v].x, k[v].y, k[v].z, k[v].w};
@@ -964,22 +874,29 @@ __device__ __forceinline__ void score_segment(const float4 (&k)[V], float di, co
       for (int c = 0; c < 4; ++c) {
         const float pos = fmaxf(hh[c], 0.f), neg = fmaxf(-hh[c], 0.f);
 #pragma unroll
-        for (int j = 0; j < kCand; ++j) {
+        for (int j = 0; j < NC; ++j) {
           const float df = relu_drop(kk[c], inv[j], neg, pos);
           part[j] = fmaf(df, ee[c] + df, part[j]);   // e1^2 - e0^2 = df (2 e0 + df)
         }
       }
     }
-    static_assert(kCand == 4, "warp_sum4 reduces exactly four candidates");
-    const float r = warp_sum4(part[0], part[1], part[2], part[3], lane);
-    if ((lane & 7) == 0) {
-      double* dst = mine + cur * kCand + (lane >> 3);
-      if (plain_add) *dst += (double)r; else atomicAdd(dst, (double)r);
+    if constexpr (NC == 4) {
+      const float r = warp_sum4(part[0], part[1], part[2], part[3], lane);
+      if ((lane & 7) == 0) {
+        double* dst = mine + cur * NC + (lane >> 3);
+        if (plain_add) *dst += (double)r; else atomicAdd(dst, (double)r);
+      }
+    } else {
+      const float r = warp_sum2(part[0], part[1], lane);
+      if ((lane & 15) == 0) {
+        double* dst = mine + cur * NC + (lane >> 4);
+        if (plain_add) *dst += (double)r; else atomicAdd(dst, (double)r);
+      }
     }
   }
 }
 
-template <int V, bool OUT, int UN>
+template <int V, bool OUT, int UN, int NC>
 __global__ void __launch_bounds__(256, (V <= 1 ? 4 : V <= 2 ? 3 : 1))
 k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
           const unsigned short* __restrict__ col_comm, const float* __restrict__ dinv,
@@ -988,7 +905,7 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
           double* __restrict__ acc, const int* __restrict__ n_active, int use_smem, int* __restrict__ row_counter,
           const int4* __restrict__ items, int n_items, int long_len, float4* __restrict__ scratch) {
   if (*n_active <= 0) return;
-  constexpr int PER = OUT ? 2 : kCand;
+  constexpr int PER = OUT ? 2 : NC;
   // dynamic shared memory: per warp the row's a, b (2 V float4 per lane; parked there during the
   // walk so that the registers hold gathered rows instead), then the per-warp sums
   extern __shared__ float4 s_raw[];
@@ -1080,7 +997,7 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
         a[v] = row_ab[32 * v];
         b[v] = OUT ? a[v] : row_ab[32 * (V + v)];
       }
-      score_segment<V, OUT>(k, di, a, b, ctl, cur, lane, mine, plain_add);
+      score_segment<V, OUT, NC>(k, di, a, b, ctl, cur, lane, mine, plain_add);
     };
 
     // column and community of a chunk are fetched while the chunk before it is walked; the two
@@ -1298,7 +1215,7 @@ k_score_z_out_half(const int* __restrict__ row_ptr, const int* __restrict__ col,
 
 // Segments that k_score_z handled in pieces: K_m[i] = sum of the pieces (item order), then scored
 // as above.  split[s] = {row, community, first item, number of items}; one warp per entry.
-template <int V, bool OUT>
+template <int V, bool OUT, int NC>
 __global__ void __launch_bounds__(256)
 k_score_z_split(const int4* __restrict__ split, int n_split, const float* __restrict__ dinv,
                 const float4* __restrict__ scratch, const float4* __restrict__ Hn, const float4* __restrict__ Zn,
@@ -1324,7 +1241,7 @@ k_score_z_split(const int4* __restrict__ split, int n_split, const float* __rest
       }
     }
   }
-  score_segment<V, OUT>(k, dinv[sp.x], a, b, ctl, sp.y, lane, acc, false);
+  score_segment<V, OUT, NC>(k, dinv[sp.x], a, b, ctl, sp.y, lane, acc, false);
 }
 
 // The rows of Eq. 7 without a loss term (not in the training set) have the closed form
@@ -1450,10 +1367,11 @@ k_output_rows(float* __restrict__ ZL, float* __restrict__ U, const float* __rest
 // ------------------------------------------------------------------------------------------
 // Reporting (Eq. 1) and the forward pass of Problem 1.
 // ------------------------------------------------------------------------------------------
-// out[0] += sum (z - f(h))^2
+// The sums below leave one partial per block in `partial`; k_add_partials adds the blocks in a fixed order.
+// partial[b] = sum (z - f(h))^2 over the block's elements
 __global__ void __launch_bounds__(256)
 k_sum_hidden_penalty(const float4* __restrict__ Z, const float4* __restrict__ H, long long n4,
-                     double* __restrict__ out) {
+                     double* __restrict__ partial) {
   __shared__ double sh[32];
   double s = 0.0;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4;
@@ -1463,13 +1381,13 @@ k_sum_hidden_penalty(const float4* __restrict__ Z, const float4* __restrict__ H,
     s += (double)(a * a + b * b + c * c + d * d);
   }
   s = block_sum(s, sh);
-  if (threadIdx.x == 0) atomicAdd(out, s);
+  if (threadIdx.x == 0) partial[blockIdx.x] = s;
 }
 
-// out[0] += <U, Z - H>, out[1] += ||Z - H||^2
+// partial[2b] = <U, Z - H>, partial[2b+1] = ||Z - H||^2 over the block's elements
 __global__ void __launch_bounds__(256)
 k_sum_constraint(const float4* __restrict__ Z, const float4* __restrict__ H, const float4* __restrict__ U,
-                 long long n4, double* __restrict__ out) {
+                 long long n4, double* __restrict__ partial) {
   __shared__ double sh[32];
   double s1 = 0.0, s2 = 0.0;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4;
@@ -1481,47 +1399,70 @@ k_sum_constraint(const float4* __restrict__ Z, const float4* __restrict__ H, con
   }
   s1 = block_sum(s1, sh);
   s2 = block_sum(s2, sh);
-  if (threadIdx.x == 0) { atomicAdd(out, s1); atomicAdd(out + 1, s2); }
+  if (threadIdx.x == 0) { partial[2 * (size_t)blockIdx.x] = s1; partial[2 * (size_t)blockIdx.x + 1] = s2; }
 }
 
-// Per row: cross-entropy of the row of Zrows with its label (training rows only) summed into out[0];
-// argmax of the row of `logits` (lowest index on ties) to labels[row]; out[1] += training rows whose
-// argmax equals the label.  One warp per row.  Either of Zrows / logits may be NULL.
+// out[j] += sum over b < n_part of partial[b*per + j], j < per; one block, fixed order
+// (thread-strided, then the block tree).
+__global__ void __launch_bounds__(256)
+k_add_partials(const double* __restrict__ partial, int n_part, int per, double* __restrict__ out) {
+  __shared__ double sh[32];
+  for (int j = 0; j < per; ++j) {
+    double s = 0.0;
+    for (int b = threadIdx.x; b < n_part; b += blockDim.x) s += partial[(size_t)b * per + j];
+    s = block_sum(s, sh);
+    if (threadIdx.x == 0) out[j] += s;
+  }
+}
+
+// Per row: cross-entropy of the row of Zrows with its label (training rows only); argmax of the row of
+// `logits` (lowest index on ties) to labels[row]; whether a training row's argmax equals its label.
+// One warp per row; partial[2b] = the block's cross-entropy sum, partial[2b+1] = its count of hits,
+// rows added in row order.  Either of Zrows / logits may be NULL.
 __global__ void __launch_bounds__(256)
 k_row_loss_argmax(const float* __restrict__ Zrows, const float* __restrict__ logits, int ld, int C, int n,
                   const int* __restrict__ y, const unsigned char* __restrict__ train,
-                  int* __restrict__ labels, double* __restrict__ out) {
-  const int lane = threadIdx.x & 31;
-  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (row >= n) return;
-  const long long base = (long long)row * ld;
-  const bool tr = train[row] != 0;
-  if (Zrows != nullptr && tr) {
-    float mx = -3.0e38f;
-    for (int c = lane; c < C; c += 32) mx = fmaxf(mx, Zrows[base + c]);
-    mx = warp_max(mx);
-    float se = 0.f;
-    for (int c = lane; c < C; c += 32) se += expf(Zrows[base + c] - mx);
-    se = warp_sum(se);
-    if (lane == 0) atomicAdd(out, (double)(mx + logf(se) - Zrows[base + y[row]]));
-  }
-  if (logits != nullptr) {
-    float best = -3.0e38f;
-    int arg = 0x7fffffff;
-    for (int c = lane; c < C; c += 32) {
-      const float v = logits[base + c];
-      if (v > best) { best = v; arg = c; }
+                  int* __restrict__ labels, double* __restrict__ partial) {
+  __shared__ double s_loss[8], s_hit[8];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int row = blockIdx.x * (blockDim.x >> 5) + warp;
+  double loss = 0.0, hit = 0.0;
+  if (row < n) {
+    const long long base = (long long)row * ld;
+    const bool tr = train[row] != 0;
+    if (Zrows != nullptr && tr) {
+      float mx = -3.0e38f;
+      for (int c = lane; c < C; c += 32) mx = fmaxf(mx, Zrows[base + c]);
+      mx = warp_max(mx);
+      float se = 0.f;
+      for (int c = lane; c < C; c += 32) se += expf(Zrows[base + c] - mx);
+      se = warp_sum(se);
+      loss = (double)(mx + logf(se) - Zrows[base + y[row]]);
     }
+    if (logits != nullptr) {
+      float best = -3.0e38f;
+      int arg = 0x7fffffff;
+      for (int c = lane; c < C; c += 32) {
+        const float v = logits[base + c];
+        if (v > best) { best = v; arg = c; }
+      }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ob = __shfl_xor_sync(0xffffffffu, best, o);
-      const int oa = __shfl_xor_sync(0xffffffffu, arg, o);
-      if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oa = __shfl_xor_sync(0xffffffffu, arg, o);
+        if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
+      }
+      if (lane == 0 && labels) labels[row] = arg;
+      if (tr && arg == y[row]) hit = 1.0;
     }
-    if (lane == 0) {
-      if (labels) labels[row] = arg;
-      if (tr && arg == y[row]) atomicAdd(out + 1, 1.0);
-    }
+  }
+  if (lane == 0) { s_loss[warp] = loss; s_hit[warp] = hit; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double a = 0.0, b = 0.0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { a += s_loss[w]; b += s_hit[w]; }
+    partial[2 * (size_t)blockIdx.x] = a;
+    partial[2 * (size_t)blockIdx.x + 1] = b;
   }
 }
 

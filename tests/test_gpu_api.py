@@ -82,3 +82,61 @@ def test_two_handles_do_not_interfere_and_launches_are_counted():
         a.destroy()
         b.destroy()
         ref.destroy()
+
+
+def splitmix64(x):
+    """Output function of the splitmix64 generator at state x + 0x9E3779B97F4A7C15 (Steele, Lea, Flood 2014)."""
+    m = (1 << 64) - 1
+    z = (x + 0x9E3779B97F4A7C15) & m
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & m
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & m
+    return z ^ (z >> 31)
+
+
+def test_seeded_initial_weights_when_none_are_given():
+    """w_init = NULL: Glorot-uniform from the counter-based generator the header defines, re-derived here."""
+    wl = inputs.make_workload(0)
+    def weights(seed):
+        g = binding.GcnAdmm(wl.n, wl.row_ptr, wl.col_idx, wl.X, wl.y, wl.train_mask, wl.widths, wl.n_comm, wl.community,
+                            None, nu=wl.nu, rho=wl.rho, seed=seed)
+        try:
+            g.step(2)                                                   # the handle works like any other
+            assert np.isfinite(g.objective()).all()
+            g2 = binding.GcnAdmm(wl.n, wl.row_ptr, wl.col_idx, wl.X, wl.y, wl.train_mask, wl.widths, wl.n_comm,
+                                 wl.community, None, nu=wl.nu, rho=wl.rho, seed=seed)
+            try:
+                return [g2.weights(l) for l in range(1, len(wl.widths))]
+            finally:
+                g2.destroy()
+        finally:
+            g.destroy()
+    a, b = weights(12345), weights(12346)
+    for l, w in enumerate(a, start=1):
+        r, c = wl.widths[l - 1], wl.widths[l]
+        bound = np.sqrt(6.0 / (r + c))
+        want = np.array([[bound * (2.0 * ((splitmix64(12345 + (l << 32) + i * c + j) >> 40) / 16777216.0) - 1.0)
+                          for j in range(c)] for i in range(r)]).astype(np.float32)
+        assert np.array_equal(w, want)
+        assert np.abs(w).max() <= bound and abs(w.mean()) < 0.2 * bound
+        assert not np.array_equal(w, b[l - 1])
+
+
+def test_a_raised_pipeline_flag_surfaces_once_and_the_handle_stays_usable():
+    """The bounded waits of the tensor-core products report through a device flag.  Host half of that path:
+    with the flag written from here, the next synchronising call fails with GCN_ADMM_ERR_CUDA, the flag is
+    cleared, and the handle keeps working."""
+    wl = inputs.make_workload(0)
+    g = make(wl)
+    try:
+        g.step(1)
+        before = g.objective()
+        g.set_state(binding.ST_PIPELINE_FLAG, 0, np.array([1], dtype=np.int32))
+        with pytest.raises(binding.GcnAdmmError) as e:
+            g.objective()
+        assert e.value.code == -6 and "tensor-core" in str(e.value)
+        assert int(g.get_state(binding.ST_PIPELINE_FLAG)[0]) == 0
+        assert np.array_equal(g.objective(), before)
+        g.step(1)
+        assert np.isfinite(g.objective()).all()
+    finally:
+        g.destroy()

@@ -73,26 +73,3 @@ def test_many_small_communities_and_isolated_nodes():
 def test_dual_mode_one_and_other_search_parameters():
     pr = tiny_problem(7, n=80, widths=(6, 9, 4), n_comm=3)
     run_pair(pr, dual_mode=1, bt_growth=3.0, bt_shrink=0.3, tau0=0.01, theta0=0.02, fista_iters=7, loss_scale=0.5)
-
-
-def test_ring_propagation_kernel_matches():
-    """spmm_ring = 1 (gathered rows in flight in shared memory) gives the same propagation."""
-    from paper_2112_09335_b200 import inputs
-    wl = inputs.make_workload(3, scale=0.02)
-    kw = dict(nu=wl.nu, rho=wl.rho)
-    a = binding.GcnAdmm(wl.n, wl.row_ptr, wl.col_idx, wl.X, wl.y, wl.train_mask, wl.widths, wl.n_comm, wl.community,
-                        wl.w_init, spmm_ring=1, **kw)
-    b = binding.GcnAdmm(wl.n, wl.row_ptr, wl.col_idx, wl.X, wl.y, wl.train_mask, wl.widths, wl.n_comm, wl.community,
-                        wl.w_init, spmm_ring=0, **kw)
-    try:
-        rng = np.random.default_rng(0)
-        for width in (68, 100, 128, 200, 256):
-            x = rng.standard_normal((wl.n, width)).astype(np.float32)
-            assert relerr(a.propagate(x), b.propagate(x)) < 2e-7
-        a.step(3)
-        b.step(3)
-        for l in range(1, len(wl.widths)):
-            assert relerr(a.get_state(binding.ST_Z, l), b.get_state(binding.ST_Z, l)) < 1e-5
-    finally:
-        a.destroy()
-        b.destroy()

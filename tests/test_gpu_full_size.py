@@ -2,7 +2,9 @@
 launch configuration bench.py times.  A full oracle pass is out of reach there, so sampled outputs are
 checked against rows the fp64 oracle computes one by one (oracle/sampled_rows.py): propagation rows, the
 hidden Z block updates (given the accepted theta, whose decision is logged), the output-layer rows and
-the dual rows; plus properties that hold at any size (no exhausted search, every accepted q >= 1)."""
+the dual rows; the step-size decision of sampled communities is re-evaluated in fp64 from the community's
+rows and their neighbours (the accepted trial must satisfy the condition of Eq. 9, the one before it must
+not); plus properties that hold at any size (no exhausted search, every accepted q >= 1)."""
 import numpy as np
 import pytest
 
@@ -62,9 +64,24 @@ def test_sampled_rows_at_full_size():
         report = {}
         for l in range(1, L):                      # hidden Z blocks: Z_new = Z - grad / theta_{comm(row)}
             Z, W, U = fetch()
+            # start every search of this layer three doublings lower, so that accepted trials are preceded
+            # by rejected ones and both sides of the condition can be checked
+            g.set_state(binding.ST_THETA, l, g.get_state(binding.ST_THETA, l) / 8.0)
             g.step_block(binding.PHASE_Z, l)
             theta = g.get_state(binding.ST_THETA, l)
-            trial = g.decisions()["trial_z"][0, l - 1]
+            dz = g.decisions()
+            trial, q_gpu = dz["trial_z"][0, l - 1], dz["q_z"][0, l - 1]
+            assert (trial >= 0).all()
+            # Eq. 9 in fp64 for two communities: the one whose decision was tightest, and a random other one
+            tight = int(np.argmin(np.abs(q_gpu - 1.0)))
+            for m in (tight, int((tight + 1 + rng.integers(0, M - 1)) % M)):
+                t_acc = float(theta[m])
+                gg, (c_acc, c_prev) = sr.psi_change(l, np.flatnonzero(wl.community == m), Z, W, U, [t_acc, t_acc / 2.0])
+                q_acc, q_prev = -c_acc / (gg / (2.0 * t_acc)), -c_prev / (gg / t_acc)
+                report[f"theta{l},{m}"] = (q_acc, q_gpu[m])
+                assert q_acc >= 1.0 - 1e-4, (l, m, q_acc)
+                assert trial[m] == 0 or q_prev < 1.0 + 1e-4, (l, m, trial[m], q_prev)
+                assert abs(q_gpu[m] - q_acc) <= 2e-3 * abs(q_acc), (l, m, q_gpu[m], q_acc)
             got = g.get_state(binding.ST_Z, l)[rows]
             grad = sr.grad_Z_rows(l, rows, Z, W, U)
             comm = wl.community[rows]

@@ -19,7 +19,7 @@ TIE = 1e-3          # decisions may differ only where the oracle is this close t
 def small_cases():
     return [("cfg0", lambda: inputs.make_workload(0)),
             ("cfg1", lambda: inputs.make_workload(1)),
-            ("cfg2@0.15", lambda: inputs.make_workload(2, scale=0.15)),
+            ("cfg2", lambda: inputs.make_workload(2)),
             ("cfg3@0.012", lambda: inputs.make_workload(3, scale=0.012)),
             ("cfg4@0.001", lambda: inputs.make_workload(4, scale=0.001)),
             ("table2@0.12", lambda: inputs.make_workload(5, scale=0.12))]
@@ -158,11 +158,11 @@ def test_single_block_updates_from_identical_state(case):
     print("\n" + "\n".join(f"  {n}: rel {a:.2e}  step-rel {b:.2e}" for n, a, b in report))
 
 
-@pytest.mark.parametrize("tensor_cores", [1, 3])
+@pytest.mark.parametrize("tensor_cores", [1, 2])
 def test_single_block_updates_at_tensor_core_sizes(tensor_cores):
     """The cases above have fewer than 4096 rows, where the weight gradient P^T R runs on the fp32 FMA
     kernel.  With 8,467 rows every dense product of a block update, the transposed one with the
-    residual operand formed inside it included, runs on the tensor cores (3: weights pre-split):
+    residual operand formed inside it included, runs on the tensor cores (2: weights pre-split):
     same single-block check, every W block and every hidden Z block of every community."""
     wl = inputs.make_workload(3, scale=0.05)
     assert wl.n >= 4096
@@ -251,10 +251,47 @@ def test_ten_iterations(case, dual_mode):
         g.destroy()
 
 
-@pytest.mark.parametrize("tensor_cores", [0, 3])
+def test_ten_iterations_on_the_large_problem_paths():
+    """powerlaw-large at a tenth of its size (16,934 rows, 128-256-256-40, 32 communities): the code paths the full-size
+    workloads take -- the weight operand split once per product and fetched by bulk copies (from 16,384 rows), the
+    transposed product on the tensor cores with the residual formed inside it, rows longer than the default
+    `long_row` walked as work items -- over ten passes against the oracle.  A pass of the oracle costs about ten
+    seconds here, so it is run once, replaying the library's step-size decisions: each must satisfy the condition
+    in fp64 and the trial before it must fail."""
+    wl = inputs.make_workload(3, scale=0.1)
+    assert wl.n >= 16384 and (np.diff(wl.row_ptr) + 1).max() > 256
+    g, o = make_pair(wl)
+    try:
+        n_it = 10
+        g.step(n_it)
+        dec = g.decisions()
+        assert (dec["trial_w"] >= -1).all() and (dec["trial_z"] >= -1).all()
+        o.forced_tol = 1e-4
+        for k in range(n_it):
+            rec = o.iterate(forced_from(dec, k, o.L, o.M))
+            bad = [(key, r) for key, r in list(rec["W"].items()) + list(rec["Z"].items()) if not r["ok"]]
+            assert not bad, f"pass {k}: decisions violate the fp64 condition: {bad[:3]}"
+        worst = 0.0
+        for l in range(1, o.L + 1):
+            ew, ez = relerr(g.get_state(binding.ST_W, l), o.W[l]), relerr(g.get_state(binding.ST_Z, l), o.Z[l])
+            worst = max(worst, ew, ez)
+            assert ew <= ITER_TOL and ez <= ITER_TOL, (l, ew, ez)
+        eu = relerr(g.get_state(binding.ST_U), o.U)
+        go, oo = g.objective(), o.objective()
+        print(f"\n  worst W/Z rel {worst:.2e}  U rel {eu:.2e}  L_rho {go[0]:.6g} vs {oo[0]:.6g}  acc {go[5]:.4f} vs {oo[5]:.4f}")
+        assert eu <= ITER_TOL
+        scale = np.abs(oo[1:5]).sum()
+        for i in range(5):
+            assert abs(go[i] - oo[i]) <= ITER_TOL * scale, (i, go[i], oo[i])
+        assert abs(go[5] - oo[5]) <= max(ITER_TOL * oo[5], 1.5 / max(int(wl.train_mask.sum()), 1))
+    finally:
+        g.destroy()
+
+
+@pytest.mark.parametrize("tensor_cores", [0, 2])
 def test_ten_iterations_other_product_kernels(tensor_cores):
     """The fp32 FMA kernels (tensor_cores = 0) stay a supported path, and the pre-split weight operand
-    (3; taken by default only from 16384 rows) must give the same iterates: same ten-pass check on one case."""
+    (2; taken by default only from 16384 rows) must give the same iterates: same ten-pass check on one case."""
     wl = inputs.make_workload(3, scale=0.012)
     g, o = make_pair(wl)
     g.destroy()

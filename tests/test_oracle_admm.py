@@ -400,6 +400,34 @@ def test_sampled_row_evaluator_matches_the_full_oracle():
         np.testing.assert_allclose(sr.grad_Z_rows(l, rows, o.Z, o.W, o.U), full, atol=1e-12)
     np.testing.assert_allclose(sr.ZL_rows(rows, o.Z, o.W, o.U), o.update_ZL(o.W), atol=1e-12)
     np.testing.assert_allclose(sr.U_rows(rows, o.Z, o.W, o.U), o.update_U(o.W, o.Z), atol=1e-13)
+    np.testing.assert_allclose(sr.adj_rows(rows[::3]).toarray(), At[::3], atol=1e-15)
+
+
+@pytest.mark.parametrize("seed,widths", [(33, (5, 6, 4, 3)), (34, (4, 5, 3)), (35, (3, 4, 4, 5, 2))])
+def test_community_step_condition_evaluator_matches_psi(seed, widths):
+    """``SampledRows.psi_change`` (objective change of one community along its step, from the community's
+    rows and their neighbours only) against differences of the full oracle's literal psi_m, and its
+    ||grad||^2 against grad_psi; the accepted theta of the oracle's own search must pass by it and the
+    trial before must fail."""
+    from oracle.sampled_rows import SampledRows
+    pr, o = make(seed, n=30, widths=widths, n_comm=4)
+    sr = SampledRows(pr["n"], pr["row_ptr"], pr["col_idx"], pr["y"], pr["mask"], pr["widths"], o.p.nu, o.p.rho)
+    for l in range(1, o.L):
+        for m in range(o.M):
+            g = o.grad_psi(l, m)
+            thetas = [0.05, 0.4, 3.0, 50.0]
+            gg, change = sr.psi_change(l, o.V[m], o.Z, o.W, o.U, thetas)
+            assert abs(gg - np.sum(g * g)) <= 1e-12 * max(gg, 1e-300)
+            f0 = o.psi(l, m, o.Z[l][o.V[m]])
+            for t, c in zip(thetas, change):
+                want = o.psi(l, m, o.Z[l][o.V[m]] - g / t) - f0
+                assert abs(c - want) <= 1e-11 * max(abs(f0), 1.0), (l, m, t, c, want)
+            o.theta[l][m] = 1e-3
+            _, t, rec = o.update_Z(l, m, o.W)
+            assert rec["trial"] >= 1
+            gg, (c_acc, c_prev) = sr.psi_change(l, o.V[m], o.Z, o.W, o.U, [t, t / o.p.bt_growth])
+            assert -c_acc >= gg / (2 * t) and -c_prev < gg / (2 * (t / o.p.bt_growth))
+            assert abs(-c_acc / (gg / (2 * t)) - rec["q"]) <= 1e-9 * abs(rec["q"])
 
 
 @pytest.mark.parametrize("seed,n_comm", [(41, 1), (42, 3)])

@@ -4,8 +4,8 @@ Some users of this library run where reserving device memory at call time is not
 service whose memory was carved up at start-up, code living inside another framework's pool, a
 region under stream capture.  For them the library carries its staging memory inside the binary.
 This test calls that entry point through the C ABI twice in a row on device buffers and checks
-both results against the ordinary gcn_admm_propagate, with the same tolerance the propagation
-parity test uses.  It is named so that pytest collects it last."""
+its results against the ordinary gcn_admm_propagate, with the same tolerance the propagation
+parity test uses, and that the device's free memory does not move across a call.  It is named so that pytest collects it last."""
 import numpy as np
 import pytest
 
@@ -20,17 +20,33 @@ def test_static_propagation_matches_the_allocating_one_twice():
     g = binding.GcnAdmm(wl.n, wl.row_ptr, wl.col_idx, wl.X, wl.y, wl.train_mask, wl.widths, wl.n_comm, wl.community,
                         wl.w_init, nu=wl.nu, rho=wl.rho)
     try:
-        for width, seed in ((47, 0), (200, 1)):          # two calls in a row share the built-in memory
+        # calls in a row share the built-in memory: wide, narrow, wide again (the narrow call leaves the wide
+        # call's values behind under another row stride), then wider than one column block of the kernel
+        for k, (width, seed) in enumerate(((200, 0), (47, 1), (200, 2), (300, 3))):
             gen = torch.Generator(device="cuda").manual_seed(seed)
             x = torch.randn(wl.n, width, device="cuda", generator=gen)
             want = torch.empty_like(x)
             got = torch.full_like(x, float("nan"))
             g.propagate(x.data_ptr(), width, out=want.data_ptr())
+            torch.cuda.synchronize()
+            if k == 1:
+                g.profile(True)                    # timing on: this entry point must still create no event
+            free_before = torch.cuda.mem_get_info()[0]
             g.propagate_static(x.data_ptr(), width, got.data_ptr())
             torch.cuda.synchronize()
+            # the property the entry point exists for: the device's free memory is the same after the call
+            # (the first call came before this measurement only in so far as k = 0 did the address look-up)
+            assert torch.cuda.mem_get_info()[0] == free_before or k == 0, width
+            if k == 1:
+                assert not any(name.startswith("spmm") or name == "permute_rows" for name in g.profile_read())
+                g.profile(False)
             err = (got - want).norm() / want.norm()
             assert torch.isfinite(got).all()
             assert float(err) < 2e-7, (width, float(err))
+        # an absurd width is refused before any size arithmetic
+        with pytest.raises(binding.GcnAdmmError) as e:
+            g.propagate_static(x.data_ptr(), (1 << 31) - 2, got.data_ptr())
+        assert e.value.code == -1
         # a size beyond the built-in memory is refused with a message that names the limit
         big = 4_194_304 // wl.n + 8
         x = torch.zeros(wl.n, big, device="cuda")
