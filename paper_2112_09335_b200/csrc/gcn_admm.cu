@@ -29,7 +29,8 @@ constexpr int kLogPasses = 256;
 constexpr int kSmCount = 148;
 constexpr long long kImageMinRows = 16384;   // row count from which the weight operand is pre-split
 constexpr int kZBlockRows = 32;      // rows per block of the hidden-layer gradient's closing sweep
-constexpr int kCandZ = 2;           // theta candidates scored per sweep (tau: gk::kCand)
+constexpr int kChunksPerGroup = 256; // chunks whose sums one block of k_reduce_chunks adds up
+constexpr int kCandZ = 4;           // theta candidates scored per sweep (2..4; steady-state searches close at trial 0..2)
 constexpr int kDefaultLongRow = 256;   // stored entries one warp walks before a row is cut into items
 
 thread_local std::string g_create_error;
@@ -166,12 +167,21 @@ struct gcn_admm {
   float* part = nullptr;     // split partial sums of the transposed product
   size_t part_elems = 0;
   SearchCtl *ctl_w = nullptr, *ctl_z = nullptr;   // [L+1], [(L+1) * M]
-  double *sums_w = nullptr, *sums_z = nullptr, *acc_z = nullptr, *obj = nullptr;
+  double *sums_w = nullptr, *sums_z = nullptr, *obj = nullptr;
   double* red_part = nullptr;               // per-block partial sums awaiting their fixed-order reduction
   int2* d_zblocks = nullptr;                // row blocks of at most kZBlockRows rows, none crossing a community
   int* d_comm_block_ptr = nullptr;          // [M+1] first row block of every community
   int n_zblocks = 0;
-  int *n_active = nullptr, *status = nullptr, *row_counter = nullptr, *d_pass = nullptr;
+  int *n_active = nullptr, *status = nullptr, *d_pass = nullptr;
+  // Z scoring: units in chunks of about equally many stored entries, dealt to the warps of the grid in a fixed order
+  int* d_chunk_ptr = nullptr;
+  int n_chunks = 0;
+  double* z_chunk_part = nullptr;           // [chunk][M][candidates] sums of one sweep, per chunk of units
+  double* z_group_part = nullptr;           // [group of chunks][M][candidates], chunks added in order
+  int* chunk_counter = nullptr;             // hands the chunks out to the warps of a sweep
+  int n_groups = 0;
+  double* split_scores = nullptr;           // [n_split][candidates] sums of the segments scored in pieces
+  int *d_split_order = nullptr, *d_split_ptr = nullptr;   // split entries grouped by community
   cudaGraphExec_t pass_graph = nullptr;   // one pass of Algorithm 1, recorded once and replayed
   int *log_trial_w = nullptr, *log_trial_z = nullptr;
   double *log_q_w = nullptr, *log_q_z = nullptr;
@@ -466,7 +476,7 @@ struct gcn_admm {
     {
       Scope sc(this, "small", 1, 0.0, 0.0);
       gk::k_search_begin_z<<<(unsigned)cdiv((long long)M * 32, 128), 128, 0, stream>>>(
-          ctl, M, red_part, d_comm_block_ptr, sums_z, p.bt_shrink, p.bt_growth, acc_z, per, n_active, status);
+          ctl, M, red_part, d_comm_block_ptr, sums_z, p.bt_shrink, p.bt_growth, n_active, status);
       CU(cudaGetLastError());
     }
     gemm_nn(B2, ldl, W[l + 1], ldn, Wt[l + 1], ldl, B1, ldn, n, C[l + 1], C[l]);         // T = G W_{l+1}
@@ -480,37 +490,45 @@ struct gcn_admm {
     const size_t smem = (size_t)warps * M * per * sizeof(double);
     const int use_smem = smem <= 96 * 1024;
     const size_t dyn = use_smem ? smem : 0;
+    // after a sweep: the chunks' sums are added group by group, in chunk order (first stage of the ordered sum)
+    auto reduce_chunks = [&]() {
+      gk::k_reduce_chunks<<<(unsigned)n_groups, 256, 0, stream>>>(z_chunk_part, n_chunks, kChunksPerGroup, M * per,
+                                                                  z_group_part, n_active);
+      ++launches;
+    };
 #define SCORE_Z_U(V, OUT, UNZ)                                                                                 \
   {                                                                                                       \
     const size_t dynv = dyn + (size_t)warps * 2 * (V) * 32 * sizeof(float4);   /* per-warp copy of the row's a, b */ \
     if (dynv > 48 * 1024)                                                                                 \
       CU(cudaFuncSetAttribute(gk::k_score_z<V, OUT, UNZ, kCandZ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dynv)); \
-    CU(cudaMemsetAsync(row_counter, 0, sizeof(int), stream));                                             \
     int occ = 1;                                                                                          \
     CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gk::k_score_z<V, OUT, UNZ, kCandZ>, warps * 32, dynv));     \
-    const unsigned grid = (unsigned)std::min<long long>(cdiv(n + n_items, warps), (long long)kSmCount * std::max(occ, 1)); \
+    const unsigned grid = (unsigned)std::min<long long>(cdiv(n_chunks, warps), (long long)kSmCount * std::max(occ, 1)); \
+    CU(cudaMemsetAsync(chunk_counter, 0, sizeof(int), stream));                                           \
     gk::k_score_z<V, OUT, UNZ, kCandZ><<<grid, warps * 32, dynv, stream>>>(d_row_ptr, d_col, d_col_comm, d_dinv,       \
         (const float4*)B1, (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0, ld4, (int)n, ctl, M, \
-        acc_z, n_active, use_smem, row_counter, d_items, n_items, long_len, reinterpret_cast<float4*>(item_sums)); \
+        z_chunk_part, n_active, use_smem, d_chunk_ptr, n_chunks, chunk_counter, d_items, n_items, long_len,      \
+        reinterpret_cast<float4*>(item_sums));                                                            \
+    reduce_chunks();                                                                                      \
     if (n_split > 0) {                                                                                    \
       gk::k_score_z_split<V, OUT, kCandZ><<<(unsigned)cdiv(n_split, warps), warps * 32, 0, stream>>>(d_split, n_split, d_dinv, \
           reinterpret_cast<const float4*>(item_sums), (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0, \
-          ld4, ctl, acc_z, n_active);                                                                     \
+          ld4, ctl, split_scores, n_active);                                                              \
       ++launches;                                                                                         \
     }                                                                                                     \
   }
-#define SCORE_Z(V, OUT)                                     \
-  {                                                         \
-    if (OUT) SCORE_Z_U(V, OUT, 4)                           \
-    else SCORE_Z_U(V, OUT, 4)                               \
+#define SCORE_Z_ANY(OUT)                        \
+  {                                             \
+    if (ld4 <= 32) SCORE_Z_U(1, OUT, 4)         \
+    else if (ld4 <= 64) SCORE_Z_U(2, OUT, 4)    \
+    else if (ld4 <= 128) SCORE_Z_U(4, OUT, 4)   \
+    else SCORE_Z_U(8, OUT, 4)                   \
   }
-#define SCORE_Z_ANY(OUT)                    \
-  {                                         \
-    if (ld4 <= 32) SCORE_Z(1, OUT)          \
-    else if (ld4 <= 64) SCORE_Z(2, OUT)     \
-    else if (ld4 <= 128) SCORE_Z(4, OUT)    \
-    else SCORE_Z(8, OUT)                    \
-  }
+    auto decide = [&](const gk::DecideArgs& args) {
+      Scope sc(this, "small", 1, 0.0, 0.0);
+      gk::k_search_decide_z<<<(unsigned)cdiv((long long)M * 32, 128), 128, 0, stream>>>(
+          ctl, M, z_group_part, n_groups, per, split_scores, d_split_order, d_split_ptr, sums_z, args, n_active, status);
+    };
     char zname[48];
     std::snprintf(zname, sizeof zname, out ? "score_z_out@%d" : "score_z_hidden@%d", ldn);
     const std::string zretry = std::string(zname) + ".retry";
@@ -519,23 +537,22 @@ struct gcn_admm {
     if (out) {
       {
         Scope sc(this, zname, 1, zbytes, 2.0 * (double)gi.nnz * ldn);
-        if (ld4 <= 16) {   // narrow output layer: two rows per warp (see k_score_z_out_half)
-          const size_t smem_h = (size_t)2 * warps * M * 2 * sizeof(double);
-          const int use_smem_h = smem_h <= 96 * 1024;
-          const size_t dyn_h = use_smem_h ? smem_h : 0;
-          if (dyn_h > 48 * 1024)
-            CU(cudaFuncSetAttribute(gk::k_score_z_out_half<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_h));
-          CU(cudaMemsetAsync(row_counter, 0, sizeof(int), stream));
+        const size_t smem_h = (size_t)2 * warps * M * 2 * sizeof(double);
+        if (ld4 <= 16 && smem_h <= 96 * 1024) {   // narrow output layer: two rows per warp (see k_score_z_out_half)
+          if (smem_h > 48 * 1024)
+            CU(cudaFuncSetAttribute(gk::k_score_z_out_half<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_h));
           int occ = 1;
-          CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gk::k_score_z_out_half<4>, warps * 32, dyn_h));
-          const unsigned grid = (unsigned)std::min<long long>(cdiv(n + n_items, 2 * warps), (long long)kSmCount * std::max(occ, 1));
-          gk::k_score_z_out_half<4><<<grid, warps * 32, dyn_h, stream>>>(d_row_ptr, d_col, d_col_comm, d_dinv,
-              (const float4*)B1, (const float4*)B0, ld4, (int)n, ctl, M, acc_z, n_active, use_smem_h, row_counter, d_items,
-              n_items, long_len, reinterpret_cast<float4*>(item_sums));
+          CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gk::k_score_z_out_half<4>, warps * 32, smem_h));
+          const unsigned grid = (unsigned)std::min<long long>(cdiv(n_chunks, warps), (long long)kSmCount * std::max(occ, 1));
+          CU(cudaMemsetAsync(chunk_counter, 0, sizeof(int), stream));
+          gk::k_score_z_out_half<4><<<grid, warps * 32, smem_h, stream>>>(d_row_ptr, d_col, d_col_comm, d_dinv,
+              (const float4*)B1, (const float4*)B0, ld4, (int)n, ctl, M, z_chunk_part, n_active, d_chunk_ptr, n_chunks,
+              chunk_counter, d_items, n_items, long_len, reinterpret_cast<float4*>(item_sums));
+          reduce_chunks();
           if (n_split > 0) {
             gk::k_score_z_split<1, true, kCandZ><<<(unsigned)cdiv(n_split, warps), warps * 32, 0, stream>>>(d_split, n_split, d_dinv,
                 reinterpret_cast<const float4*>(item_sums), (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0,
-                ld4, ctl, acc_z, n_active);
+                ld4, ctl, split_scores, n_active);
             ++launches;
           }
         } else {
@@ -545,8 +562,7 @@ struct gcn_admm {
       a.mode = 1;
       a.quad_coef = 0.5 * p.rho;
       a.last_pass = 1;
-      Scope sc(this, "small", 1, 0.0, 0.0);
-      gk::k_search_decide<<<(unsigned)cdiv(M, 128), 128, 0, stream>>>(ctl, M, acc_z, per, sums_z, 3, a, n_active, status);
+      decide(a);
     } else {
       a.mode = 0;
       a.scale = 0.5 * p.nu;
@@ -558,13 +574,10 @@ struct gcn_admm {
           SCORE_Z_ANY(false)
         }
         a.last_pass = (ps == passes - 1);
-        Scope sc(this, "small", 1, 0.0, 0.0);
-        gk::k_search_decide<<<(unsigned)cdiv(M, 128), 128, 0, stream>>>(ctl, M, acc_z, per, sums_z, 3, a, n_active,
-                                                                        status);
+        decide(a);
       }
     }
 #undef SCORE_Z_ANY
-#undef SCORE_Z
 #undef SCORE_Z_U
     CU(cudaGetLastError());
     {
@@ -854,6 +867,39 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
     h->n_long = (int)lt.rows.size();
     h->d_items = reinterpret_cast<int4*>(upload(h, lt.items));
     h->d_split = reinterpret_cast<int4*>(upload(h, lt.split));
+    {   // split entries grouped by community (stable), for the ordered sums of k_search_decide_z
+      std::vector<int> sptr((size_t)n_comm + 1, 0), order(lt.split.size());
+      for (const auto& q : lt.split) ++sptr[(size_t)q.y + 1];
+      for (int m = 0; m < n_comm; ++m) sptr[m + 1] += sptr[m];
+      std::vector<int> at(sptr.begin(), sptr.end() - 1);
+      for (size_t k = 0; k < lt.split.size(); ++k) order[(size_t)at[lt.split[k].y]++] = (int)k;
+      h->d_split_order = upload(h, order);
+      h->d_split_ptr = upload(h, sptr);
+      h->split_scores = h->alloc<double>(std::max<size_t>(1, lt.split.size() * gk::kCand));
+    }
+    {   // chunks of units (items first, then rows) holding about the same number of stored entries each
+      const long long n_units = (long long)lt.items.size() + n;
+      const long long warps_guess = (long long)kSmCount * 3 * 8;
+      // few enough chunks that their sums (M x candidates doubles each) stay small next to the entries they cover
+      const long long target = std::max<long long>({64, std::min<long long>(1024, (long long)g.nnz / (warps_guess * 16)), 16LL * n_comm});
+      std::vector<int> cp;
+      cp.push_back(0);
+      long long in_chunk = 0;
+      for (long long u = 0; u < n_units; ++u) {
+        long long len;
+        if (u < (long long)lt.items.size()) len = lt.items[(size_t)u].z - lt.items[(size_t)u].y;
+        else {
+          const long long r = u - (long long)lt.items.size();
+          len = g.row_ptr[r + 1] - g.row_ptr[r];
+          if (len > h->long_len) len = 0;                 // walked as items
+        }
+        in_chunk += len + 2;                              // a unit costs a little even when it is short
+        if (in_chunk >= target) { cp.push_back((int)(u + 1)); in_chunk = 0; }
+      }
+      if (cp.back() != (int)n_units) cp.push_back((int)n_units);
+      h->n_chunks = (int)cp.size() - 1;
+      h->d_chunk_ptr = upload(h, cp);
+    }
     h->d_long_rows = reinterpret_cast<int4*>(upload(h, lt.rows));
   }
 
@@ -896,7 +942,6 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
   h->ctl_z = h->alloc<SearchCtl>((size_t)(L + 1) * n_comm);
   h->sums_w = h->alloc<double>(2);
   h->sums_z = h->alloc<double>((size_t)3 * n_comm);
-  h->acc_z = h->alloc<double>((size_t)gk::kCand * n_comm);
   h->obj = h->alloc<double>(8);
   {   // row blocks of the hidden-layer gradient's closing sweep, cut at community boundaries
     std::vector<int2> zb;
@@ -911,11 +956,14 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
     h->d_zblocks = upload(h, zb);
     h->d_comm_block_ptr = upload(h, cbp);
   }
+  h->n_groups = (int)cdiv(h->n_chunks, kChunksPerGroup);
+  h->z_chunk_part = h->alloc<double>((size_t)h->n_chunks * n_comm * gk::kCand);
+  h->z_group_part = h->alloc<double>((size_t)h->n_groups * n_comm * gk::kCand);
+  h->chunk_counter = h->alloc<int>(1);
   h->red_part = h->alloc<double>(std::max<size_t>({(size_t)kSmCount * 8 * gk::kCand, (size_t)h->n_zblocks * 3,
                                                    (size_t)cdiv(n, 8) * 2}));
   h->n_active = h->alloc<int>(1);
   h->status = h->alloc<int>(1);
-  h->row_counter = h->alloc<int>(1);
   h->d_pass = h->alloc<int>(1);
   CU(cudaMemset(h->d_pass, 0, sizeof(int)));
   h->log_trial_w = h->alloc<int>((size_t)kLogPasses * L);

@@ -593,11 +593,10 @@ __global__ void k_search_begin(SearchCtl* ctl, const double* __restrict__ sums, 
 // Starts the searches of the `count` communities of a hidden layer, one warp each.  k_zgrad_finish left
 // three sums per row block in `partial`; the blocks of community i are block_ptr[i] .. block_ptr[i+1]-1
 // and are added up in a fixed order (lane-strided, then the shuffle tree).  sums[i*3 + ..] receives
-// { ||G_i||^2, ||Z_i||^2, <Z_i - f(H_i), G_i> }; acc (acc_per doubles per community) is cleared.
+// { ||G_i||^2, ||Z_i||^2, <Z_i - f(H_i), G_i> }.
 __global__ void k_search_begin_z(SearchCtl* ctl, int count, const double* __restrict__ partial,
                                  const int* __restrict__ block_ptr, double* __restrict__ sums, double shrink,
-                                 double growth, double* __restrict__ acc, int acc_per, int* __restrict__ n_active,
-                                 int* __restrict__ status) {
+                                 double growth, int* __restrict__ n_active, int* __restrict__ status) {
   const int lane = threadIdx.x & 31;
   const int i = (int)(((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
   if (i >= count) return;
@@ -608,7 +607,6 @@ __global__ void k_search_begin_z(SearchCtl* ctl, int count, const double* __rest
   s0 = warp_sum(s0); s1 = warp_sum(s1); s2 = warp_sum(s2);
   if (lane != 0) return;
   sums[i * 3] = s0; sums[i * 3 + 1] = s1; sums[i * 3 + 2] = s2;
-  for (int j = 0; j < acc_per; ++j) acc[i * acc_per + j] = 0.0;
   begin_one(ctl + i, s0, s1, shrink, growth, n_active, status);
 }
 
@@ -681,17 +679,49 @@ __device__ __forceinline__ bool decide_one(SearchCtl* c, const double* __restric
   return true;
 }
 
-// Decisions of `count` searches whose pass sums are in acc (acc_per doubles each).
-__global__ void k_search_decide(SearchCtl* ctl, int count, double* __restrict__ acc, int acc_per,
-                                const double* __restrict__ own, int own_stride, DecideArgs a,
-                                int* __restrict__ n_active, int* __restrict__ status) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+// Sums of a scoring sweep, first stage: group g adds the chunks g*per_group .. (g+1)*per_group - 1 in chunk
+// order, value by value (width = communities x sums per community): group_part[g][v] = sum_ch chunk_part[ch][v].
+__global__ void k_reduce_chunks(const double* __restrict__ chunk_part, int n_chunks, int per_group, int width,
+                                double* __restrict__ group_part, const int* __restrict__ n_active) {
+  if (*n_active <= 0) return;
+  const int c0 = blockIdx.x * per_group, c1 = min(n_chunks, c0 + per_group);
+  for (int v = threadIdx.x; v < width; v += blockDim.x) {
+    double s = 0.0;
+    for (int ch = c0; ch < c1; ++ch) s += chunk_part[(size_t)ch * width + v];
+    group_part[(size_t)blockIdx.x * width + v] = s;
+  }
+}
+
+// Decisions of the `count` communities of a hidden layer, one warp each.  k_reduce_chunks left the sweep's
+// sums in block_part[(b*count + i)*per + j], b < n_blocks; they are added in a fixed order (lane-strided
+// over b, then the shuffle tree), followed by the sums of the segments scored in pieces
+// (split_scores, in the order split_order lists those of community i: split_ptr[i] .. split_ptr[i+1]-1).
+// own[i*3 + 2] = <Z_i - f(H_i), G_i>.
+__global__ void k_search_decide_z(SearchCtl* ctl, int count, const double* __restrict__ block_part, int n_blocks,
+                                  int per, const double* __restrict__ split_scores,
+                                  const int* __restrict__ split_order, const int* __restrict__ split_ptr,
+                                  const double* __restrict__ own, DecideArgs a, int* __restrict__ n_active,
+                                  int* __restrict__ status) {
+  const int lane = threadIdx.x & 31;
+  const int i = (int)(((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
   if (i >= count) return;
   SearchCtl* c = ctl + i;
   if (c->done) return;
-  const double sag = (a.own_nu != 0.0) ? own[i * own_stride + 2] : 0.0;
-  if (decide_one(c, acc + i * acc_per, sag, a, n_active, status))
-    for (int j = 0; j < acc_per; ++j) acc[i * acc_per + j] = 0.0;
+  double s[kCand];
+#pragma unroll
+  for (int j = 0; j < kCand; ++j) s[j] = 0.0;
+  for (int b = lane; b < n_blocks; b += 32)
+#pragma unroll
+    for (int j = 0; j < kCand; ++j)
+      if (j < per) s[j] += block_part[((size_t)b * count + i) * per + j];
+#pragma unroll
+  for (int j = 0; j < kCand; ++j) s[j] = warp_sum(s[j]);
+  if (lane != 0) return;
+  for (int k = split_ptr[i]; k < split_ptr[i + 1]; ++k)
+#pragma unroll
+    for (int j = 0; j < kCand; ++j)
+      if (j < per) s[j] += split_scores[(size_t)split_order[k] * per + j];
+  decide_one(c, s, own[i * 3 + 2], a, n_active, status);
 }
 
 // Decision of a W block: the `n_part` blocks of the scoring kernel left `per` sums each in `partial`;
@@ -821,15 +851,14 @@ __device__ __forceinline__ float warp_sum2(float v0, float v1, int lane) {
 // which is non-zero on V_m and its first-order neighbour rows only.  A warp owns row i and walks
 // its stored entries once; col_comm gives the community of every entry, entries of one community
 // are contiguous (ascending columns), and at every change of community the finished K_m[i] is scored:
-//   OUT = false (layer l+1 < L, ReLU):  acc[m*NC + j] += sum_c (z - f(h - k/t_j))^2 - (z - f(h))^2, j < NC
-//                                        (NC = candidates scored per sweep, 2 or 4: almost every search
-//                                        closes at its first or second trial, and a candidate costs two
-//                                        instructions per element, so the first sweep scores two and the
-//                                        rare search that needs more is served by a further sweep)
-//   OUT = true  (layer l+1 = L):        acc[m*2] += <k, R'>, acc[m*2+1] += ||k||^2   (closed form)
-// Sums are kept per warp in shared memory (no atomics on the hot path) and added to `acc` once per
-// block; with too many communities for that (use_smem == 0) they go to `acc` directly.
-// V = float4 columns per lane (width <= 128 V).  Persistent grid; `row_counter` must be zero at launch.
+//   OUT = false (layer l+1 < L, ReLU):  per community, sum_c (z - f(h - k/t_j))^2 - (z - f(h))^2 for j < NC
+//                                        (NC = candidates scored per sweep, 2..4: a candidate costs two
+//                                        instructions per element, and a search that needs more trials
+//                                        than one sweep scores is served by a further sweep)
+//   OUT = true  (layer l+1 = L):        sums <k, R'> and ||k||^2 per community   (closed form)
+// Sums are kept per warp in shared memory (no atomics on the hot path) and leave the kernel per chunk of
+// units (see the scheduling note in the kernel).  V = float4 columns per lane (width <= 128 V).
+// Persistent grid.
 //
 // Rows longer than `long_len` come as `n_items` items {row, first entry, one past the last, split}
 // (see k_spmm): an item of whole community segments (split < 0) is scored like a short row; an
@@ -842,11 +871,17 @@ __device__ __forceinline__ float4 twice_error(const float4& h, const float4& z) 
 }
 
 // Scores one finished K_m[i] (k, still without the factor di) against the row's a, b:
-// OUT: a = R'; else a = h and b = twice_error(h, z).
+// OUT: a = R'; else a = h and b = twice_error(h, z).  The sums (2 when OUT, else NC) go to `slots`:
+// how = 0 added by plain stores (the slots belong to this warp), 1 added atomically, 2 stored.
+__device__ __forceinline__ void put_sum(double* dst, float r, int how) {
+  if (how == 0) *dst += (double)r;
+  else if (how == 1) atomicAdd(dst, (double)r);
+  else *dst = (double)r;
+}
 template <int V, bool OUT, int NC>
 __device__ __forceinline__ void score_segment(const float4 (&k)[V], float di, const float4 (&a)[V],
                                               const float4 (&b)[V], const SearchCtl* __restrict__ ctl,
-                                              int cur, int lane, double* mine, bool plain_add) {
+                                              int cur, int lane, double* slots, int how) {
   if (OUT) {
     float p1 = 0.f, p2 = 0.f;
 #pragma unroll
@@ -856,12 +891,9 @@ __device__ __forceinline__ void score_segment(const float4 (&k)[V], float di, co
       p2 += kx * kx + ky * ky + kz * kz + kw * kw;
     }
     const float r = warp_sum2(p1, p2, lane);
-    if ((lane & 15) == 0) {
-      double* dst = mine + cur * 2 + (lane >> 4);
-      if (plain_add) *dst += (double)r; else atomicAdd(dst, (double)r);
-    }
+    if ((lane & 15) == 0) put_sum(slots + (lane >> 4), r, how);
   } else {
-    static_assert(NC == 2 || NC == 4, "two or four candidates per sweep");
+    static_assert(NC >= 2 && NC <= 4, "two to four candidates per sweep");
     float inv[NC], part[NC];
 #pragma unroll
     for (int j = 0; j < NC; ++j) { inv[j] = di * ctl[cur].inv_cand[j]; part[j] = 0.f; }   // K_m[i] = di * k
@@ -880,18 +912,12 @@ __device__ __forceinline__ void score_segment(const float4 (&k)[V], float di, co
         }
       }
     }
-    if constexpr (NC == 4) {
-      const float r = warp_sum4(part[0], part[1], part[2], part[3], lane);
-      if ((lane & 7) == 0) {
-        double* dst = mine + cur * NC + (lane >> 3);
-        if (plain_add) *dst += (double)r; else atomicAdd(dst, (double)r);
-      }
+    if constexpr (NC >= 3) {
+      const float r = warp_sum4(part[0], part[1], part[2], NC == 4 ? part[NC - 1] : 0.f, lane);
+      if ((lane & 7) == 0 && (lane >> 3) < NC) put_sum(slots + (lane >> 3), r, how);
     } else {
       const float r = warp_sum2(part[0], part[1], lane);
-      if ((lane & 15) == 0) {
-        double* dst = mine + cur * NC + (lane >> 4);
-        if (plain_add) *dst += (double)r; else atomicAdd(dst, (double)r);
-      }
+      if ((lane & 15) == 0) put_sum(slots + (lane >> 4), r, how);
     }
   }
 }
@@ -902,7 +928,8 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
           const unsigned short* __restrict__ col_comm, const float* __restrict__ dinv,
           const float4* __restrict__ T, const float4* __restrict__ Hn, const float4* __restrict__ Zn,
           const float4* __restrict__ Rn, int ld4, int n, const SearchCtl* __restrict__ ctl, int n_comm,
-          double* __restrict__ acc, const int* __restrict__ n_active, int use_smem, int* __restrict__ row_counter,
+          double* __restrict__ chunk_part, const int* __restrict__ n_active, int use_smem,
+          const int* __restrict__ chunk_ptr, int n_chunks, int* __restrict__ chunk_counter,
           const int4* __restrict__ items, int n_items, int long_len, float4* __restrict__ scratch) {
   if (*n_active <= 0) return;
   constexpr int PER = OUT ? 2 : NC;
@@ -913,26 +940,38 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
   const int warps_per_block = blockDim.x >> 5;
   float4* row_ab = s_raw + (size_t)warp * (2 * V * 32) + lane;
   double* s_acc = reinterpret_cast<double*>(s_raw + (size_t)warps_per_block * (2 * V * 32));
-  double* mine = acc;
+  double* mine = nullptr;   // the sums of the chunk in hand, [community][PER]
   if (use_smem) {
     for (int i = threadIdx.x; i < warps_per_block * n_comm * PER; i += blockDim.x) s_acc[i] = 0.0;
-    __syncthreads();
     mine = s_acc + (size_t)warp * n_comm * PER;
   }
-  const bool plain_add = use_smem != 0;
+  __syncthreads();
   const float4* __restrict__ T_lane = T + lane;   // rows of T are addressed by 32-bit float4 offsets (n * ld4 < 2^32)
   bool in_row[V];
 #pragma unroll
   for (int v = 0; v < V; ++v) in_row[v] = lane + 32 * v < ld4;
-  const int n_units = n + n_items;
-  // units (items first, then rows) are handed out four at a time from a global counter: row lengths
-  // follow a power law, a static deal leaves most warps waiting at the closing barrier for the unlucky ones
+  // Units (items first, then rows) come in chunks of about equally many stored entries (chunk_ptr, built
+  // on the host).  Chunks are handed out from a global counter (`chunk_counter`, zero at launch): row
+  // lengths follow a power law and the time a chunk takes depends on what its rows find in L2, so any
+  // static deal leaves most warps waiting for the unlucky ones.  A chunk is scored by one warp, units in
+  // order, and its sums go to chunk_part[chunk][community][PER]; they are added up in chunk order
+  // afterwards (k_reduce_chunks, k_search_decide_z), so no sum depends on which warp took which chunk.
+  // With room in shared memory the chunk's sums are kept there and copied out at the end of the chunk;
+  // otherwise (too many communities) the warp adds into the chunk's slice of chunk_part directly.
   for (;;) {
-    int unit_base = 0;
-    if (lane == 0) unit_base = atomicAdd(row_counter, 4);
-    unit_base = __shfl_sync(0xffffffffu, unit_base, 0);
-    if (unit_base >= n_units) break;
-    const int unit_end = min(n_units, unit_base + 4);
+    int ch = 0;
+    if (lane == 0) ch = atomicAdd(chunk_counter, 1);
+    ch = __shfl_sync(0xffffffffu, ch, 0);
+    if (ch >= n_chunks) break;
+    double* const out_part = chunk_part + (size_t)ch * n_comm * PER;
+    if (!use_smem) {
+      for (int i = lane; i < n_comm * PER; i += 32) out_part[i] = 0.0;
+      mine = out_part;
+      __syncwarp();
+    }
+    const int chunk_end = chunk_ptr[ch + 1];
+  for (int unit_base = chunk_ptr[ch]; unit_base < chunk_end; unit_base += 4) {
+    const int unit_end = min(chunk_end, unit_base + 4);
     // lanes 0..3 fetch the descriptions of the four units together (one load latency, not four)
     int4 my_unit = make_int4(0, 0, 0, -1);   // row, first entry, one past the last, split (>= 0: a piece)
     if (lane < 4 && unit_base + lane < unit_end) {
@@ -997,7 +1036,7 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
         a[v] = row_ab[32 * v];
         b[v] = OUT ? a[v] : row_ab[32 * (V + v)];
       }
-      score_segment<V, OUT, NC>(k, di, a, b, ctl, cur, lane, mine, plain_add);
+      score_segment<V, OUT, NC>(k, di, a, b, ctl, cur, lane, mine + cur * PER, 0);
     };
 
     // column and community of a chunk are fetched while the chunk before it is walked; the two
@@ -1024,6 +1063,14 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
       unsigned chg = __ballot_sync(0xffffffffu, valid && m != mprev);
       unsigned on = __ballot_sync(0xffffffffu, live);
       const int cnt = min(32, re - base);
+      if (on == 0u) {   // nothing to gather in this chunk (the usual case in a sweep after the first)
+        if (chg != 0u) {   // an open segment ends at the chunk's first entry; a later one starts from scratch
+          finish_segment();
+          cur = __shfl_sync(0xffffffffu, m, cnt - 1);
+          cur_on = false;
+        }
+        continue;
+      }
       for (int t = 0; t < cnt; t += UN, chg >>= UN, on >>= UN) {
         unsigned oj[UN];
         float wj[UN];
@@ -1059,13 +1106,10 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
     finish_segment();
   }
   }
-  if (use_smem) {
-    __syncthreads();
-    for (int i = threadIdx.x; i < n_comm * PER; i += blockDim.x) {
-      double t = 0.0;
-      for (int wq = 0; wq < warps_per_block; ++wq) t += s_acc[(size_t)wq * n_comm * PER + i];
-      if (t != 0.0) atomicAdd(acc + i, t);
-    }
+    __syncwarp();
+    if (use_smem)
+      for (int i = lane; i < n_comm * PER; i += 32) { out_part[i] = mine[i]; mine[i] = 0.0; }
+    __syncwarp();
   }
 }
 
@@ -1077,14 +1121,15 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
 // and no segment start), shuffles use width 16, and only the closing of a segment is a divergent
 // branch, inside which nothing is exchanged beyond the half's own 16 lanes.  Sums go to one array
 // per half-warp (the halves may close segments of the same community at the same time).
-// Dynamic shared memory: 2 x warps x n_comm x 2 doubles when use_smem != 0.
+// Dynamic shared memory: 2 x warps x n_comm x 2 doubles (the caller uses k_score_z when that does not fit).
 template <int UN>
 __global__ void __launch_bounds__(256, 4)
 k_score_z_out_half(const int* __restrict__ row_ptr, const int* __restrict__ col,
                    const unsigned short* __restrict__ col_comm, const float* __restrict__ dinv,
                    const float4* __restrict__ T, const float4* __restrict__ Rn, int ld4, int n,
-                   const SearchCtl* __restrict__ ctl, int n_comm, double* __restrict__ acc,
-                   const int* __restrict__ n_active, int use_smem, int* __restrict__ row_counter,
+                   const SearchCtl* __restrict__ ctl, int n_comm, double* __restrict__ chunk_part,
+                   const int* __restrict__ n_active, const int* __restrict__ chunk_ptr, int n_chunks,
+                   int* __restrict__ chunk_counter,
                    const int4* __restrict__ items, int n_items, int long_len, float4* __restrict__ scratch) {
   if (*n_active <= 0) return;
   static_assert(16 % UN == 0, "UN divides the chunk");
@@ -1092,26 +1137,23 @@ k_score_z_out_half(const int* __restrict__ row_ptr, const int* __restrict__ col,
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, half = lane >> 4, hl = lane & 15;
   const int warps_per_block = blockDim.x >> 5;
   const unsigned hmask = 0xffffu << (16 * half);
-  double* mine = acc;
-  if (use_smem) {
-    for (int i = threadIdx.x; i < 2 * warps_per_block * n_comm * 2; i += blockDim.x) s_half[i] = 0.0;
-    __syncthreads();
-    mine = s_half + (size_t)(2 * warp + half) * n_comm * 2;
-  }
-  const bool plain_add = use_smem != 0;
+  for (int i = threadIdx.x; i < 2 * warps_per_block * n_comm * 2; i += blockDim.x) s_half[i] = 0.0;
+  double* const mine = s_half + (size_t)(2 * warp + half) * n_comm * 2;   // the half-warp's sums of the chunk in hand
+  __syncthreads();
   const bool in_row = hl < ld4;
   const float4* __restrict__ T_lane = T + hl;
-  const int n_units = n + n_items;
-  for (;;) {
-    int unit_base = 0;
-    if (lane == 0) unit_base = atomicAdd(row_counter, 4);
-    unit_base = __shfl_sync(0xffffffffu, unit_base, 0);
-    if (unit_base >= n_units) break;
+  for (;;) {   // chunks from a global counter, their sums to chunk_part: see k_score_z
+    int ch = 0;
+    if (lane == 0) ch = atomicAdd(chunk_counter, 1);
+    ch = __shfl_sync(0xffffffffu, ch, 0);
+    if (ch >= n_chunks) break;
+    const int chunk_end = chunk_ptr[ch + 1];
+  for (int unit_base = chunk_ptr[ch]; unit_base < chunk_end; unit_base += 4) {
     for (int pair = 0; pair < 2; ++pair) {
       const int unit = unit_base + 2 * pair + half;
       int row = 0, rs = 0, re = 0;
       bool piece = false;
-      if (unit < n_units) {
+      if (unit < chunk_end) {
         if (unit < n_items) {
           const int4 it = items[unit];
           row = it.x; rs = it.y; re = it.z;
@@ -1143,10 +1185,7 @@ k_score_z_out_half(const int* __restrict__ row_ptr, const int* __restrict__ col,
         c += __shfl_xor_sync(hmask, c, 4, 16);
         c += __shfl_xor_sync(hmask, c, 2, 16);
         c += __shfl_xor_sync(hmask, c, 1, 16);
-        if ((hl & 7) == 0) {
-          double* dst = mine + cur * 2 + (hl >> 3);
-          if (plain_add) *dst += (double)c; else atomicAdd(dst, (double)c);
-        }
+        if ((hl & 7) == 0) put_sum(mine + cur * 2 + (hl >> 3), c, 0);
       };
 
       const int len = re - rs;
@@ -1170,8 +1209,17 @@ k_score_z_out_half(const int* __restrict__ row_ptr, const int* __restrict__ col,
         int mprev = __shfl_up_sync(0xffffffffu, m, 1, 16);
         if (hl == 0) mprev = cur;
         unsigned chg = (__ballot_sync(0xffffffffu, valid && m != mprev) >> (16 * half)) & 0xffffu;
-        unsigned on = (__ballot_sync(0xffffffffu, live) >> (16 * half)) & 0xffffu;
+        const unsigned on_both = __ballot_sync(0xffffffffu, live);
+        unsigned on = (on_both >> (16 * half)) & 0xffffu;
         const int cnt_max = min(16, len_max - o);
+        if (on_both == 0u) {   // neither half has anything to gather in this chunk
+          if (chg != 0u) {     // per half: an open segment ends at the chunk's first entry
+            finish_segment();
+            cur = __shfl_sync(hmask, m, min(16, len - o) - 1, 16);
+            cur_on = false;
+          }
+          continue;
+        }
         for (int t = 0; t < cnt_max; t += UN, chg >>= UN, on >>= UN) {
           unsigned oj[UN];
           float wj[UN];
@@ -1203,24 +1251,24 @@ k_score_z_out_half(const int* __restrict__ row_ptr, const int* __restrict__ col,
       __syncwarp();
     }
   }
-  if (use_smem) {
-    __syncthreads();
-    for (int i = threadIdx.x; i < n_comm * 2; i += blockDim.x) {
-      double t = 0.0;
-      for (int q = 0; q < 2 * warps_per_block; ++q) t += s_half[(size_t)q * n_comm * 2 + i];
-      if (t != 0.0) atomicAdd(acc + i, t);
-    }
+    // the chunk's sums: lower half-warp first, then the upper one
+    double* const lo = s_half + (size_t)(2 * warp) * n_comm * 2;
+    double* const hi = lo + (size_t)n_comm * 2;
+    double* const out_part = chunk_part + (size_t)ch * n_comm * 2;
+    for (int i = lane; i < n_comm * 2; i += 32) { out_part[i] = lo[i] + hi[i]; lo[i] = 0.0; hi[i] = 0.0; }
+    __syncwarp();
   }
 }
 
 // Segments that k_score_z handled in pieces: K_m[i] = sum of the pieces (item order), then scored
-// as above.  split[s] = {row, community, first item, number of items}; one warp per entry.
+// as above.  split[s] = {row, community, first item, number of items}; one warp per entry, whose sums
+// go to split_scores[s*PER ..] (PER = 2 when OUT, else NC); k_search_decide_z adds them in table order.
 template <int V, bool OUT, int NC>
 __global__ void __launch_bounds__(256)
 k_score_z_split(const int4* __restrict__ split, int n_split, const float* __restrict__ dinv,
                 const float4* __restrict__ scratch, const float4* __restrict__ Hn, const float4* __restrict__ Zn,
                 const float4* __restrict__ Rn, int ld4, const SearchCtl* __restrict__ ctl,
-                double* __restrict__ acc, const int* __restrict__ n_active) {
+                double* __restrict__ split_scores, const int* __restrict__ n_active) {
   if (*n_active <= 0) return;
   const int lane = threadIdx.x & 31;
   const int s = (int)(((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
@@ -1241,7 +1289,7 @@ k_score_z_split(const int4* __restrict__ split, int n_split, const float* __rest
       }
     }
   }
-  score_segment<V, OUT, NC>(k, dinv[sp.x], a, b, ctl, sp.y, lane, acc, false);
+  score_segment<V, OUT, NC>(k, dinv[sp.x], a, b, ctl, sp.y, lane, split_scores + (size_t)s * (OUT ? 2 : NC), 2);
 }
 
 // The rows of Eq. 7 without a loss term (not in the training set) have the closed form
