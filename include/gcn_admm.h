@@ -207,6 +207,28 @@ enum {
 };
 int gcn_admm_index(gcn_admm* h, int which, int comm, const int** data, long long* len);
 
+/* ---- plan for several GPUs (host only; Section 2: a community per agent; Appendix A, Eq. 4: the first-order
+ * messages p and the second-order messages s) ----------------------------------------------------
+ * This library runs a handle on one GPU and issues no collective.  For a caller that spreads the communities
+ * over n_ranks GPUs it plans the split: rank r owns a contiguous range of communities (hence of rows in the
+ * community order of gcn_admm_index), balanced by stored entries of A + I, and for every ordered pair
+ * (receiver, sender) the rows of the sender that the receiver depends on.
+ *  GCN_ADMM_SHARD_RANGES        [2 (n_ranks + 1)]: first community of every rank and one past the last,
+ *                               then first row of every rank and one past the last (receiver, sender ignored)
+ *  GCN_ADMM_SHARD_FIRST_ORDER   rows of `sender` adjacent to a row of `receiver`: the rows the receiver needs a
+ *                               copy of before a pass (Z_{l-1} for its propagation; H_{l+1}, Z_{l+1}, U for the
+ *                               gradient and the step-size search of its Z_{l,m} blocks).  The send list of
+ *                               (sender -> receiver) is this same list.
+ *  GCN_ADMM_SHARD_SECOND_ORDER  rows of `sender` that are neither the receiver's own nor first-order rows but
+ *                               adjacent to one: their Z_l reaches the receiver only through a neighbour's
+ *                               aggregate (the paper's second-order message); nothing is sent for them when
+ *                               owners compute H_{l+1} for their own rows.
+ * Lists are ascending new ids, owned by the handle, valid until the next call with another n_ranks or destroy.
+ * n_ranks must lie between 1 and the number of communities. */
+enum { GCN_ADMM_SHARD_RANGES = 0, GCN_ADMM_SHARD_FIRST_ORDER = 1, GCN_ADMM_SHARD_SECOND_ORDER = 2 };
+int gcn_admm_shard_plan(gcn_admm* h, int n_ranks, int which, int receiver, int sender, const int** data,
+                        long long* len);
+
 /* ---- state access (checkpointing and single-block tests) -------------------------------------
  * Host buffers, dense row-major, original node order.
  *  GCN_ADMM_ST_W      layer 1..L   float  C_{l-1} x C_l

@@ -19,6 +19,7 @@ EXPORTS = [
     "gcn_admm_predict", "gcn_admm_destroy", "gcn_admm_last_error", "gcn_admm_propagate", "gcn_admm_index",
     "gcn_admm_get_state", "gcn_admm_set_state", "gcn_admm_step_block", "gcn_admm_decisions",
     "gcn_admm_launches", "gcn_admm_profile", "gcn_admm_profile_read", "gcn_admm_propagate_static", "gcn_admm_dense_product", "gcn_admm_dense_product_tn",
+    "gcn_admm_shard_plan",
 ]
 
 IX = dict(perm=0, inv_perm=1, comm_ptr=2, nbr=3, halo1=4, halo2=5, csr_row_ptr=6, csr_col=7,
@@ -69,6 +70,7 @@ def load():
     lib.gcn_admm_dense_product.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32]
     lib.gcn_admm_dense_product_tn.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32]
     lib.gcn_admm_index.argtypes = [vp, i32, i32, C.POINTER(C.POINTER(i32)), C.POINTER(i64)]
+    lib.gcn_admm_shard_plan.argtypes = [vp, i32, i32, i32, i32, C.POINTER(C.POINTER(i32)), C.POINTER(i64)]
     lib.gcn_admm_get_state.argtypes = [vp, i32, i32, vp]
     lib.gcn_admm_set_state.argtypes = [vp, i32, i32, vp]
     lib.gcn_admm_step_block.argtypes = [vp, i32, i32]
@@ -200,6 +202,16 @@ class GcnAdmm:
         data = C.POINTER(C.c_int)()
         length = C.c_longlong()
         self._check(self._lib.gcn_admm_index(self._h, IX[which], int(comm), C.byref(data), C.byref(length)))
+        if length.value == 0:
+            return np.zeros(0, dtype=np.int32)
+        return np.ctypeslib.as_array(data, shape=(length.value,)).copy()
+
+    def shard_plan(self, n_ranks, which, receiver=0, sender=0):
+        """which: 0 ranges (first community / row of every rank, concatenated), 1 first-order rows, 2 second-order rows."""
+        data = C.POINTER(C.c_int)()
+        length = C.c_longlong()
+        self._check(self._lib.gcn_admm_shard_plan(self._h, int(n_ranks), int(which), int(receiver), int(sender),
+                                                  C.byref(data), C.byref(length)))
         if length.value == 0:
             return np.zeros(0, dtype=np.int32)
         return np.ctypeslib.as_array(data, shape=(length.value,)).copy()

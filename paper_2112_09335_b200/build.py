@@ -6,7 +6,7 @@ import subprocess
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 SOURCES = [os.path.join(HERE, "csrc", "gcn_admm.cu")]
-HEADERS = [os.path.join(HERE, "csrc", "kernels.cuh"), os.path.join(HERE, "csrc", "gemm_tc.cuh"), os.path.join(HERE, "csrc", "graph_index.hpp"),
+HEADERS = [os.path.join(HERE, "csrc", "kernels.cuh"), os.path.join(HERE, "csrc", "gemm_tc.cuh"), os.path.join(HERE, "csrc", "graph_index.hpp"), os.path.join(HERE, "csrc", "shard_plan.hpp"),
            os.path.join(os.path.dirname(HERE), "include", "gcn_admm.h")]
 LIB = os.path.join(HERE, "libgcn_admm.so")
 

@@ -19,6 +19,7 @@
 #include "gemm_tc.cuh"
 #include "graph_index.hpp"
 #include "kernels.cuh"
+#include "shard_plan.hpp"
 
 using gcn_admm_host::GraphIndex;
 using gk::SearchCtl;
@@ -190,6 +191,8 @@ struct gcn_admm {
   bool fresh = false;        // P_l, H_l agree with the stored W, Z
   std::string err;
   std::vector<int> ix_cache[16];
+  gcn_admm_host::ShardPlan shard_plan;      // last plan asked for (host only)
+  std::vector<int> shard_ranges;
 
   template <typename T>
   T* alloc(size_t count) {
@@ -1438,6 +1441,28 @@ int gcn_admm_index(gcn_admm* h, int which, int comm, const int** data, long long
         else c = gcn_admm_host::halo2_of(g, comm);
         v = &c;
       }
+    }
+    *data = v->data();
+    *len = (long long)v->size();
+  });
+}
+
+int gcn_admm_shard_plan(gcn_admm* h, int n_ranks, int which, int receiver, int sender, const int** data, long long* len) {
+  return guarded(h, [&] {
+    if (!data || !len || which < GCN_ADMM_SHARD_RANGES || which > GCN_ADMM_SHARD_SECOND_ORDER)
+      throw Fail{GCN_ADMM_ERR_ARG, "bad selector"};
+    if (h->shard_plan.n_ranks != n_ranks) {
+      if (!gcn_admm_host::build_shard_plan(h->gi, n_ranks, h->shard_plan))
+        throw Fail{GCN_ADMM_ERR_ARG, "n_ranks must be between 1 and the number of communities"};
+      h->shard_ranges = h->shard_plan.comm_begin;
+      h->shard_ranges.insert(h->shard_ranges.end(), h->shard_plan.row_begin.begin(), h->shard_plan.row_begin.end());
+    }
+    const std::vector<int>* v = &h->shard_ranges;
+    if (which != GCN_ADMM_SHARD_RANGES) {
+      if (receiver < 0 || receiver >= n_ranks || sender < 0 || sender >= n_ranks)
+        throw Fail{GCN_ADMM_ERR_ARG, "rank out of range"};
+      const auto& lists = which == GCN_ADMM_SHARD_FIRST_ORDER ? h->shard_plan.first_order : h->shard_plan.second_order;
+      v = &lists[(size_t)receiver * n_ranks + sender];
     }
     *data = v->data();
     *len = (long long)v->size();

@@ -140,3 +140,26 @@ def test_a_raised_pipeline_flag_surfaces_once_and_the_handle_stays_usable():
         assert np.isfinite(g.objective()).all()
     finally:
         g.destroy()
+
+
+def test_shard_plan_through_the_library():
+    """The multi-GPU plan (host logic, covered in depth on the CPU) as the library hands it out."""
+    from oracle import gcn_admm_oracle as orc
+    wl = inputs.make_workload(0)
+    g = make(wl)
+    try:
+        R = 2
+        ranges = g.shard_plan(R, 0)
+        comm_begin, row_begin = ranges[:R + 1], ranges[R + 1:]
+        ix = orc.community_index(wl.n, wl.row_ptr, wl.col_idx, wl.community, wl.n_comm)
+        assert np.array_equal(row_begin, ix["comm_ptr"][comm_begin]) and comm_begin[0] == 0 and comm_begin[-1] == wl.n_comm
+        for r in range(R):
+            h1 = np.unique(np.concatenate([ix["halo1"][m] for m in range(comm_begin[r], comm_begin[r + 1])]))
+            h1 = h1[(h1 < row_begin[r]) | (h1 >= row_begin[r + 1])]
+            got = np.concatenate([g.shard_plan(R, 1, r, s) for s in range(R)])
+            assert np.array_equal(np.sort(got), h1)
+            assert len(g.shard_plan(R, 1, r, r)) == 0
+        with pytest.raises(binding.GcnAdmmError):
+            g.shard_plan(wl.n_comm + 1, 0)
+    finally:
+        g.destroy()
