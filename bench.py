@@ -35,10 +35,18 @@ FP32_LANES_PER_SM = 128
 SM_COUNT = 148
 
 
-# DRAM bytes (read + write) per launch from the committed ncu capture of k_spmm at leading dimension 256 on the
-# workload's recipe at scale 0.1 (profiles/k_spmm_powerlaw_xlarge_scale0.1.md); a full-size launch is estimated by
-# the ratio of stored entries, since the excess traffic is neighbour rows that miss L2 (one per such entry).
-NCU_SPMM256 = dict(dram_bytes=1.461740e9 + 0.271949e9, nnz=2 * 5653426 + 244903)
+# DRAM bytes (read + write) per stored entry of A + I moved by one launch of the propagation at leading dimension
+# 256, from ncu (dram__bytes_read.sum + dram__bytes_write.sum) on this workload's recipe.  FULL: a one-pass capture
+# of a launch at full size (126,404,737 stored entries); SCALED: a capture at scale 0.25 (30,189,629 stored entries),
+# used for other sizes in proportion to the stored entries (the share of neighbour rows that miss L2 grows with
+# the size, so scaling up from 0.25 understates the traffic).
+NCU_SPMM256 = dict(
+    scaled=dict(dram_bytes=5066328832.0 + 715988992.0, nnz=30189629, scale=0.25),
+    full=dict(dram_bytes=34.20e9 + 3.03e9, nnz=126404737),
+)
+# SM-to-L2 fabric: ncu reports l1tex__m_xbar2l1tex_read_bytes at 51.2 % of its peak for 29.15 GB in 1.578 ms at
+# 1.906 GHz, i.e. a peak of 128 bytes per clock per SM
+XBAR_BYTES_PER_CLK_PER_SM = 128.0
 
 
 def measured_peaks():
@@ -112,20 +120,27 @@ def config_dict(wl, extra=None):
     return d
 
 
-def oracle_rate(index, scale, iters, warm):
-    """Seconds per oracle iteration on a scaled-down sample of workload `index`."""
+def oracle_rate(index, scale, iters, warm, threads=None):
+    """Seconds per oracle iteration on a scaled-down sample of workload `index` (optionally with the BLAS and
+    OpenMP pools limited to `threads`)."""
     from oracle import gcn_admm_oracle as orc
     from paper_2112_09335_b200 import inputs
     wl = inputs.make_workload(index, scale=scale)
-    o = orc.OracleADMM(wl.n, wl.row_ptr, wl.col_idx, wl.X, wl.y, wl.train_mask, wl.widths,
-                       orc.Params(nu=wl.nu, rho=wl.rho), wl.n_comm, wl.community, wl.w_init)
-    for _ in range(warm):
-        o.iterate()
-    t0 = time.perf_counter()
-    for _ in range(iters):
-        o.iterate()
-    dt = (time.perf_counter() - t0) / max(iters, 1)
-    return wl, dt
+
+    def run():
+        o = orc.OracleADMM(wl.n, wl.row_ptr, wl.col_idx, wl.X, wl.y, wl.train_mask, wl.widths,
+                           orc.Params(nu=wl.nu, rho=wl.rho), wl.n_comm, wl.community, wl.w_init)
+        for _ in range(warm):
+            o.iterate()
+        t0 = time.perf_counter()
+        for _ in range(iters):
+            o.iterate()
+        return (time.perf_counter() - t0) / max(iters, 1)
+    if threads is None:
+        return wl, run()
+    from threadpoolctl import threadpool_limits
+    with threadpool_limits(limits=threads):
+        return wl, run()
 
 
 def blas_threads():
@@ -136,27 +151,56 @@ def blas_threads():
         return os.cpu_count() or 1
 
 
+def oracle_baseline(index, full_nodes, full_edges, nodes=(1225, 2450, 4900), iters=1, warm=1):
+    """The oracle, as it stands, timed on this host at three sizes of the workload's recipe (all cores, and one
+    core at the smallest size), a power law t = a * edges^b fitted through the three points, and the rate that
+    fit gives at the full size.  Returns (iterations/s at full size, description, points)."""
+    pts = []
+    for k in nodes:
+        wl, dt = oracle_rate(index, min(1.0, k / full_nodes), iters, warm)
+        pts.append((wl.n, wl.n_edges, wl.n_comm, dt))
+    _, dt1 = oracle_rate(index, min(1.0, nodes[0] / full_nodes), 1, warm, threads=1)
+    e = np.log([q[1] for q in pts])
+    t = np.log([q[3] for q in pts])
+    b, a = np.polyfit(e, t, 1)
+    t_full = float(np.exp(a + b * np.log(full_edges)))
+    cores = blas_threads()
+    sample = (f"{iters} oracle iteration(s) (after {warm}) on the same recipe at "
+              + ", ".join(f"{q[0]} nodes / {q[1]} edges: {q[3]:.2f} s" for q in pts)
+              + f" per iteration on {cores} threads ({dt1:.2f} s on one thread at the smallest size); fitted "
+              f"t = a * edges^{b:.2f}; extrapolated to {full_edges} edges: {t_full:.3g} s per iteration "
+              f"(largest measured point: {pts[-1][3]:.2f} s at {pts[-1][1]} edges)")
+    return 1.0 / t_full, cores, sample, pts
+
+
 def run_reference(args):
-    """The fp64 CPU oracle, as it stands, on a bounded sample: the workload's recipe at 1/1000 of
-    its node and edge counts (same widths, same number of communities).  The figure is scaled to
-    the full workload in proportion to the edge count, which flatters the oracle (its cost grows
-    faster than linearly)."""
+    """The fp64 CPU oracle, as it stands, on a bounded sample: the workload's recipe at 2,450 nodes (same widths,
+    same number of communities) for the timed steps, plus one iteration each at half and twice that size to fit
+    how its cost grows; the printed value is the fitted cost at the full workload's edge count."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     from paper_2112_09335_b200 import inputs
-    scale = 0.001
     full = inputs.CONFIGS[WORKLOAD_INDEX]
+    scale = 2450.0 / full["n"]
     wl, dt = oracle_rate(WORKLOAD_INDEX, scale, args.steps, args.warmup)
-    frac = wl.n_edges / full["edges"]
-    value = (1.0 / dt) * frac
+    pts = [(wl.n_edges, dt)]
+    for k in (1225, 4900):
+        w2, d2 = oracle_rate(WORKLOAD_INDEX, k / full["n"], 1, 2)
+        pts.append((w2.n_edges, d2))
+    b, a = np.polyfit(np.log([q[0] for q in pts]), np.log([q[1] for q in pts]), 1)
+    t_full = float(np.exp(a + b * np.log(full["edges"])))
+    value = 1.0 / t_full
     cores = blas_threads()
-    sample = (f"oracle iteration on the same recipe at scale {scale} ({wl.n} nodes, {wl.n_edges} edges, "
-              f"{wl.n_comm} communities); rate multiplied by edge ratio {frac:.3e}")
+    sample = (f"{args.steps} oracle iterations (after {args.warmup}) on the same recipe at {wl.n} nodes / {wl.n_edges} edges / "
+              f"{wl.n_comm} communities: {dt:.2f} s each on {cores} threads; one iteration each at "
+              + ", ".join(f"{q[0]} edges: {q[1]:.2f} s" for q in pts[1:])
+              + f"; fitted t = a * edges^{b:.2f}, extrapolated to {full['edges']} edges")
     line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
-                warmup=args.warmup, ms_per_step=dt * 1e3 / frac, higher_is_better=True, scaling="weak",
+                warmup=args.warmup, ms_per_step=t_full * 1e3, higher_is_better=True, scaling="weak",
                 vs_baseline=None, dtype="f64", data="synthetic",
-                config=config_dict(wl, dict(workload=full["name"], sampled_as=wl.name)),
+                config=config_dict(wl, dict(workload=full["name"], sampled_as=wl.name,
+                                            measured_ms_per_step_on_sample=dt * 1e3)),
                 cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
     print(json.dumps(line))
@@ -303,19 +347,29 @@ def run_ours(args):
                     peak_source=(peaks["source"] if bound == "hbm" else
                                  "148 SMs x 128 fp32 lanes x 2 flop x max SM clock" if bound == "alu" else
                                  peaks["source"] + " bf16 x (1.1/2.25) / 3 passes"))
+    nnz_stored = 2 * wl.n_edges + wl.n
     if dominant["kernel"] == "spmm@256":
-        roofline["traffic"] = NCU_SPMM256["dram_bytes"] * (2 * wl.n_edges + wl.n) / NCU_SPMM256["nnz"]
-        roofline["note"] = ("gather kernel: every stored entry pulls a full operand row through L2 (nnz x ld x 4 B, about "
-                            "23x the algorithmic bytes at mean degree 50), so it runs at the L2-to-SM rate, not at the HBM "
-                            "rate; algorithmic bytes = 4 nnz + 8 N + 8 N ld")
+        cap = NCU_SPMM256["full"] if (NCU_SPMM256["full"] and args.scale == 1.0 and args.config == WORKLOAD_INDEX) else NCU_SPMM256["scaled"]
+        roofline["traffic"] = cap["dram_bytes"] * nnz_stored / cap["nnz"]
+        roofline["traffic_source"] = ("ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch at full size" if cap is NCU_SPMM256["full"]
+                                      else f"ncu capture of one launch at scale {cap['scale']} ({cap['nnz']} stored entries), scaled by stored entries")
+        per_launch = dominant["ms_per_iter"] / max(dominant["launches_per_iter"], 1e-9) * 1e-3
+        roofline["traffic_gbs"] = roofline["traffic"] / per_launch / 1e9
+        roofline["traffic_frac"] = roofline["traffic_gbs"] / peaks["hbm_gbs"]
+        roofline["note"] = ("gather kernel: every stored entry pulls a full operand row (nnz x ld x 4 B, about 23x the algorithmic "
+                            "bytes at mean degree 50); the 2.5 GB operand is 20x the L2, so about a quarter of the gathered rows "
+                            "come from DRAM: `traffic` (measured) is 6.7x the algorithmic bytes and moves at `traffic_frac` of "
+                            "the copy rate; algorithmic bytes = 4 nnz + 8 N + 8 N ld")
     if dominant["kernel"].startswith("spmm@"):
         # what the kernel pulls through L2: one operand row per stored entry of A + I
         ldw = int(dominant["kernel"].split("@")[1])
-        gathered = float(2 * wl.n_edges + wl.n) * ldw * 4.0
+        gathered = float(nnz_stored) * ldw * 4.0
         per_launch_s = dominant["ms_per_iter"] / max(dominant["launches_per_iter"], 1e-9) * 1e-3
+        clk = (clocks or {}).get("sm_mhz") or peaks["sm_max_mhz"]
+        xbar_peak = XBAR_BYTES_PER_CLK_PER_SM * SM_COUNT * clk * 1e6 / 1e9
         roofline["l2_gather"] = dict(bytes_per_launch=gathered, gbs=gathered / per_launch_s / 1e9,
-                                     ncu_l2_sector_rate_of_peak=0.79,
-                                     source="profiles/k_spmm_powerlaw_xlarge_scale0.1.md (lts__t_sectors_srcunit_tex)")
+                                     peak_gbs=xbar_peak, frac=gathered / per_launch_s / 1e9 / xbar_peak,
+                                     peak_source="128 B/clk/SM x 148 SMs x median SM clock of this run (ncu: l1tex__m_xbar2l1tex_read_bytes peak)")
     roofline.update(kernel=dominant["kernel"], ms_per_launch=dominant["ms_per_iter"] / max(dominant["launches_per_iter"], 1e-9),
                     share_of_kernel_time=dominant["share"])
 
@@ -335,13 +389,14 @@ def run_ours(args):
                 objective=dict(L_rho=obj[0], R=obj[1], train_acc=obj[5], exhausted_searches=exhausted,
                                e2e_L_rho=obj2[0]))
     if world == 1 and not args.no_cpu_baseline:
-        scale = min(1.0, 2450.0 / inputs.CONFIGS[args.config]["n"])      # about 2.4 k nodes of the same recipe
-        wl_s, dt = oracle_rate(args.config, scale, 3, 1)
-        frac = wl_s.n_edges / max(wl.n_edges, 1)
-        line["cpu_baseline"] = dict(value=(1.0 / dt) * frac, unit=UNIT, cores=blas_threads(), kind="oracle",
-                                    sample=(f"3 oracle iterations (after 1) on the same recipe at {wl_s.n} nodes / "
-                                            f"{wl_s.n_edges} edges / {wl_s.n_comm} communities, {dt:.2f} s each; rate "
-                                            f"multiplied by the edge ratio {frac:.3e} (linear scaling flatters the oracle)"))
+        full_cfg = inputs.CONFIGS[args.config]
+        if wl.n <= 6000:          # small workloads: the oracle runs the workload itself
+            _, dt = oracle_rate(args.config, args.scale, 2, 1)
+            line["cpu_baseline"] = dict(value=1.0 / dt, unit=UNIT, cores=blas_threads(), kind="oracle",
+                                        sample=f"2 oracle iterations (after 1) on the workload itself, {dt:.2f} s each")
+        else:
+            value_cpu, cores, sample, _ = oracle_baseline(args.config, full_cfg["n"], wl.n_edges)
+            line["cpu_baseline"] = dict(value=value_cpu, unit=UNIT, cores=cores, kind="oracle", sample=sample)
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

@@ -34,7 +34,7 @@ namespace gtc {
 constexpr int kBlockM = 128;
 constexpr int kChunkK = 32;                 // floats per K chunk (128 bytes)
 constexpr int kATileBytes = kBlockM * kChunkK * 4;     // 16 KiB, one of hi / lo
-constexpr uint32_t kSpinLimit = 4u << 20;
+constexpr long long kWaitClocks = 1LL << 31;   // bound of every mbarrier wait, in SM clocks (about a second)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -104,8 +104,11 @@ __device__ __forceinline__ uint32_t swz(int r, int c16) { return (uint32_t)r * 1
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// Waits for a phase, giving up when another role has raised the abort flag or after kWaitClocks (a try_wait
+// may itself suspend the thread for a while, so the bound is on elapsed clocks, not on attempts).
 __device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+  const long long t0 = clock64();
+  for (uint32_t i = 0;; ++i) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -115,7 +118,10 @@ __device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parit
         : "r"(bar), "r"(parity)
         : "memory");
     if (ok) return true;
-    if ((i & 255u) == 255u && *abort_flag) return false;
+    if ((i & 63u) == 63u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitClocks) break;
+    }
   }
   *abort_flag = 1;
   return false;
