@@ -183,24 +183,28 @@ def run_reference(args):
     from paper_2112_09335_b200 import inputs
     full = inputs.CONFIGS[WORKLOAD_INDEX]
     scale = 2450.0 / full["n"]
+    wl_full = inputs.make_workload(WORKLOAD_INDEX)            # only for the line's `config` (the other arm's workload)
+    full_config = config_dict(wl_full)
+    full_edges = wl_full.n_edges
+    del wl_full
     wl, dt = oracle_rate(WORKLOAD_INDEX, scale, args.steps, args.warmup)
     pts = [(wl.n_edges, dt)]
     for k in (1225, 4900):
         w2, d2 = oracle_rate(WORKLOAD_INDEX, k / full["n"], 1, 2)
         pts.append((w2.n_edges, d2))
     b, a = np.polyfit(np.log([q[0] for q in pts]), np.log([q[1] for q in pts]), 1)
-    t_full = float(np.exp(a + b * np.log(full["edges"])))
+    t_full = float(np.exp(a + b * np.log(full_edges)))
     value = 1.0 / t_full
     cores = blas_threads()
     sample = (f"{args.steps} oracle iterations (after {args.warmup}) on the same recipe at {wl.n} nodes / {wl.n_edges} edges / "
               f"{wl.n_comm} communities: {dt:.2f} s each on {cores} threads; one iteration each at "
               + ", ".join(f"{q[0]} edges: {q[1]:.2f} s" for q in pts[1:])
-              + f"; fitted t = a * edges^{b:.2f}, extrapolated to {full['edges']} edges")
+              + f"; fitted t = a * edges^{b:.2f}, extrapolated to {full_edges} edges")
     line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
                 warmup=args.warmup, ms_per_step=t_full * 1e3, higher_is_better=True, scaling="weak",
                 vs_baseline=None, dtype="f64", data="synthetic",
-                config=config_dict(wl, dict(workload=full["name"], sampled_as=wl.name,
-                                            measured_ms_per_step_on_sample=dt * 1e3)),
+                config=dict(full_config, sampled_as=f"{wl.name}: {wl.n} nodes, {wl.n_edges} edges",
+                            measured_ms_per_step_on_sample=dt * 1e3),
                 cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
     print(json.dumps(line))
