@@ -176,6 +176,9 @@ struct gcn_admm {
   int *n_active = nullptr, *status = nullptr, *d_pass = nullptr;
   // Z scoring: units in chunks of about equally many stored entries, dealt to the warps of the grid in a fixed order
   int* d_chunk_ptr = nullptr;
+  int* d_row_order = nullptr;               // rows per community by falling length: the order of the kernels that put several rows in a warp
+  int* d_chunk_ptr_sorted = nullptr;        // chunk table of the units in that order
+  int n_chunks_sorted = 0;
   int n_chunks = 0;
   double* z_chunk_part = nullptr;           // [chunk][M][candidates] sums of one sweep, per chunk of units
   double* z_group_part = nullptr;           // [group of chunks][M][candidates], chunks added in order
@@ -221,8 +224,9 @@ struct gcn_admm {
 #define SPMM_CASE(G, V, UN)                                                                    \
   {                                                                                            \
     const long long threads = (n + items_used) * (G);                                          \
-    gk::k_spmm<G, V, UN><<<(unsigned)cdiv(threads, 64), 64, 0, stream>>>(d_row_ptr, d_col, d_dinv, x4, o4, nn, ld4, \
-        d_items, items_used, cut ? long_len : INT_MAX, reinterpret_cast<float4*>(item_sums));  \
+    /* several rows per warp (G < 32): rows of equal length side by side */                     \
+    gk::k_spmm<G, V, UN, ((G) < 32)><<<(unsigned)cdiv(threads, 64), 64, 0, stream>>>(d_row_ptr, d_col, d_dinv, x4, o4, nn, ld4, \
+        d_items, items_used, cut ? long_len : INT_MAX, reinterpret_cast<float4*>(item_sums), d_row_order); \
   }
     if (ld4 <= 1) SPMM_CASE(1, 1, 4)
     else if (ld4 <= 2) SPMM_CASE(2, 1, 4)
@@ -494,9 +498,11 @@ struct gcn_admm {
     const int use_smem = smem <= 96 * 1024;
     const size_t dyn = use_smem ? smem : 0;
     // after a sweep: the chunks' sums are added group by group, in chunk order (first stage of the ordered sum)
-    auto reduce_chunks = [&]() {
-      gk::k_reduce_chunks<<<(unsigned)n_groups, 256, 0, stream>>>(z_chunk_part, n_chunks, kChunksPerGroup, M * per,
-                                                                  z_group_part, n_active);
+    int groups_used = 0;   // groups of chunks the last sweep filled (the chunk table depends on the kernel)
+    auto reduce_chunks = [&](int chunks) {
+      groups_used = (int)cdiv(chunks, kChunksPerGroup);
+      gk::k_reduce_chunks<<<(unsigned)groups_used, 256, 0, stream>>>(z_chunk_part, chunks, kChunksPerGroup, M * per,
+                                                                     z_group_part, n_active);
       ++launches;
     };
 #define SCORE_Z_U(V, OUT, UNZ)                                                                                 \
@@ -511,8 +517,8 @@ struct gcn_admm {
     gk::k_score_z<V, OUT, UNZ, kCandZ><<<grid, warps * 32, dynv, stream>>>(d_row_ptr, d_col, d_col_comm, d_dinv,       \
         (const float4*)B1, (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0, ld4, (int)n, ctl, M, \
         z_chunk_part, n_active, use_smem, d_chunk_ptr, n_chunks, chunk_counter, d_items, n_items, long_len,      \
-        reinterpret_cast<float4*>(item_sums));                                                            \
-    reduce_chunks();                                                                                      \
+        reinterpret_cast<float4*>(item_sums), nullptr);                                                         \
+    reduce_chunks(n_chunks);                                                                              \
     if (n_split > 0) {                                                                                    \
       gk::k_score_z_split<V, OUT, kCandZ><<<(unsigned)cdiv(n_split, warps), warps * 32, 0, stream>>>(d_split, n_split, d_dinv, \
           reinterpret_cast<const float4*>(item_sums), (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0, \
@@ -530,7 +536,7 @@ struct gcn_admm {
     auto decide = [&](const gk::DecideArgs& args) {
       Scope sc(this, "small", 1, 0.0, 0.0);
       gk::k_search_decide_z<<<(unsigned)cdiv((long long)M * 32, 128), 128, 0, stream>>>(
-          ctl, M, z_group_part, n_groups, per, split_scores, d_split_order, d_split_ptr, sums_z, args, n_active, status);
+          ctl, M, z_group_part, groups_used, per, split_scores, d_split_order, d_split_ptr, sums_z, args, n_active, status);
     };
     char zname[48];
     std::snprintf(zname, sizeof zname, out ? "score_z_out@%d" : "score_z_hidden@%d", ldn);
@@ -546,12 +552,12 @@ struct gcn_admm {
             CU(cudaFuncSetAttribute(gk::k_score_z_out_half<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_h));
           int occ = 1;
           CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gk::k_score_z_out_half<4>, warps * 32, smem_h));
-          const unsigned grid = (unsigned)std::min<long long>(cdiv(n_chunks, warps), (long long)kSmCount * std::max(occ, 1));
+          const unsigned grid = (unsigned)std::min<long long>(cdiv(n_chunks_sorted, warps), (long long)kSmCount * std::max(occ, 1));
           CU(cudaMemsetAsync(chunk_counter, 0, sizeof(int), stream));
           gk::k_score_z_out_half<4><<<grid, warps * 32, smem_h, stream>>>(d_row_ptr, d_col, d_col_comm, d_dinv,
-              (const float4*)B1, (const float4*)B0, ld4, (int)n, ctl, M, z_chunk_part, n_active, d_chunk_ptr, n_chunks,
-              chunk_counter, d_items, n_items, long_len, reinterpret_cast<float4*>(item_sums));
-          reduce_chunks();
+              (const float4*)B1, (const float4*)B0, ld4, (int)n, ctl, M, z_chunk_part, n_active, d_chunk_ptr_sorted, n_chunks_sorted,
+              chunk_counter, d_items, n_items, long_len, reinterpret_cast<float4*>(item_sums), d_row_order);
+          reduce_chunks(n_chunks_sorted);
           if (n_split > 0) {
             gk::k_score_z_split<1, true, kCandZ><<<(unsigned)cdiv(n_split, warps), warps * 32, 0, stream>>>(d_split, n_split, d_dinv,
                 reinterpret_cast<const float4*>(item_sums), (const float4*)H[l + 1], (const float4*)Z[l + 1], (const float4*)B0,
@@ -880,28 +886,43 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
       h->d_split_ptr = upload(h, sptr);
       h->split_scores = h->alloc<double>(std::max<size_t>(1, lt.split.size() * gk::kCand));
     }
-    {   // chunks of units (items first, then rows) holding about the same number of stored entries each
+    std::vector<int> row_order((size_t)n);
+    for (long long i = 0; i < n; ++i) row_order[(size_t)i] = (int)i;
+    for (int m = 0; m < n_comm; ++m)   // inside a community: longest rows first, ties by row id
+      std::stable_sort(row_order.begin() + g.comm_ptr[m], row_order.begin() + g.comm_ptr[m + 1], [&](int a, int b) {
+        return g.row_ptr[a + 1] - g.row_ptr[a] > g.row_ptr[b + 1] - g.row_ptr[b];
+      });
+    h->d_row_order = upload(h, row_order);
+    {   // chunks of units (items first, then rows) holding about the same number of stored entries each,
+        // once for rows in storage order and once for rows in the sorted order
       const long long n_units = (long long)lt.items.size() + n;
       const long long warps_guess = (long long)kSmCount * 3 * 8;
       // few enough chunks that their sums (M x candidates doubles each) stay small next to the entries they cover
       const long long target = std::max<long long>({64, std::min<long long>(1024, (long long)g.nnz / (warps_guess * 16)), 16LL * n_comm});
-      std::vector<int> cp;
-      cp.push_back(0);
-      long long in_chunk = 0;
-      for (long long u = 0; u < n_units; ++u) {
-        long long len;
-        if (u < (long long)lt.items.size()) len = lt.items[(size_t)u].z - lt.items[(size_t)u].y;
-        else {
-          const long long r = u - (long long)lt.items.size();
-          len = g.row_ptr[r + 1] - g.row_ptr[r];
-          if (len > h->long_len) len = 0;                 // walked as items
+      auto build_chunks = [&](const int* order) {
+        std::vector<int> cp;
+        cp.push_back(0);
+        long long in_chunk = 0;
+        for (long long u = 0; u < n_units; ++u) {
+          long long len;
+          if (u < (long long)lt.items.size()) len = lt.items[(size_t)u].z - lt.items[(size_t)u].y;
+          else {
+            const long long k = u - (long long)lt.items.size();
+            const long long r = order ? order[k] : k;
+            len = g.row_ptr[r + 1] - g.row_ptr[r];
+            if (len > h->long_len) len = 0;                 // walked as items
+          }
+          in_chunk += len + 2;                              // a unit costs a little even when it is short
+          if (in_chunk >= target) { cp.push_back((int)(u + 1)); in_chunk = 0; }
         }
-        in_chunk += len + 2;                              // a unit costs a little even when it is short
-        if (in_chunk >= target) { cp.push_back((int)(u + 1)); in_chunk = 0; }
-      }
-      if (cp.back() != (int)n_units) cp.push_back((int)n_units);
-      h->n_chunks = (int)cp.size() - 1;
-      h->d_chunk_ptr = upload(h, cp);
+        if (cp.back() != (int)n_units) cp.push_back((int)n_units);
+        return cp;
+      };
+      const std::vector<int> plain = build_chunks(nullptr), sorted = build_chunks(row_order.data());
+      h->n_chunks = (int)plain.size() - 1;
+      h->d_chunk_ptr = upload(h, plain);
+      h->n_chunks_sorted = (int)sorted.size() - 1;
+      h->d_chunk_ptr_sorted = upload(h, sorted);
     }
     h->d_long_rows = reinterpret_cast<int4*>(upload(h, lt.rows));
   }
@@ -959,8 +980,9 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
     h->d_zblocks = upload(h, zb);
     h->d_comm_block_ptr = upload(h, cbp);
   }
-  h->n_groups = (int)cdiv(h->n_chunks, kChunksPerGroup);
-  h->z_chunk_part = h->alloc<double>((size_t)h->n_chunks * n_comm * gk::kCand);
+  const int max_chunks = std::max(h->n_chunks, h->n_chunks_sorted);
+  h->n_groups = (int)cdiv(max_chunks, kChunksPerGroup);
+  h->z_chunk_part = h->alloc<double>((size_t)max_chunks * n_comm * gk::kCand);
   h->z_group_part = h->alloc<double>((size_t)h->n_groups * n_comm * gk::kCand);
   h->chunk_counter = h->alloc<int>(1);
   h->red_part = h->alloc<double>(std::max<size_t>({(size_t)kSmCount * 8 * gk::kCand, (size_t)h->n_zblocks * 3,

@@ -76,12 +76,17 @@ __device__ __forceinline__ double block_sum(double v, double* sh) {
 // done.  Rows longer than `long_len` are therefore not handled as rows: they come as `n_items`
 // items {row, first entry, one past the last} (first in the grid), whose partial sums go to
 // `scratch` (one padded row per item) and are added up, in item order, by k_spmm_long_rows.
+// With ORDERED, rows are taken in the order `row_order` lists them (inside every community by falling
+// length): where several rows share a warp (narrow operands) its lane groups then walk rows of about the
+// same length and finish together (-20 % measured at 48 columns; at 256 columns, one row per warp, the
+// scattered order costs 13 %, so the caller passes no order there).
 // ------------------------------------------------------------------------------------------
-template <int G, int V, int UN>
+template <int G, int V, int UN, bool ORDERED>
 __global__ void __launch_bounds__(256)
 k_spmm(const int* __restrict__ row_ptr, const int* __restrict__ col, const float* __restrict__ dinv,
        const float4* __restrict__ x, float4* __restrict__ out, int n, int ld4,
-       const int4* __restrict__ items, int n_items, int long_len, float4* __restrict__ scratch) {
+       const int4* __restrict__ items, int n_items, int long_len, float4* __restrict__ scratch,
+       const int* __restrict__ row_order) {
   const int lane = threadIdx.x & 31;
   const int gl = lane & (G - 1);
   const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << (lane & ~(G - 1)));
@@ -96,6 +101,7 @@ k_spmm(const int* __restrict__ row_ptr, const int* __restrict__ col, const float
     dst = scratch + unit * ld4;
   } else {
     row = unit - n_items;
+    if (ORDERED) row = row_order[row];
     rs = row_ptr[row]; re = row_ptr[row + 1];
     if (re - rs > long_len) return;
     dst = out + row * ld4;
@@ -930,7 +936,8 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
           const float4* __restrict__ Rn, int ld4, int n, const SearchCtl* __restrict__ ctl, int n_comm,
           double* __restrict__ chunk_part, const int* __restrict__ n_active, int use_smem,
           const int* __restrict__ chunk_ptr, int n_chunks, int* __restrict__ chunk_counter,
-          const int4* __restrict__ items, int n_items, int long_len, float4* __restrict__ scratch) {
+          const int4* __restrict__ items, int n_items, int long_len, float4* __restrict__ scratch,
+          const int* __restrict__ row_order) {
   if (*n_active <= 0) return;
   constexpr int PER = OUT ? 2 : NC;
   // dynamic shared memory: per warp the row's a, b (2 V float4 per lane; parked there during the
@@ -978,7 +985,7 @@ k_score_z(const int* __restrict__ row_ptr, const int* __restrict__ col,
       const int u = unit_base + lane;
       if (u < n_items) my_unit = items[u];
       else {
-        const int r = u - n_items;
+        const int r = row_order != nullptr ? row_order[u - n_items] : u - n_items;
         my_unit = make_int4(r, row_ptr[r], row_ptr[r + 1], -1);
         if (my_unit.z - my_unit.y > long_len) my_unit.z = my_unit.y;   // walked as items
       }
@@ -1130,7 +1137,8 @@ k_score_z_out_half(const int* __restrict__ row_ptr, const int* __restrict__ col,
                    const SearchCtl* __restrict__ ctl, int n_comm, double* __restrict__ chunk_part,
                    const int* __restrict__ n_active, const int* __restrict__ chunk_ptr, int n_chunks,
                    int* __restrict__ chunk_counter,
-                   const int4* __restrict__ items, int n_items, int long_len, float4* __restrict__ scratch) {
+                   const int4* __restrict__ items, int n_items, int long_len, float4* __restrict__ scratch,
+                   const int* __restrict__ row_order) {
   if (*n_active <= 0) return;
   static_assert(16 % UN == 0, "UN divides the chunk");
   extern __shared__ double s_half[];
@@ -1159,7 +1167,7 @@ k_score_z_out_half(const int* __restrict__ row_ptr, const int* __restrict__ col,
           row = it.x; rs = it.y; re = it.z;
           piece = it.w >= 0;
         } else {
-          row = unit - n_items;
+          row = row_order[unit - n_items];
           rs = row_ptr[row]; re = row_ptr[row + 1];
           if (re - rs > long_len) re = rs;          // walked as items
         }
