@@ -73,3 +73,14 @@ def test_many_small_communities_and_isolated_nodes():
 def test_dual_mode_one_and_other_search_parameters():
     pr = tiny_problem(7, n=80, widths=(6, 9, 4), n_comm=3)
     run_pair(pr, dual_mode=1, bt_growth=3.0, bt_shrink=0.3, tau0=0.01, theta0=0.02, fista_iters=7, loss_scale=0.5)
+
+
+def test_first_hidden_layer_wider_than_1024():
+    """Only C_2 .. C_L are limited to 1024 columns (the row width of the theta scoring); C_0 and C_1 may be
+    wider.  A three-layer net with C_1 = 1100 must run and match; C_2 = 1100 must be refused."""
+    run_pair(tiny_problem(8, n=48, widths=(6, 1100, 5, 3), n_comm=3), n_it=3)
+    pr = tiny_problem(8, n=48, widths=(6, 7, 1100, 3), n_comm=3)
+    with pytest.raises(binding.GcnAdmmError) as e:
+        binding.GcnAdmm(pr["n"], pr["row_ptr"], pr["col_idx"], pr["X"].astype(np.float32), pr["y"], pr["mask"],
+                        pr["widths"], pr["n_comm"], pr["community"], [w.astype(np.float32) for w in pr["W"]])
+    assert e.value.code == -4
