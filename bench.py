@@ -394,7 +394,7 @@ def run_ours(args):
                                e2e_L_rho=obj2[0]))
     if world == 1 and not args.no_cpu_baseline:
         full_cfg = inputs.CONFIGS[args.config]
-        if wl.n <= 6000:          # small workloads: the oracle runs the workload itself
+        if wl.n <= 25000:         # small workloads: the oracle runs the workload itself
             _, dt = oracle_rate(args.config, args.scale, 2, 1)
             line["cpu_baseline"] = dict(value=1.0 / dt, unit=UNIT, cores=blas_threads(), kind="oracle",
                                         sample=f"2 oracle iterations (after 1) on the workload itself, {dt:.2f} s each")

@@ -700,7 +700,7 @@ __global__ void k_reduce_chunks(const double* __restrict__ chunk_part, int n_chu
 
 // Decisions of the `count` communities of a hidden layer, one warp each.  k_reduce_chunks left the sweep's
 // sums in block_part[(b*count + i)*per + j], b < n_blocks; they are added in a fixed order (lane-strided
-// over b, then the shuffle tree), followed by the sums of the segments scored in pieces
+// over b, then the shuffle tree), together with the sums of the segments scored in pieces
 // (split_scores, in the order split_order lists those of community i: split_ptr[i] .. split_ptr[i+1]-1).
 // own[i*3 + 2] = <Z_i - f(H_i), G_i>.
 __global__ void k_search_decide_z(SearchCtl* ctl, int count, const double* __restrict__ block_part, int n_blocks,
@@ -720,13 +720,15 @@ __global__ void k_search_decide_z(SearchCtl* ctl, int count, const double* __res
 #pragma unroll
     for (int j = 0; j < kCand; ++j)
       if (j < per) s[j] += block_part[((size_t)b * count + i) * per + j];
+  for (int k = split_ptr[i] + lane; k < split_ptr[i + 1]; k += 32) {
+    const size_t at = (size_t)split_order[k] * per;
+#pragma unroll
+    for (int j = 0; j < kCand; ++j)
+      if (j < per) s[j] += split_scores[at + j];
+  }
 #pragma unroll
   for (int j = 0; j < kCand; ++j) s[j] = warp_sum(s[j]);
   if (lane != 0) return;
-  for (int k = split_ptr[i]; k < split_ptr[i + 1]; ++k)
-#pragma unroll
-    for (int j = 0; j < kCand; ++j)
-      if (j < per) s[j] += split_scores[(size_t)split_order[k] * per + j];
   decide_one(c, s, own[i * 3 + 2], a, n_active, status);
 }
 
