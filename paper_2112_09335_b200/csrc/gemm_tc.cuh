@@ -26,6 +26,7 @@
 // drain finished accumulators (see k_gemm_tc_ws).  Every wait on an mbarrier is bounded; a wait that runs
 // out raises `*error_flag` and the CTA leaves through the normal exit (tensor memory released).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -169,11 +170,20 @@ __global__ void k_split_b(const float* __restrict__ Bk, int ldbk, int N, int K, 
   }
 }
 
-template <int NT, bool IMG>
-__global__ void __launch_bounds__(WsCfg<NT>::kThreads, 1)
+// TMA = true (needs IMG): the A operand is not loaded by the producers at all.  One more warp (its lane 0)
+// fetches each 128 x 32 tile of A with a tensor copy (cp.async.bulk.tensor, 128-byte swizzle: the copy
+// engine writes exactly the K-major layout the MMA descriptors read) straight into the stage's "hi" slot
+// as soon as the stage is free, up to S - 1 chunks ahead.  The tensor core reads a 32-bit operand as TF32
+// by dropping its 13 low mantissa bits, so the raw tile IS the hi operand, hi = x with those bits cleared,
+// and the producers only form lo = x - hi from the tile in shared memory (exact) and store it: no global
+// loads and half the stores, and the A stream no longer passes through L1.  Rows past M and columns
+// past the matrix are filled with zeros by the copy.
+template <int NT, bool IMG, bool TMA = false>
+__global__ void __launch_bounds__(WsCfg<NT>::kThreads + (TMA ? 32 : 0), 1)
 k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk, int ldbk, float* __restrict__ C, int ldc,
              int M, int N, int K, const int* __restrict__ skip, int* __restrict__ error_flag,
-             const uint8_t* __restrict__ b_image) {
+             const uint8_t* __restrict__ b_image, const __grid_constant__ CUtensorMap tmap_a) {
+  static_assert(!TMA || IMG, "the tensor-copy form stages no B tile");
   using Cfg = WsCfg<NT>;
   constexpr int S = Cfg::kStagesWs;
   constexpr int B_PASSES = (NT + 31) / 32;
@@ -183,7 +193,7 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
   if (skip != nullptr && *skip) return;
 
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * S + 4];      // full[S], empty[S], acc_full[2], acc_empty[2]
+  __shared__ __align__(8) uint64_t bars[3 * S + 4];      // full[S], empty[S], acc_full[2], acc_empty[2], raw_full[S]
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -191,9 +201,10 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[S]);
   const uint32_t bar_acc_full = smem_u32(&bars[2 * S]), bar_acc_empty = smem_u32(&bars[2 * S + 2]);
+  const uint32_t bar_raw_full = smem_u32(&bars[2 * S + 4]);
 
   if (tid == 0) {
-    for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 256); mbar_init(bar_empty + 8 * s, 1); }
+    for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 256); mbar_init(bar_empty + 8 * s, 1); mbar_init(bar_raw_full + 8 * s, 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, 32 * Cfg::kEpiWarps); }
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -274,6 +285,27 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
         }
       }
     };
+    if (TMA) {
+      // the raw tile of chunk j lands in the stage's hi slot (see the copy warp below); form lo beside it
+      for (int j = 0; j < total; ++j) {
+        const int stage = j % S;
+        if (!mbar_wait_abortable(bar_raw_full + 8 * stage, (j / S) & 1, abortp)) break;
+        uint8_t* st = smem + (size_t)stage * Cfg::kStage;
+#pragma unroll
+        for (int i = 0; i < A_PASSES; ++i) {
+          const uint32_t off = swz(ld_row + 32 * i, ld_c16);
+          const float4 x = *reinterpret_cast<const float4*>(st + off);
+          float4 l;
+          l.x = x.x - __uint_as_float(__float_as_uint(x.x) & 0xffffe000u);
+          l.y = x.y - __uint_as_float(__float_as_uint(x.y) & 0xffffe000u);
+          l.z = x.z - __uint_as_float(__float_as_uint(x.z) & 0xffffe000u);
+          l.w = x.w - __uint_as_float(__float_as_uint(x.w) & 0xffffe000u);
+          *reinterpret_cast<float4*>(st + kATileBytes + off) = l;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(bar_full + 8 * stage);
+      }
+    } else {
 #pragma unroll
     for (int d = 0; d < DEPTH; ++d) load_chunk(d, ra[d], rb[d]);
     bool stop = false;
@@ -299,6 +331,28 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
         load_chunk(j + DEPTH, ra[d], rb[d]);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         mbar_arrive(bar_full + 8 * stage);
+      }
+    }
+    }
+  } else if (TMA && warp == Cfg::kMmaWarp + 1) {
+    // ---------------- copies (tensor-copy form only): A tile and B image of chunk j as soon as stage j mod S is free ----------------
+    if (lane == 0) {
+      for (int j = 0; j < total; ++j) {
+        const int stage = j % S;
+        if (j >= S && !mbar_wait_abortable(bar_empty + 8 * stage, ((j / S) - 1) & 1, abortp)) break;
+        const int tile = blockIdx.x + (j / kc_count) * gridDim.x, kc = j % kc_count;
+        const uint32_t dst_a = smem_base + (uint32_t)stage * Cfg::kStage;
+        const uint32_t raw_bar = bar_raw_full + 8 * stage;
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(raw_bar), "r"((uint32_t)kATileBytes) : "memory");
+        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                     ::"r"(dst_a), "l"(&tmap_a), "r"(kc * kChunkK), "r"(tile * kBlockM), "r"(raw_bar)
+                     : "memory");
+        const uint32_t bytes = 2u * (uint32_t)Cfg::kBTile;
+        const uint8_t* src = b_image + ((size_t)blockIdx.y * kc_count + (size_t)kc) * bytes;
+        asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar_full + 8 * stage), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(dst_a + 2u * kATileBytes), "l"(src), "r"(bytes), "r"(bar_full + 8 * stage)
+                     : "memory");
       }
     }
   } else if (warp == Cfg::kMmaWarp) {
