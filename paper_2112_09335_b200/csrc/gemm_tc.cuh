@@ -102,6 +102,14 @@ __device__ __forceinline__ uint32_t swz(int r, int c16) { return (uint32_t)r * 1
 // ------------------------------------------------------------------------------------------------
 
 
+// One arrival for the whole warp: an mbarrier arrival is an atomic update of one shared-memory word, and 256
+// of them per K chunk, one after the other, were the floor of about 1,600 clocks per chunk that no change to
+// the staging itself had moved.  Every lane has made its shared-memory stores visible to the async proxy
+// (fence.proxy.async) before the call; __syncwarp orders them before lane 0's releasing arrival.
+__device__ __forceinline__ void mbar_arrive_warp(uint32_t bar) {
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -204,8 +212,8 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
   const uint32_t bar_raw_full = smem_u32(&bars[2 * S + 4]);
 
   if (tid == 0) {
-    for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 256); mbar_init(bar_empty + 8 * s, 1); mbar_init(bar_raw_full + 8 * s, 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, 32 * Cfg::kEpiWarps); }
+    for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 8); mbar_init(bar_empty + 8 * s, 1); mbar_init(bar_raw_full + 8 * s, 1); }   // full: one arrival per producer warp
+    for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, Cfg::kEpiWarps); }
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -289,7 +297,7 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
       // the raw tile of chunk j lands in the stage's hi slot (see the copy warp below); form lo beside it
       for (int j = 0; j < total; ++j) {
         const int stage = j % S;
-        if (!mbar_wait_abortable(bar_raw_full + 8 * stage, (j / S) & 1, abortp)) break;
+        if (!__all_sync(0xffffffffu, mbar_wait_abortable(bar_raw_full + 8 * stage, (j / S) & 1, abortp))) break;   // warp-uniform: the arrival below is per warp
         uint8_t* st = smem + (size_t)stage * Cfg::kStage;
 #pragma unroll
         for (int i = 0; i < A_PASSES; ++i) {
@@ -303,7 +311,7 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
           *reinterpret_cast<float4*>(st + kATileBytes + off) = l;
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(bar_full + 8 * stage);
+        mbar_arrive_warp(bar_full + 8 * stage);
       }
     } else {
 #pragma unroll
@@ -315,7 +323,7 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
         const int j = j0 + d;
         if (j >= total) break;
         const int stage = j % S;
-        if (j >= S && !mbar_wait_abortable(bar_empty + 8 * stage, ((j / S) - 1) & 1, abortp)) { stop = true; break; }
+        if (j >= S && !__all_sync(0xffffffffu, mbar_wait_abortable(bar_empty + 8 * stage, ((j / S) - 1) & 1, abortp))) { stop = true; break; }
         if (IMG && tid == 0) {
           // the stage is free (its MMAs have retired): fetch both B tiles of this chunk with one bulk copy
           // that reports its bytes to the stage's full barrier; this thread's own arrival comes below
@@ -330,7 +338,7 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
         store_chunk(stage, ra[d], rb[d]);
         load_chunk(j + DEPTH, ra[d], rb[d]);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(bar_full + 8 * stage);
+        mbar_arrive_warp(bar_full + 8 * stage);
       }
     }
     }
@@ -393,7 +401,7 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
     uint8_t* tbuf = smem + (size_t)S * Cfg::kStage + (size_t)(warp - 8) * 4096;
     for (int tile_i = 0; tile_i < my_tiles; ++tile_i) {
       const int set = tile_i % SETS;
-      if (!mbar_wait_abortable(bar_acc_full + 8 * set, (tile_i / SETS) & 1, abortp)) break;
+      if (!__all_sync(0xffffffffu, mbar_wait_abortable(bar_acc_full + 8 * set, (tile_i / SETS) & 1, abortp))) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const long long row0 = (long long)(blockIdx.x + tile_i * gridDim.x) * kBlockM + quarter * 32;
 #pragma unroll 1
@@ -427,7 +435,7 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
         __syncwarp();
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      mbar_arrive(bar_acc_empty + 8 * set);
+      mbar_arrive_warp(bar_acc_empty + 8 * set);
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -509,7 +517,7 @@ k_gemm_tn_tc(const float* __restrict__ A, int lda, const float* __restrict__ B, 
   const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[S]), bar_acc = smem_u32(&bars[2 * S]);
 
   if (tid == 0) {
-    for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 256); mbar_init(bar_empty + 8 * s, 1); }
+    for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 8); mbar_init(bar_empty + 8 * s, 1); }   // full: one arrival per producer warp
     mbar_init(bar_acc, 1);
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -606,7 +614,7 @@ k_gemm_tn_tc(const float* __restrict__ A, int lda, const float* __restrict__ B, 
     }
     for (int j = 0; j < total; ++j) {
       const int stage = j % S;
-      if (j >= S && !mbar_wait_abortable(bar_empty + 8 * stage, ((j / S) - 1) & 1, abortp)) break;
+      if (j >= S && !__all_sync(0xffffffffu, mbar_wait_abortable(bar_empty + 8 * stage, ((j / S) - 1) & 1, abortp))) break;
       if (RESID) {
         if (j & 1) { store_chunk(stage, ra[1], rb[0], rb[1]); load_a(j + 2, ra[1]); }
         else       { store_chunk(stage, ra[0], rb[0], rb[1]); load_a(j + 2, ra[0]); }
@@ -617,7 +625,7 @@ k_gemm_tn_tc(const float* __restrict__ A, int lda, const float* __restrict__ B, 
         else       { store_chunk(stage, ra[0], rb[0], nullptr); load_a(j + 2, ra[0]); load_b(j + 2, B, rb[0]); }
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      mbar_arrive(bar_full + 8 * stage);
+      mbar_arrive_warp(bar_full + 8 * stage);
     }
   } else if (lane == 0) {
     // ---------------- MMA issue ----------------
