@@ -84,3 +84,12 @@ def test_first_hidden_layer_wider_than_1024():
         binding.GcnAdmm(pr["n"], pr["row_ptr"], pr["col_idx"], pr["X"].astype(np.float32), pr["y"], pr["mask"],
                         pr["widths"], pr["n_comm"], pr["community"], [w.astype(np.float32) for w in pr["W"]])
     assert e.value.code == -4
+
+
+@pytest.mark.parametrize("n,widths,n_comm", [(2000, (6, 9, 7, 4), 400), (2400, (6, 8, 4), 800)])
+def test_more_communities_than_shared_memory_holds(n, widths, n_comm):
+    """The theta scoring keeps its per-community sums in shared memory while they fit (384 communities with
+    four candidates, 768 with the closed form); beyond that a warp adds into its chunk's slice in global
+    memory.  400 communities put the hidden-layer scoring on that path, 800 the output-layer scoring too."""
+    pr = tiny_problem(9, n=n, widths=widths, n_comm=n_comm, p=4.0 / n)
+    run_pair(pr, n_it=3)
