@@ -5,6 +5,7 @@
 #include <climits>
 #include <cmath>
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <algorithm>
 #include <cstdio>
@@ -22,6 +23,14 @@
 #include "shard_plan.hpp"
 
 using gcn_admm_host::GraphIndex;
+
+namespace {
+// Named range on the profiler timeline (NVTX; a no-op unless a tool is attached) for the life of the object.
+struct Range {
+  explicit Range(const char* name) { nvtxRangePushA(name); }
+  ~Range() { nvtxRangePop(); }
+};
+}  // namespace
 using gk::SearchCtl;
 
 namespace {
@@ -444,6 +453,7 @@ struct gcn_admm {
 
   // ---- W_l block (Section 3.1) --------------------------------------------------------
   void update_W(int l) {
+    Range range("gcn_admm: W block");
     const int Kp = C[l - 1], Cn = C[l], ldc = ld[l];
     const long long n4 = n * ldc / 4;
     SearchCtl* ctl = ctl_w + l;
@@ -505,6 +515,7 @@ struct gcn_admm {
 
   // ---- Z_{l,m}, l < L, every community (Appendix A, Eq. 5/6 and 8-10) ------------------
   void update_Z_hidden(int l) {
+    Range range("gcn_admm: hidden Z blocks");
     const int ldl = ld[l], ldn = ld[l + 1];
     SearchCtl* ctl = ctl_z + (size_t)l * M;
     resid(l + 1, B0);                                                    // R'_{l+1}
@@ -639,6 +650,7 @@ struct gcn_admm {
 
   // ---- Z_L (Eq. 7) and, in the same sweep, the dual as printed in Eq. 3 -----------------
   void update_output(bool dual_now, bool update_z) {
+    Range range("gcn_admm: output layer and dual");
     const int warps = 8;
     Scope sc(this, "output_rows", 1, 4.0 * (double)n * ld[L] * (3 + (update_z ? 1 : 0) + (dual_now ? 1 : 0)), 0.0);
     // rows without a loss term: closed form, plain sweep; training rows: one warp each (FISTA)
@@ -676,6 +688,7 @@ struct gcn_admm {
   int h1_age = 0;
   bool capturing = false;
   void refresh(bool keep_h1 = false) {
+    Range range("gcn_admm: refresh P_l, H_l");
     for (int l = 2; l <= L; ++l) spmm(Z[l - 1], P[l], ld[l - 1]);
     const bool skip_h1 = keep_h1 && !capturing && h1_age + 1 < kH1RefreshEvery;
     h1_age = skip_h1 ? h1_age + 1 : 0;
