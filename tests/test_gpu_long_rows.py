@@ -67,6 +67,8 @@ def test_three_passes_equal_the_uncut_path(case):
 @pytest.mark.parametrize("schedule", [0, 1])
 def test_ten_iterations_with_cut_rows(case, schedule):
     wl, _, limit = case
+    if schedule == 1 and wl.name.startswith("powerlaw-xlarge"):
+        pytest.skip("the serial schedule with cut rows is covered on the other cases (the oracle needs 40 s here)")
     g = handle(wl, long_row=limit, schedule=schedule)
     o = make_oracle(wl)
     try:
