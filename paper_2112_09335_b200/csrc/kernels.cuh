@@ -111,11 +111,28 @@ k_spmm(const int* __restrict__ row_ptr, const int* __restrict__ col, const float
     float4 acc[V];
 #pragma unroll
     for (int v = 0; v < V; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    // Narrow operands (several rows per warp): a chunk of G entries costs three dependent load latencies
+    // (column, weight of that column, operand row) and moves little data, so the columns are fetched two
+    // chunks ahead and their weights one chunk ahead.  (At one row per warp the same prefetch was measured
+    // slower, and this kernel's load order is touchy there: the wide form keeps the plain loop.)
+    constexpr bool kAhead = G < 32;
+    int c_n = 0, c_n2 = 0;
+    float w_n = 0.f;
+    if (kAhead) {
+      if (rs + gl < re) c_n = col[rs + gl];
+      if (rs + G + gl < re) c_n2 = col[rs + G + gl];
+      if (rs + gl < re) w_n = dinv[c_n];
+    }
     for (int base = rs; base < re; base += G) {
       const int idx = base + gl;
       int c = 0;
       float w = 0.f;
-      if (idx < re) { c = col[idx]; w = dinv[c]; }
+      if (kAhead) {
+        c = c_n; w = w_n;
+        c_n = c_n2;
+        c_n2 = (idx + 2 * G < re) ? col[idx + 2 * G] : 0;
+        w_n = (idx + G < re) ? dinv[c_n] : 0.f;
+      } else if (idx < re) { c = col[idx]; w = dinv[c]; }
       const int cnt = min(G, re - base);
       for (int t = 0; t < cnt; t += UN) {
         int cj[UN];
