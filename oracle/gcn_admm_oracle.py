@@ -419,18 +419,18 @@ class OracleADMM:
         fW = (forced or {}).get("W", {})
         fZ = (forced or {}).get("Z", {})
         Wn, taun = list(self.W), list(self.tau)
-        for l in range(1, L + 1):                      # line 3: every W_l from (W^k, Z^k, U^k)
+        for l in range(1, L + 1):                      # every W_l from (W^k, Z^k, U^k)
             Wn[l], taun[l], rec["W"][l] = self.update_W(l, forced=fW.get(l))
         Zn = [z for z in self.Z]
         thetan = [None] + [list(t) for t in self.theta[1:]]
-        for l in range(1, L):                          # line 4: every Z_{l,m} from (W^{k+1}, Z^k, U^k)
+        for l in range(1, L):                          # every Z_{l,m} from (W^{k+1}, Z^k, U^k)
             Zl = self.Z[l].copy()
             for m in range(M):
                 Zlm, thetan[l][m], rec["Z"][(l, m)] = self.update_Z(l, m, Wn, forced=fZ.get((l, m)))
                 Zl[self.V[m]] = Zlm
             Zn[l] = Zl
         Zn[L] = self.update_ZL(Wn)
-        if self.p.dual_mode == 0:                      # line 5, Eq. (3) as printed
+        if self.p.dual_mode == 0:                      # dual update, Eq. (3) as printed
             Un = self.update_U(Wn, self.Z)
         else:
             Un = self.update_U(Wn, Zn)

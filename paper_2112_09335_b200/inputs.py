@@ -83,7 +83,7 @@ CONFIGS = [
          train_p=0.08, widths=[100, 256, 256, 47], n_comm=64, n_iters=20),
     # shaped like the paper's own speed-up experiment (Section 4.1, Table 2): 13,752 nodes, 767 features,
     # 1000 hidden units, 10 classes, 1000 training nodes, 3 communities; the paper gives no edge count, so the
-    # mean degree (30) and the feature density (0.3) are free choices of this build
+    # mean degree (30) and the feature density (0.3) are free choices made here
     dict(name="table2-shaped", n=13752, kind="dcsbm", blocks=10, edges=206280, alpha=1.5,
          draw_factor=1.068, feat="bow", feat_p=0.3, c0=767, classes=10, label="block",
          train=1000, widths=[767, 1000, 10], n_comm=3, n_iters=50),
