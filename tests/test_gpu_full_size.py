@@ -19,9 +19,37 @@ def rows_close(got, want, scale, tol):
     return float(np.max(err / (scale + 1e-30))), tol
 
 
-def test_sampled_rows_at_full_size():
+@pytest.fixture(scope="module")
+def wl_full():
+    return inputs.make_workload(4)
+
+
+def test_two_runs_give_the_same_bits_at_full_size(wl_full):
+    """At this size the chunks of the theta scoring are taken by whichever warp is free, thousands at a time;
+    the sums are kept per chunk and added in chunk order, so two runs must still agree bit for bit."""
+    wl = wl_full
+    L = len(wl.widths) - 1
+    outs = []
+    for _ in range(2):
+        g = binding.GcnAdmm(wl.n, wl.row_ptr, wl.col_idx, wl.X, wl.y, wl.train_mask, wl.widths, wl.n_comm, wl.community,
+                            wl.w_init, nu=wl.nu, rho=wl.rho)
+        try:
+            g.step(6)
+            d = g.decisions()
+            outs.append(dict(trial_w=d["trial_w"], trial_z=d["trial_z"], q_w=d["q_w"], q_z=d["q_z"], obj=g.objective(),
+                             ZL=g.get_state(binding.ST_Z, L), U=g.get_state(binding.ST_U),
+                             **{f"W{l}": g.get_state(binding.ST_W, l) for l in range(1, L + 1)},
+                             **{f"theta{l}": g.get_state(binding.ST_THETA, l) for l in range(1, L)}))
+        finally:
+            g.destroy()
+    assert (outs[0]["trial_z"][3:] >= 0).all()          # the searches were really running
+    for key in outs[0]:
+        assert np.array_equal(outs[0][key], outs[1][key]), key
+
+
+def test_sampled_rows_at_full_size(wl_full):
     import torch
-    wl = inputs.make_workload(4)
+    wl = wl_full
     g = binding.GcnAdmm(wl.n, wl.row_ptr, wl.col_idx, wl.X, wl.y, wl.train_mask, wl.widths, wl.n_comm, wl.community,
                         wl.w_init, nu=wl.nu, rho=wl.rho)
     try:
