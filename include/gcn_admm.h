@@ -110,6 +110,8 @@ void gcn_admm_default_params(gcn_admm_params* p);
  *  row_ptr, col_idx  CSR pattern of the undirected, unweighted adjacency A (host or device):
  *                    row_ptr[n+1] ascending from 0, columns strictly ascending inside a row,
  *                    symmetric.  Diagonal entries are dropped; the identity of A~ is added here.
+ *                    Range and order are checked entry by entry; symmetry by comparing the number
+ *                    and two 64-bit fingerprints of the entries above and below the diagonal.
  *  X                 Z_0, n x C_0 (host or device)
  *  y                 class id per node, 0..C_L-1 (only rows with train_mask != 0 are read as labels)
  *  train_mask        n bytes, non-zero = the node's loss term is part of R

@@ -828,8 +828,8 @@ struct HostView {
   const T& operator[](size_t i) const { return ptr[i]; }
 };
 
-template <typename T>
-T* upload(gcn_admm* h, const std::vector<T>& v) {
+template <typename T, typename A>
+T* upload(gcn_admm* h, const std::vector<T, A>& v) {
   T* d = h->alloc<T>(v.size());
   if (!v.empty()) CU(cudaMemcpy(d, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice));
   return d;
@@ -891,13 +891,8 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
   h->d_row_comm = upload(h, g.row_comm);
   h->d_perm = upload(h, g.perm);
   h->d_dinv = upload(h, g.dinv);
-  {
-    std::vector<unsigned short> cc(g.col.size());
-    const long long n_entries = (long long)cc.size();
-#pragma omp parallel for schedule(static)
-    for (long long e = 0; e < n_entries; ++e) cc[e] = (unsigned short)g.row_comm[g.col[e]];
-    h->d_col_comm = upload(h, cc);
-  }
+  h->d_col_comm = upload(h, g.col_comm);
+  { gcn_admm_host::Table<unsigned short>().swap(h->gi.col_comm); }   // needed on the device only
   h->d_y = upload(h, y_new);
   h->d_train = upload(h, t_new);
   {
@@ -939,6 +934,7 @@ void create_impl(gcn_admm* h, long long n, const long long* row_ptr, const int* 
     }
     std::vector<int> row_order((size_t)n);
     for (long long i = 0; i < n; ++i) row_order[(size_t)i] = (int)i;
+#pragma omp parallel for schedule(dynamic, 1)
     for (int m = 0; m < n_comm; ++m)   // inside a community: longest rows first, ties by row id
       std::stable_sort(row_order.begin() + g.comm_ptr[m], row_order.begin() + g.comm_ptr[m + 1], [&](int a, int b) {
         return g.row_ptr[a + 1] - g.row_ptr[a] > g.row_ptr[b + 1] - g.row_ptr[b];
@@ -1496,27 +1492,25 @@ int gcn_admm_index(gcn_admm* h, int which, int comm, const int** data, long long
   return guarded(h, [&] {
     if (!data || !len || which < 0 || which > GCN_ADMM_IX_SEG_BEGIN) throw Fail{GCN_ADMM_ERR_ARG, "bad selector"};
     const GraphIndex& g = h->gi;
-    const std::vector<int>* v = nullptr;
+    auto give = [&](const auto& v) { *data = v.data(); *len = (long long)v.size(); };
     switch (which) {
-      case GCN_ADMM_IX_PERM: v = &g.perm; break;
-      case GCN_ADMM_IX_INV_PERM: v = &g.inv; break;
-      case GCN_ADMM_IX_COMM_PTR: v = &g.comm_ptr; break;
-      case GCN_ADMM_IX_CSR_ROW_PTR: v = &g.row_ptr; break;
-      case GCN_ADMM_IX_CSR_COL: v = &g.col; break;
-      case GCN_ADMM_IX_SEG_ROW_PTR: v = &g.seg_row_ptr; break;
-      case GCN_ADMM_IX_SEG_COMM: v = &g.seg_comm; break;
-      case GCN_ADMM_IX_SEG_BEGIN: v = &g.seg_begin; break;
+      case GCN_ADMM_IX_PERM: give(g.perm); break;
+      case GCN_ADMM_IX_INV_PERM: give(g.inv); break;
+      case GCN_ADMM_IX_COMM_PTR: give(g.comm_ptr); break;
+      case GCN_ADMM_IX_CSR_ROW_PTR: give(g.row_ptr); break;
+      case GCN_ADMM_IX_CSR_COL: give(g.col); break;
+      case GCN_ADMM_IX_SEG_ROW_PTR: give(g.seg_row_ptr); break;
+      case GCN_ADMM_IX_SEG_COMM: give(g.seg_comm); break;
+      case GCN_ADMM_IX_SEG_BEGIN: give(g.seg_begin); break;
       default: {
         if (comm < 0 || comm >= h->M) throw Fail{GCN_ADMM_ERR_ARG, "community out of range"};
         std::vector<int>& c = h->ix_cache[which];
         if (which == GCN_ADMM_IX_NBR) c = gcn_admm_host::nbr_of(g, comm);
         else if (which == GCN_ADMM_IX_HALO1) c = gcn_admm_host::halo1_of(g, comm);
         else c = gcn_admm_host::halo2_of(g, comm);
-        v = &c;
+        give(c);
       }
     }
-    *data = v->data();
-    *len = (long long)v->size();
   });
 }
 
