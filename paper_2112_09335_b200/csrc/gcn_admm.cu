@@ -309,9 +309,12 @@ struct gcn_admm {
       const long long work = (long long)groups * cdiv(K, gtc::kChunkK) * (NT) * 8;                             \
       gtc::k_split_b<<<(unsigned)std::min<long long>(cdiv(work, 256), 4 * kSmCount), 256, 0, stream>>>(Bk, ldbk, N, K, NT, b_image); \
       ++launches;                                                                                              \
-      if ((NT) <= 128 && make_a_tile_map(A, Mr, lda, &tmap)) {   /* A tiles by tensor copies (measured: -7..-10 % up to 128 columns, +3 % at 256) */ \
-        CU(cudaFuncSetAttribute(gtc::k_gemm_tc_ws<NT, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-        gtc::k_gemm_tc_ws<NT, true, true><<<grid, gtc::WsCfg<NT>::kThreads + 32, smem, stream>>>(A, lda, Bk, ldbk, Cm, ldc, (int)Mr, N, K, skip, tc_error, b_image, tmap); \
+      /* up to 128 columns: A tiles by tensor copies into a ring of their own (at 256 columns shared memory    \
+         leaves no room for it, and the form measured no faster there) */                                      \
+      if ((NT) <= 128 && make_a_tile_map(A, Mr, lda, &tmap)) {                                                 \
+        const size_t smem_ring = gtc::WsCfg<NT>::kSmemRing;                                                    \
+        CU(cudaFuncSetAttribute(gtc::k_gemm_tc_ws<NT, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_ring)); \
+        gtc::k_gemm_tc_ws<NT, true, true><<<grid, gtc::WsCfg<NT>::kThreads + 32, smem_ring, stream>>>(A, lda, Bk, ldbk, Cm, ldc, (int)Mr, N, K, skip, tc_error, b_image, tmap); \
       } else {                                                                                                 \
         CU(cudaFuncSetAttribute(gtc::k_gemm_tc_ws<NT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
         gtc::k_gemm_tc_ws<NT, true><<<grid, gtc::WsCfg<NT>::kThreads, smem, stream>>>(A, lda, Bk, ldbk, Cm, ldc, (int)Mr, N, K, skip, tc_error, b_image, tmap); \

@@ -42,24 +42,28 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-// Shared-memory operand descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t operand_desc(uint32_t smem_addr) {
-  const uint32_t lo = ((smem_addr >> 4) & 0x3fffu) | (1u << 16);          // start address, LBO field = 1
-  const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);             // SBO, version 1, SWIZZLE_128B
-  return ((uint64_t)hi << 32) | lo;
-}
-
 // Instruction descriptor: D fp32, A and B TF32, both K-major, M = 128, N = nt.
 __device__ __forceinline__ uint32_t instr_desc(int nt) {
   return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(nt >> 3) << 17) | ((uint32_t)(kBlockM >> 4) << 24);
 }
 
-__device__ __forceinline__ void mma_tf32(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+// Shared-memory operand descriptor of a K-major tile with the 128-byte swizzle, 8-row groups 1024 bytes
+// apart: the low word holds the start address (in 16-byte units) and the LBO field (= 1), the high word the
+// SBO, the version and the swizzle mode, and is the same for every tile.  The MMA wrapper takes the low
+// words: the one issuing thread of a CTA then spends one addition per operand (its instruction count per
+// chunk is a floor of the whole pipeline: rebuilding 64-bit descriptors and dividing by the chunk count
+// there cost 16 % of the narrow products).
+constexpr uint32_t kOperandDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);   // SBO, version 1, SWIZZLE_128B
+__device__ __forceinline__ uint32_t operand_desc_lo(uint32_t smem_addr) { return ((smem_addr >> 4) & 0x3fffu) | (1u << 16); }
+__device__ __forceinline__ void mma_tf32_lo(uint32_t tmem_d, uint32_t da_lo, uint32_t db_lo, uint32_t idesc, uint32_t accumulate,
+                                            uint32_t desc_hi = kOperandDescHi) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %6};\n\t"
+      "mov.b64 db, {%2, %6};\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
-      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u)
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], da, db, %3, {%5, %5, %5, %5}, p;\n\t}"
+      ::"r"(tmem_d), "r"(da_lo), "r"(db_lo), "r"(idesc), "r"(accumulate), "r"(0u), "r"(desc_hi)
       : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
@@ -116,7 +120,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 // Waits for a phase, giving up when another role has raised the abort flag or after kWaitClocks (a try_wait
 // may itself suspend the thread for a while, so the bound is on elapsed clocks, not on attempts).
 __device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  const long long t0 = clock64();
+  long long t0 = 0;   // read only once the wait has proved long: a wait that succeeds at once costs one try
   for (uint32_t i = 0;; ++i) {
     uint32_t ok;
     asm volatile(
@@ -129,7 +133,8 @@ __device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parit
     if (ok) return true;
     if ((i & 63u) == 63u) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitClocks) break;
+      if (t0 == 0) t0 = clock64();
+      else if (clock64() - t0 > kWaitClocks) break;
     }
   }
   *abort_flag = 1;
@@ -151,6 +156,13 @@ struct WsCfg {
   static constexpr int kAccCols = kSets * 2 * NT;
   static constexpr uint32_t kTmemCols = kAccCols <= 64 ? 64 : kAccCols <= 128 ? 128 : kAccCols <= 256 ? 256 : 512;
   static constexpr size_t kSmem = (size_t)kStagesWs * kStage + kEpiWarps * 4096 + 1024;   // + the epilogue warps' buffers
+  // Tensor-copy form (NT <= 128): a ring of R slots {raw A tile (read in place as the hi operand), B_hi, B_lo},
+  // filled by copies alone and therefore a DRAM latency ahead of the MMAs, and a ring of S A_lo tiles that the
+  // producers fill from the raw tiles; a lo tile is held only from the producers' stores to the end of its MMAs.
+  static constexpr int kRawSlots = NT > 64 ? 3 : 5;
+  static constexpr int kLoStages = 3;
+  static constexpr int kRawSlot = kATileBytes + 2 * kBTile;
+  static constexpr size_t kSmemRing = (size_t)kRawSlots * kRawSlot + (size_t)kLoStages * kATileBytes + kEpiWarps * 4096 + 1024;
 };
 
 // The weight operand split once, in the layout the MMA descriptors read: for column group g and K
@@ -193,7 +205,8 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
              const uint8_t* __restrict__ b_image, const __grid_constant__ CUtensorMap tmap_a) {
   static_assert(!TMA || IMG, "the tensor-copy form stages no B tile");
   using Cfg = WsCfg<NT>;
-  constexpr int S = Cfg::kStagesWs;
+  constexpr int S = TMA ? Cfg::kLoStages : Cfg::kStagesWs;   // stages of the ring the producers fill
+  constexpr int R = TMA ? Cfg::kRawSlots : 1;                // slots of the ring the copies fill (tensor-copy form only)
   constexpr int B_PASSES = (NT + 31) / 32;
   constexpr int A_PASSES = kBlockM / 32;
   constexpr int SETS = Cfg::kSets;
@@ -201,7 +214,7 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
   if (skip != nullptr && *skip) return;
 
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[3 * S + 4];      // full[S], empty[S], acc_full[2], acc_empty[2], raw_full[S]
+  __shared__ __align__(8) uint64_t bars[2 * S + 4 + 2 * R];      // full[S], empty[S], acc_full[2], acc_empty[2], raw_full[R], raw_empty[R]
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -209,10 +222,16 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[S]);
   const uint32_t bar_acc_full = smem_u32(&bars[2 * S]), bar_acc_empty = smem_u32(&bars[2 * S + 2]);
-  const uint32_t bar_raw_full = smem_u32(&bars[2 * S + 4]);
+  const uint32_t bar_raw_full = smem_u32(&bars[2 * S + 4]), bar_raw_empty = smem_u32(&bars[2 * S + 4 + R]);
+  // shared-memory map of the tensor-copy form: R slots of {raw A, B_hi, B_lo}, then S tiles of A_lo
+  constexpr uint32_t kRawSlot = (uint32_t)Cfg::kRawSlot;
+  constexpr uint32_t kLoBase = (uint32_t)R * kRawSlot;
+  constexpr uint32_t kStageBytes = TMA ? (uint32_t)kATileBytes : (uint32_t)Cfg::kStage;
+  constexpr uint32_t kRingBytes = TMA ? kLoBase + (uint32_t)S * kStageBytes : (uint32_t)S * kStageBytes;
 
   if (tid == 0) {
-    for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 8); mbar_init(bar_empty + 8 * s, 1); mbar_init(bar_raw_full + 8 * s, 1); }   // full: one arrival per producer warp
+    for (int s = 0; s < S; ++s) { mbar_init(bar_full + 8 * s, 8); mbar_init(bar_empty + 8 * s, 1); }   // full: one arrival per producer warp
+    for (int r = 0; r < R; ++r) { mbar_init(bar_raw_full + 8 * r, 1); mbar_init(bar_raw_empty + 8 * r, 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, Cfg::kEpiWarps); }
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -241,11 +260,15 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
     const int ld_c16 = tid & 7, ld_row = tid >> 3;
     constexpr int DEPTH = IMG ? 4 : (NT > 128 ? 1 : 2);   // chunks a thread holds in registers ahead of the one it stores
     float4 ra[DEPTH][A_PASSES], rb[DEPTH][IMG ? 1 : B_PASSES];
-    auto load_chunk = [&](int j, float4* pa, float4* pb) {
-      if (j >= total) return;
-      const int tile = blockIdx.x + (j / kc_count) * gridDim.x, kc = j % kc_count;
-      const int k0 = kc * kChunkK + ld_c16 * 4;
-      const long long row0 = (long long)tile * kBlockM;
+    // chunks are loaded strictly in order, so tile and K chunk of the next load are counters (no division per chunk)
+    int ld_j = 0, ld_kc = 0, st_kc = 0;
+    long long ld_row0 = (long long)blockIdx.x * kBlockM;
+    auto load_chunk = [&](float4* pa, float4* pb) {
+      if (ld_j >= total) return;
+      const int k0 = ld_kc * kChunkK + ld_c16 * 4;
+      const long long row0 = ld_row0;
+      ++ld_j;
+      if (++ld_kc == kc_count) { ld_kc = 0; ld_row0 += (long long)gridDim.x * kBlockM; }
 #pragma unroll
       for (int i = 0; i < A_PASSES; ++i) {
         const long long r = row0 + ld_row + 32 * i;
@@ -294,28 +317,33 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
       }
     };
     if (TMA) {
-      // the raw tile of chunk j lands in the stage's hi slot (see the copy warp below); form lo beside it
+      // chunk j: raw tile and weight tiles in slot j mod R (see the copy warp below), lo in stage j mod S
+      int stage = 0, slot = 0;
+      uint32_t empty_parity = 1, raw_parity = 0;   // a fresh barrier passes a wait on parity 1
       for (int j = 0; j < total; ++j) {
-        const int stage = j % S;
-        if (!__all_sync(0xffffffffu, mbar_wait_abortable(bar_raw_full + 8 * stage, (j / S) & 1, abortp))) break;   // warp-uniform: the arrival below is per warp
-        uint8_t* st = smem + (size_t)stage * Cfg::kStage;
+        if (!__all_sync(0xffffffffu, mbar_wait_abortable(bar_empty + 8 * stage, empty_parity, abortp))) break;   // warp-uniform: the arrival below is per warp
+        if (!__all_sync(0xffffffffu, mbar_wait_abortable(bar_raw_full + 8 * slot, raw_parity, abortp))) break;
+        const uint8_t* raw = smem + (size_t)slot * kRawSlot;
+        uint8_t* st = smem + kLoBase + (size_t)stage * kStageBytes;
 #pragma unroll
         for (int i = 0; i < A_PASSES; ++i) {
           const uint32_t off = swz(ld_row + 32 * i, ld_c16);
-          const float4 x = *reinterpret_cast<const float4*>(st + off);
+          const float4 x = *reinterpret_cast<const float4*>(raw + off);
           float4 l;
           l.x = x.x - __uint_as_float(__float_as_uint(x.x) & 0xffffe000u);
           l.y = x.y - __uint_as_float(__float_as_uint(x.y) & 0xffffe000u);
           l.z = x.z - __uint_as_float(__float_as_uint(x.z) & 0xffffe000u);
           l.w = x.w - __uint_as_float(__float_as_uint(x.w) & 0xffffe000u);
-          *reinterpret_cast<float4*>(st + kATileBytes + off) = l;
+          *reinterpret_cast<float4*>(st + off) = l;
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         mbar_arrive_warp(bar_full + 8 * stage);
+        if (++stage == S) { stage = 0; empty_parity ^= 1u; }
+        if (++slot == R) { slot = 0; raw_parity ^= 1u; }
       }
     } else {
 #pragma unroll
-    for (int d = 0; d < DEPTH; ++d) load_chunk(d, ra[d], rb[d]);
+    for (int d = 0; d < DEPTH; ++d) load_chunk(ra[d], rb[d]);
     bool stop = false;
     for (int j0 = 0; j0 < total && !stop; j0 += DEPTH) {
 #pragma unroll
@@ -328,63 +356,89 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
           // the stage is free (its MMAs have retired): fetch both B tiles of this chunk with one bulk copy
           // that reports its bytes to the stage's full barrier; this thread's own arrival comes below
           const uint32_t bytes = 2u * (uint32_t)Cfg::kBTile;
-          const uint8_t* src = b_image + ((size_t)blockIdx.y * kc_count + (size_t)(j % kc_count)) * bytes;
+          const uint8_t* src = b_image + ((size_t)blockIdx.y * kc_count + (size_t)st_kc) * bytes;
           const uint32_t dst = smem_base + (uint32_t)stage * Cfg::kStage + 2u * kATileBytes;
           asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar_full + 8 * stage), "r"(bytes) : "memory");
           asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar_full + 8 * stage)
                        : "memory");
         }
+        if (++st_kc == kc_count) st_kc = 0;
         store_chunk(stage, ra[d], rb[d]);
-        load_chunk(j + DEPTH, ra[d], rb[d]);
+        load_chunk(ra[d], rb[d]);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         mbar_arrive_warp(bar_full + 8 * stage);
       }
     }
     }
   } else if (TMA && warp == Cfg::kMmaWarp + 1) {
-    // ---------------- copies (tensor-copy form only): A tile and B image of chunk j as soon as stage j mod S is free ----------------
+    // ---------------- copies (tensor-copy form only): A tile and weight tiles of chunk j as soon as slot j mod R is free ----------------
     if (lane == 0) {
+      const uint32_t b_bytes = 2u * (uint32_t)Cfg::kBTile;
+      const uint8_t* const b_src = b_image + (size_t)blockIdx.y * kc_count * b_bytes;
+      int kc = 0, tile = blockIdx.x, slot = 0;
+      uint32_t empty_parity = 1;   // a fresh barrier passes a wait on parity 1
       for (int j = 0; j < total; ++j) {
-        const int stage = j % S;
-        if (j >= S && !mbar_wait_abortable(bar_empty + 8 * stage, ((j / S) - 1) & 1, abortp)) break;
-        const int tile = blockIdx.x + (j / kc_count) * gridDim.x, kc = j % kc_count;
-        const uint32_t dst_a = smem_base + (uint32_t)stage * Cfg::kStage;
-        const uint32_t raw_bar = bar_raw_full + 8 * stage;
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(raw_bar), "r"((uint32_t)kATileBytes) : "memory");
+        if (!mbar_wait_abortable(bar_raw_empty + 8 * slot, empty_parity, abortp)) break;
+        const uint32_t dst_a = smem_base + (uint32_t)slot * kRawSlot;
+        const uint32_t raw_bar = bar_raw_full + 8 * slot;
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(raw_bar), "r"((uint32_t)kATileBytes + b_bytes) : "memory");
         asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                      ::"r"(dst_a), "l"(&tmap_a), "r"(kc * kChunkK), "r"(tile * kBlockM), "r"(raw_bar)
                      : "memory");
-        const uint32_t bytes = 2u * (uint32_t)Cfg::kBTile;
-        const uint8_t* src = b_image + ((size_t)blockIdx.y * kc_count + (size_t)kc) * bytes;
-        asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar_full + 8 * stage), "r"(bytes) : "memory");
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     ::"r"(dst_a + 2u * kATileBytes), "l"(src), "r"(bytes), "r"(bar_full + 8 * stage)
+                     ::"r"(dst_a + (uint32_t)kATileBytes), "l"(b_src + (size_t)kc * b_bytes), "r"(b_bytes), "r"(raw_bar)
                      : "memory");
+        if (++kc == kc_count) { kc = 0; tile += gridDim.x; }
+        if (++slot == R) { slot = 0; empty_parity ^= 1u; }
       }
     }
   } else if (warp == Cfg::kMmaWarp) {
     // ---------------- MMA issue ----------------
+    // One thread issues everything, so its instruction count per chunk is a floor of the whole pipeline
+    // (no division by kc_count, no 64-bit descriptor arithmetic: counters that wrap, one addition per operand).
     if (lane == 0) {
-      const uint32_t idesc = instr_desc(NT);
+      const uint32_t idesc = instr_desc(NT), idesc2 = instr_desc(NT <= 128 ? 2 * NT : NT);
+      int stage = 0, kc = 0, tile_i = 0, slot = 0;
+      uint32_t full_parity = 0;
       for (int j = 0; j < total; ++j) {
-        const int stage = j % S, kc = j % kc_count, tile_i = j / kc_count, set = tile_i % SETS;
+        const int set = SETS == 1 ? 0 : (tile_i & 1);
         if (kc == 0 && tile_i >= SETS && !mbar_wait_abortable(bar_acc_empty + 8 * set, ((tile_i / SETS) - 1) & 1, abortp)) break;
-        if (!mbar_wait_abortable(bar_full + 8 * stage, (j / S) & 1, abortp)) break;
+        if (!mbar_wait_abortable(bar_full + 8 * stage, full_parity, abortp)) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t a_hi = smem_base + stage * Cfg::kStage, a_lo = a_hi + kATileBytes;
-        const uint32_t b_hi = a_hi + 2 * kATileBytes, b_lo = b_hi + Cfg::kBTile;
+        // shared memory ends below 2^18, so additions to a descriptor's low word never carry out of the address field
+        const uint32_t a_hi = operand_desc_lo(TMA ? smem_base + slot * kRawSlot : smem_base + stage * kStageBytes);
+        const uint32_t a_lo = TMA ? operand_desc_lo(smem_base + kLoBase + stage * kStageBytes) : a_hi + (kATileBytes >> 4);
+        const uint32_t b_hi = TMA ? a_hi + (kATileBytes >> 4) : a_hi + (2 * kATileBytes >> 4), b_lo = b_hi + (Cfg::kBTile >> 4);
         const uint32_t acc = tmem_base + (uint32_t)(set * 2 * NT);
 #pragma unroll
         for (int ks = 0; ks < kChunkK / 8; ++ks) {
-          const uint32_t o = ks * 32;
-          const uint32_t first = (kc > 0 || ks > 0) ? 1u : 0u;
-          mma_tf32(acc + NT, operand_desc(a_lo + o), operand_desc(b_hi + o), idesc, first);   // corrections
-          mma_tf32(acc + NT, operand_desc(a_hi + o), operand_desc(b_lo + o), idesc, 1u);
-          mma_tf32(acc, operand_desc(a_hi + o), operand_desc(b_hi + o), idesc, first);        // main product
+          const uint32_t o = ks * 2;   // 32 bytes per K step, in 16-byte units
+          const uint32_t first = (ks > 0) ? 1u : (kc > 0 ? 1u : 0u);
+          if constexpr (NT <= 128) {
+            // B_lo follows B_hi in shared memory in the same 8-row groups, so the two are one operand of 2 NT
+            // rows: A_hi [B_hi; B_lo] fills the main accumulator (columns 0 .. NT-1) and starts the correction
+            // (columns NT .. 2 NT - 1) in one MMA; A_lo B_hi is added to the correction.  Two MMAs per K step
+            // instead of three: narrow MMAs have a floor on their duration, and each one costs the issuing thread.
+            mma_tf32_lo(acc, a_hi + o, b_hi + o, idesc2, first);
+            mma_tf32_lo(acc + NT, a_lo + o, b_hi + o, idesc, 1u);
+          } else {
+            mma_tf32_lo(acc + NT, a_lo + o, b_hi + o, idesc, first);   // corrections
+            mma_tf32_lo(acc + NT, a_hi + o, b_lo + o, idesc, 1u);
+            mma_tf32_lo(acc, a_hi + o, b_hi + o, idesc, first);        // main product
+          }
         }
         mma_commit(bar_empty + 8 * stage);
-        if (kc + 1 == kc_count) mma_commit(bar_acc_full + 8 * set);
+        if (TMA) {
+          mma_commit(bar_raw_empty + 8 * slot);
+          if (++slot == R) slot = 0;
+        }
+        if (++kc == kc_count) {
+          mma_commit(bar_acc_full + 8 * set);
+          kc = 0;
+          ++tile_i;
+        }
+        if (++stage == S) { stage = 0; full_parity ^= 1u; }
       }
     }
   } else {
@@ -398,7 +452,7 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
     constexpr int SLOTS = CW / 4;                      // float4 per row and step
     constexpr int ROWS_PER_STORE = 32 / SLOTS;
     const int turn = (warp - 8) >> 2;                  // which of the quarter's two warps this is
-    uint8_t* tbuf = smem + (size_t)S * Cfg::kStage + (size_t)(warp - 8) * 4096;
+    uint8_t* tbuf = smem + kRingBytes + (size_t)(warp - 8) * 4096;
     for (int tile_i = 0; tile_i < my_tiles; ++tile_i) {
       const int set = tile_i % SETS;
       if (!__all_sync(0xffffffffu, mbar_wait_abortable(bar_acc_full + 8 * set, (tile_i / SETS) & 1, abortp))) break;
@@ -465,11 +519,9 @@ k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk,
 constexpr int kTnThreads = 9 * 32;
 constexpr int kTnRows = 32;                       // rows (reduction steps) per chunk
 
-__device__ __forceinline__ uint64_t operand_desc_mn(uint32_t smem_addr) {
-  const uint32_t lo = ((smem_addr >> 4) & 0x3fffu) | ((4096u >> 4) << 16);   // start address, LBO = 4096
-  const uint32_t hi = (512u >> 4) | (1u << 14) | (1u << 29);                 // SBO = 512, version 1, 128B swizzle / 32B base
-  return ((uint64_t)hi << 32) | lo;
-}
+// MN-major tile: LBO = 4096, SBO = 512, version 1, 128-byte swizzle with 32-byte base (low / high word as above)
+constexpr uint32_t kOperandDescMnHi = (512u >> 4) | (1u << 14) | (1u << 29);
+__device__ __forceinline__ uint32_t operand_desc_mn_lo(uint32_t smem_addr) { return ((smem_addr >> 4) & 0x3fffu) | ((4096u >> 4) << 16); }
 __device__ __forceinline__ uint32_t instr_desc_mn(int nt) {
   return (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(nt >> 3) << 17) |
          ((uint32_t)(kBlockM >> 4) << 24);
@@ -629,23 +681,26 @@ k_gemm_tn_tc(const float* __restrict__ A, int lda, const float* __restrict__ B, 
     }
   } else if (lane == 0) {
     // ---------------- MMA issue ----------------
+    // one issuing thread: counters that wrap and one addition per operand descriptor (see k_gemm_tc_ws)
     const uint32_t idesc = instr_desc_mn(NT);
+    int stage = 0;
+    uint32_t full_parity = 0;
     for (int j = 0; j < total; ++j) {
-      const int stage = j % S;
-      if (!mbar_wait_abortable(bar_full + 8 * stage, (j / S) & 1, abortp)) break;
+      if (!mbar_wait_abortable(bar_full + 8 * stage, full_parity, abortp)) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t a_hi = smem_base + stage * Cfg::kStage, a_lo = a_hi + Cfg::kATile;
-      const uint32_t b_hi = a_hi + 2 * Cfg::kATile, b_lo = b_hi + Cfg::kBTile;
+      const uint32_t a_hi = operand_desc_mn_lo(smem_base + stage * Cfg::kStage), a_lo = a_hi + (Cfg::kATile >> 4);
+      const uint32_t b_hi = a_hi + (2 * Cfg::kATile >> 4), b_lo = b_hi + (Cfg::kBTile >> 4);
 #pragma unroll
       for (int ks = 0; ks < kTnRows / 8; ++ks) {
-        const uint32_t o = ks * 1024;              // the next group of 8 rows
-        const uint32_t first = (j > 0 || ks > 0) ? 1u : 0u;
-        mma_tf32(tmem_base + NT, operand_desc_mn(a_lo + o), operand_desc_mn(b_hi + o), idesc, first);   // corrections
-        mma_tf32(tmem_base + NT, operand_desc_mn(a_hi + o), operand_desc_mn(b_lo + o), idesc, 1u);
-        mma_tf32(tmem_base, operand_desc_mn(a_hi + o), operand_desc_mn(b_hi + o), idesc, first);        // main product
+        const uint32_t o = ks * (1024 >> 4);       // the next group of 8 rows, in 16-byte units
+        const uint32_t first = (ks > 0) ? 1u : (j > 0 ? 1u : 0u);
+        mma_tf32_lo(tmem_base + NT, a_lo + o, b_hi + o, idesc, first, kOperandDescMnHi);   // corrections
+        mma_tf32_lo(tmem_base + NT, a_hi + o, b_lo + o, idesc, 1u, kOperandDescMnHi);
+        mma_tf32_lo(tmem_base, a_hi + o, b_hi + o, idesc, first, kOperandDescMnHi);        // main product
       }
       mma_commit(bar_empty + 8 * stage);
       if (j + 1 == total) mma_commit(bar_acc);
+      if (++stage == S) { stage = 0; full_parity ^= 1u; }
     }
   }
   __syncwarp();
