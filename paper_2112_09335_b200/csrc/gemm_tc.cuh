@@ -21,8 +21,9 @@
 // One CTA owns 128 rows of A and all N <= 256 columns; the accumulators (128 lanes x 2 NT columns of
 // fp32) live in tensor memory.  K is walked in chunks of 32 floats = one 128-byte swizzle row.
 // Producer warps stage each chunk (128-bit loads from global memory, split into hi/lo, stores into shared
-// memory in the canonical K-major 128-byte-swizzled operand layout); one thread issues the twelve MMAs
-// (3 products x 4 steps of K = 8) and commits them to the mbarrier that frees the stage; epilogue warps
+// memory in the canonical K-major 128-byte-swizzled operand layout); one thread issues the MMAs
+// (4 steps of K = 8, three products each; up to 128 columns two of the three share one MMA, see the
+// issuing loop) and commits them to the mbarrier that frees the stage; epilogue warps
 // drain finished accumulators (see k_gemm_tc_ws).  Every wait on an mbarrier is bounded; a wait that runs
 // out raises `*error_flag` and the CTA leaves through the normal exit (tensor memory released).
 #pragma once
@@ -97,7 +98,7 @@ __device__ __forceinline__ uint32_t swz(int r, int c16) { return (uint32_t)r * 1
 //               tensor memory -> registers -> C, arrive on acc_empty[set]  (warp w reads lanes
 //               32 (w mod 4) .. +31; with eight warps the two of a quarter take the column steps in turn)
 //   next warp   MMA: waits full[stage] (and, at the first chunk of a tile, acc_empty[set]), issues
-//               the twelve MMAs, commits to empty[stage] and, at the last chunk, to acc_full[set]
+//               the chunk's MMAs, commits to empty[stage] and, at the last chunk, to acc_full[set]
 // Up to 128 output columns, two accumulator sets (main + correction each) alternate between consecutive
 // tiles (4 NT <= 512 columns of tensor memory); from 129 to 256 columns there is room for one set, and
 // the MMAs of the next tile wait for the epilogue of the current one while the producers keep staging.
@@ -192,12 +193,14 @@ __global__ void k_split_b(const float* __restrict__ Bk, int ldbk, int N, int K, 
 
 // TMA = true (needs IMG): the A operand is not loaded by the producers at all.  One more warp (its lane 0)
 // fetches each 128 x 32 tile of A with a tensor copy (cp.async.bulk.tensor, 128-byte swizzle: the copy
-// engine writes exactly the K-major layout the MMA descriptors read) straight into the stage's "hi" slot
-// as soon as the stage is free, up to S - 1 chunks ahead.  The tensor core reads a 32-bit operand as TF32
-// by dropping its 13 low mantissa bits, so the raw tile IS the hi operand, hi = x with those bits cleared,
-// and the producers only form lo = x - hi from the tile in shared memory (exact) and store it: no global
-// loads and half the stores, and the A stream no longer passes through L1.  Rows past M and columns
-// past the matrix are filled with zeros by the copy.
+// engine writes exactly the K-major layout the MMA descriptors read) and the chunk's two weight tiles with
+// a bulk copy into slot j mod R of a ring that only copies fill, up to R chunks ahead of the MMAs.  The
+// tensor core reads a 32-bit operand as TF32 by dropping its 13 low mantissa bits, so the raw tile IS the
+// hi operand, hi = x with those bits cleared, and the producers only form lo = x - hi from the tile in
+// shared memory (exact) and store it into stage j mod S of a second ring: no global loads and half the
+// stores, and the A stream no longer passes through L1.  A slot is freed by the commit of its chunk's
+// MMAs (raw_empty), a lo stage likewise (empty).  Rows past M and columns past the matrix are filled with
+// zeros by the copy.
 template <int NT, bool IMG, bool TMA = false>
 __global__ void __launch_bounds__(WsCfg<NT>::kThreads + (TMA ? 32 : 0), 1)
 k_gemm_tc_ws(const float* __restrict__ A, int lda, const float* __restrict__ Bk, int ldbk, float* __restrict__ C, int ldc,
