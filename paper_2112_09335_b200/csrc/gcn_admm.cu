@@ -329,6 +329,11 @@ struct gcn_admm {
       else if (N <= 48) TC_WS(48)
       else if (N <= 64) TC_WS(64)
       else if (N <= 128) TC_WS(128)
+      // 129..256 columns with a short reduction (K <= 128: a tile has at most four chunks of MMAs, so the epilogue
+      // that the single accumulator set of the 256-column form leaves uncovered dominates): two groups of 128 columns
+      // in the tensor-copy form instead, whose two accumulator sets put the epilogue under the next tile's MMAs
+      // (measured on 1.2 M rows: 0.372 -> 0.326 ms at K = 47, 0.560 -> 0.463 at 100, 0.518 -> 0.456 at 128; no gain at 256)
+      else if (K <= 128 && lda >= gtc::kChunkK && Mr >= kImageMinRows) TC_WS(128)
       else TC_WS(256)
 #undef TC_WS
       CU(cudaGetLastError());
