@@ -8,7 +8,8 @@ from paper_2112_09335_b200 import binding, inputs
 pytestmark = pytest.mark.gpu
 
 SHAPES = [(1000, 16, 128), (5000, 256, 256), (4097, 256, 100), (3000, 47, 256), (2049, 16, 1433), (700, 5, 37),
-          (130, 256, 8), (40000, 128, 500), (33000, 256, 256), (20001, 47, 256), (16384, 256, 100), (777, 3, 128), (12345, 40, 256), (9000, 1000, 767), (6000, 10, 1000), (3000, 300, 64)]    # (m, n, k)
+          (130, 256, 8), (40000, 128, 500), (33000, 256, 256), (20001, 47, 256), (16384, 256, 100), (777, 3, 128), (12345, 40, 256), (9000, 1000, 767), (6000, 10, 1000), (3000, 300, 64),
+          (17001, 200, 47), (16500, 130, 128), (16390, 129, 33)]    # (m, n, k); the last three: two groups of 128 columns, the second one ragged
 
 
 @pytest.fixture(scope="module")
