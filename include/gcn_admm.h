@@ -232,6 +232,20 @@ enum { GCN_ADMM_SHARD_RANGES = 0, GCN_ADMM_SHARD_FIRST_ORDER = 1, GCN_ADMM_SHARD
 int gcn_admm_shard_plan(gcn_admm* h, int n_ranks, int which, int receiver, int sender, const int** data,
                         long long* len);
 
+/* The propagation A~ x (Problem 1; Section 2: every agent forms the rows of its own communities from its rows
+ * and its neighbours' first-order rows) carried out the way the n_ranks ranks of that plan would, one rank
+ * after the other on this handle's one device: for each rank, the rows it owns and, behind them, copies of
+ * the first-order rows of every sender are gathered into a local matrix (on several devices that second
+ * part is what the receives from the rows' owners fill), the rank's rows of A + I are renumbered to
+ * positions in that local matrix, and the propagation kernel runs on those local tables alone and writes
+ * the rank's rows of the result.  Entry order inside a row is kept, so a row is summed in the same order
+ * as by gcn_admm_propagate (rows longer than `long_row` excepted: there the unsharded call adds partial
+ * sums of pieces).  x, out: n x width, original node order, both host or both device; staged_rows (may be
+ * NULL) receives the number of copied first-order rows summed over the ranks.  Allocates per rank and
+ * synchronises; a check of the plan on the device, not a fast path.  No collective is issued. */
+int gcn_admm_propagate_sharded(gcn_admm* h, int n_ranks, const float* x, int width, float* out,
+                               long long* staged_rows);
+
 /* ---- state access (checkpointing and single-block tests) -------------------------------------
  * Host buffers, dense row-major, original node order.
  *  GCN_ADMM_ST_W      layer 1..L   float  C_{l-1} x C_l

@@ -19,7 +19,7 @@ EXPORTS = [
     "gcn_admm_predict", "gcn_admm_destroy", "gcn_admm_last_error", "gcn_admm_propagate", "gcn_admm_index",
     "gcn_admm_get_state", "gcn_admm_set_state", "gcn_admm_step_block", "gcn_admm_decisions",
     "gcn_admm_launches", "gcn_admm_profile", "gcn_admm_profile_read", "gcn_admm_propagate_static", "gcn_admm_dense_product", "gcn_admm_dense_product_tn",
-    "gcn_admm_shard_plan",
+    "gcn_admm_shard_plan", "gcn_admm_propagate_sharded",
 ]
 
 IX = dict(perm=0, inv_perm=1, comm_ptr=2, nbr=3, halo1=4, halo2=5, csr_row_ptr=6, csr_col=7,
@@ -67,6 +67,7 @@ def load():
     lib.gcn_admm_last_error.restype = C.c_char_p
     lib.gcn_admm_propagate.argtypes = [vp, vp, i32, vp]
     lib.gcn_admm_propagate_static.argtypes = [vp, vp, i32, vp]
+    lib.gcn_admm_propagate_sharded.argtypes = [vp, i32, vp, i32, vp, C.POINTER(i64)]
     lib.gcn_admm_dense_product.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32]
     lib.gcn_admm_dense_product_tn.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32]
     lib.gcn_admm_index.argtypes = [vp, i32, i32, C.POINTER(C.POINTER(i32)), C.POINTER(i64)]
@@ -215,6 +216,16 @@ class GcnAdmm:
         if length.value == 0:
             return np.zeros(0, dtype=np.int32)
         return np.ctypeslib.as_array(data, shape=(length.value,)).copy()
+
+    def propagate_sharded(self, n_ranks, x):
+        """A~ x formed rank by rank from each rank's own rows and copies of its first-order rows (numpy in,
+        numpy out); also returns the number of first-order rows copied, summed over the ranks."""
+        x = np.ascontiguousarray(x, dtype=np.float32)
+        res = np.empty_like(x)
+        staged = C.c_longlong()
+        self._check(self._lib.gcn_admm_propagate_sharded(self._h, int(n_ranks), _ptr(x), x.shape[1], _ptr(res),
+                                                         C.byref(staged)))
+        return res, staged.value
 
     def _state_shape(self, which, layer):
         if which in (ST_W, ST_Z) and not 1 <= layer <= self.L:

@@ -249,24 +249,36 @@ struct gcn_admm {
 
   // ---- launches -----------------------------------------------------------------------
   void spmm(const float* x, float* out, int ldx) {
-    const int ld4 = ldx / 4;
-    const float4* x4 = reinterpret_cast<const float4*>(x);
-    float4* o4 = reinterpret_cast<float4*>(out);
-    const int nn = (int)n;
     char name[48];
     std::snprintf(name, sizeof name, "spmm@%d", ldx);
     Scope sc(this, name, 1, 4.0 * gi.nnz + 8.0 * n + 8.0 * (double)n * ldx, 2.0 * (double)gi.nnz * ldx);
-    // 64-thread blocks: rows differ widely in length, small blocks keep the SMs evenly loaded.
     // Long rows go as items unless the operand is wider than the item buffer was sized for (a
     // caller's matrix wider than every layer): then they are walked whole, slower but the same sums.
     const bool cut = n_items > 0 && (size_t)n_items * ldx <= item_sums_elems;
-    const int items_used = cut ? n_items : 0;
+    spmm_launch(d_row_ptr, d_col, d_dinv, d_row_order, (int)n, d_items, cut ? n_items : 0, cut ? long_len : INT_MAX, x, out, ldx);
+    if (cut) {
+      gk::k_spmm_long_rows<<<(unsigned)n_long, 64, 0, stream>>>(d_long_rows, reinterpret_cast<const float4*>(item_sums),
+                                                                reinterpret_cast<float4*>(out), ldx / 4);
+      CU(cudaGetLastError());
+      ++launches;   // booked with the propagation it completes
+    }
+  }
+
+  // The propagation kernel on a graph given by its tables (the handle's own, or a rank's local part of it):
+  // rows 0 .. nn-1 of out = A~ x, columns of `cl` index rows of x.  `order` lists the rows by falling length
+  // (used by the forms that put several rows in a warp).
+  void spmm_launch(const int* rp, const int* cl, const float* dv, const int* order, int nn, const int4* its, int items_used,
+                   int long_eff, const float* x, float* out, int ldx) {
+    const int ld4 = ldx / 4;
+    const float4* x4 = reinterpret_cast<const float4*>(x);
+    float4* o4 = reinterpret_cast<float4*>(out);
+    // 64-thread blocks: rows differ widely in length, small blocks keep the SMs evenly loaded.
 #define SPMM_CASE(G, V, UN)                                                                    \
   {                                                                                            \
-    const long long threads = (n + items_used) * (G);                                          \
+    const long long threads = ((long long)nn + items_used) * (G);                              \
     /* several rows per warp (G < 32): rows of equal length side by side */                     \
-    gk::k_spmm<G, V, UN, ((G) < 32)><<<(unsigned)cdiv(threads, 64), 64, 0, stream>>>(d_row_ptr, d_col, d_dinv, x4, o4, nn, ld4, \
-        d_items, items_used, cut ? long_len : INT_MAX, reinterpret_cast<float4*>(item_sums), d_row_order); \
+    gk::k_spmm<G, V, UN, ((G) < 32)><<<(unsigned)cdiv(threads, 64), 64, 0, stream>>>(rp, cl, dv, x4, o4, nn, ld4, \
+        its, items_used, long_eff, reinterpret_cast<float4*>(item_sums), order);               \
   }
     if (ld4 <= 1) SPMM_CASE(1, 1, 4)
     else if (ld4 <= 2) SPMM_CASE(2, 1, 4)
@@ -277,11 +289,6 @@ struct gcn_admm {
     else SPMM_CASE(32, 2, 2)   // two neighbours in flight per lane beat four (fewer registers, more warps): measured
 #undef SPMM_CASE
     CU(cudaGetLastError());
-    if (cut) {
-      gk::k_spmm_long_rows<<<(unsigned)n_long, 64, 0, stream>>>(d_long_rows, reinterpret_cast<const float4*>(item_sums), o4, ld4);
-      CU(cudaGetLastError());
-      ++launches;   // booked with the propagation it completes
-    }
   }
 
   // C = A B.  B is handed over twice: row-major K x N (ldb) for the fp32-ALU kernels and K-major
@@ -1522,16 +1529,21 @@ int gcn_admm_index(gcn_admm* h, int which, int comm, const int** data, long long
   });
 }
 
+namespace {
+void ensure_shard_plan(gcn_admm* h, int n_ranks) {
+  if (h->shard_plan.n_ranks == n_ranks) return;
+  if (!gcn_admm_host::build_shard_plan(h->gi, n_ranks, h->shard_plan))
+    throw Fail{GCN_ADMM_ERR_ARG, "n_ranks must be between 1 and the number of communities"};
+  h->shard_ranges = h->shard_plan.comm_begin;
+  h->shard_ranges.insert(h->shard_ranges.end(), h->shard_plan.row_begin.begin(), h->shard_plan.row_begin.end());
+}
+}  // namespace
+
 int gcn_admm_shard_plan(gcn_admm* h, int n_ranks, int which, int receiver, int sender, const int** data, long long* len) {
   return guarded(h, [&] {
     if (!data || !len || which < GCN_ADMM_SHARD_RANGES || which > GCN_ADMM_SHARD_SECOND_ORDER)
       throw Fail{GCN_ADMM_ERR_ARG, "bad selector"};
-    if (h->shard_plan.n_ranks != n_ranks) {
-      if (!gcn_admm_host::build_shard_plan(h->gi, n_ranks, h->shard_plan))
-        throw Fail{GCN_ADMM_ERR_ARG, "n_ranks must be between 1 and the number of communities"};
-      h->shard_ranges = h->shard_plan.comm_begin;
-      h->shard_ranges.insert(h->shard_ranges.end(), h->shard_plan.row_begin.begin(), h->shard_plan.row_begin.end());
-    }
+    ensure_shard_plan(h, n_ranks);
     const std::vector<int>* v = &h->shard_ranges;
     if (which != GCN_ADMM_SHARD_RANGES) {
       if (receiver < 0 || receiver >= n_ranks || sender < 0 || sender >= n_ranks)
@@ -1541,6 +1553,102 @@ int gcn_admm_shard_plan(gcn_admm* h, int n_ranks, int which, int receiver, int s
     }
     *data = v->data();
     *len = (long long)v->size();
+  });
+}
+
+// The propagation as the ranks of a sharded run would carry it out, rank after rank on this one device.
+int gcn_admm_propagate_sharded(gcn_admm* h, int n_ranks, const float* x, int width, float* out, long long* staged_rows) {
+  return guarded(h, [&] {
+    if (!x || !out || width < 1 || width > kMaxWidth) throw Fail{GCN_ADMM_ERR_ARG, "bad argument"};
+    ensure_shard_plan(h, n_ranks);
+    const gcn_admm_host::ShardPlan& plan = h->shard_plan;
+    const gcn_admm_host::GraphIndex& g = h->gi;
+    const int ldw = ldpad(width), R = n_ranks;
+    const size_t rows = (size_t)h->n;
+    const bool dev_in = is_device_pointer(x), dev_out = is_device_pointer(out);
+    if (dev_in != dev_out) throw Fail{GCN_ADMM_ERR_ARG, "x and out must both be host or both be device pointers"};
+    std::vector<void*> mine;   // freed on every way out
+    auto take = [&](size_t bytes) { void* q = dalloc<char>(std::max<size_t>(bytes, 16)); mine.push_back(q); return q; };
+    auto release = [&] { for (void* q : mine) cudaFree(q); mine.clear(); };
+    long long staged = 0;
+    try {
+      float* dense = static_cast<float*>(take(rows * width * sizeof(float)));
+      float* a = static_cast<float*>(take(rows * ldw * sizeof(float)));
+      float* b = static_cast<float*>(take(rows * ldw * sizeof(float)));
+      CU(cudaMemcpyAsync(dense, x, rows * width * sizeof(float), dev_in ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice,
+                         h->stream));
+      gk::k_permute_rows<<<h->grid_for(h->n * ldw), 256, 0, h->stream>>>(dense, a, h->d_perm, h->n, width, ldw, 1);
+      CU(cudaGetLastError());
+      for (int r = 0; r < R; ++r) {
+        const int lo = plan.row_begin[r], hi = plan.row_begin[r + 1], n_own = hi - lo;
+        // rows this rank holds: its own, then the first-order rows of every sender (ascending in new ids,
+        // because senders own ascending row ranges)
+        std::vector<int> held((size_t)n_own);
+        for (int i = 0; i < n_own; ++i) held[(size_t)i] = lo + i;
+        for (int sdr = 0; sdr < R; ++sdr) {
+          const std::vector<int>& f = plan.first_order[(size_t)r * R + sdr];
+          held.insert(held.end(), f.begin(), f.end());
+        }
+        const int n_held = (int)held.size();
+        staged += n_held - n_own;
+        // local tables: the rank's rows of A + I with columns renumbered to positions in `held`
+        // (entry order kept, so every row is summed in the order of the unsharded kernel)
+        std::vector<int> rp((size_t)n_own + 1), order((size_t)n_own);
+        const long long e0 = g.row_ptr[lo], e1 = g.row_ptr[hi];
+        std::vector<int> cl((size_t)(e1 - e0));
+        std::vector<float> dv((size_t)n_held);
+        for (int k = 0; k < n_held; ++k) dv[(size_t)k] = g.dinv[(size_t)held[(size_t)k]];
+        for (int i = 0; i <= n_own; ++i) rp[(size_t)i] = (int)(g.row_ptr[lo + i] - e0);
+        for (long long e = e0; e < e1; ++e) {
+          const int j = g.col[(size_t)e];
+          int local;
+          if (j >= lo && j < hi) local = j - lo;
+          else {
+            const auto it = std::lower_bound(held.begin() + n_own, held.end(), j);
+            if (it == held.end() || *it != j) throw Fail{GCN_ADMM_ERR_CUDA, "plan misses a neighbour row"};
+            local = (int)(it - held.begin());
+          }
+          cl[(size_t)(e - e0)] = local;
+        }
+        for (int i = 0; i < n_own; ++i) order[(size_t)i] = i;
+        std::stable_sort(order.begin(), order.end(), [&](int p_, int q_) { return rp[p_ + 1] - rp[p_] > rp[q_ + 1] - rp[q_]; });
+        int* d_rp = static_cast<int*>(take(rp.size() * sizeof(int)));
+        int* d_cl = static_cast<int*>(take(cl.size() * sizeof(int)));
+        int* d_order = static_cast<int*>(take(order.size() * sizeof(int)));
+        int* d_held = static_cast<int*>(take(held.size() * sizeof(int)));
+        float* d_dv = static_cast<float*>(take(dv.size() * sizeof(float)));
+        float* xl = static_cast<float*>(take((size_t)n_held * ldw * sizeof(float)));
+        CU(cudaMemcpyAsync(d_rp, rp.data(), rp.size() * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+        if (!cl.empty()) CU(cudaMemcpyAsync(d_cl, cl.data(), cl.size() * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+        if (n_own > 0) CU(cudaMemcpyAsync(d_order, order.data(), order.size() * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+        if (n_held > 0) {
+          CU(cudaMemcpyAsync(d_held, held.data(), held.size() * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+          CU(cudaMemcpyAsync(d_dv, dv.data(), dv.size() * sizeof(float), cudaMemcpyHostToDevice, h->stream));
+          // own rows and, behind them, the copies of the first-order rows: on several devices the second part
+          // is what the receives from the rows' owners fill
+          gk::k_gather_rows<<<h->grid_for((long long)n_held * (ldw / 4)), 256, 0, h->stream>>>(
+              reinterpret_cast<const float4*>(a), d_held, reinterpret_cast<float4*>(xl), ldw / 4, n_held);
+          CU(cudaGetLastError());
+          ++h->launches;
+        }
+        if (n_own > 0) {
+          gcn_admm::Scope sc(h, "spmm.sharded", 1, 0.0, 0.0);
+          h->spmm_launch(d_rp, d_cl, d_dv, d_order, n_own, nullptr, 0, INT_MAX, xl, b + (size_t)lo * ldw, ldw);
+        }
+        CU(cudaStreamSynchronize(h->stream));   // the host vectors of this rank go out of scope
+      }
+      gk::k_permute_rows<<<h->grid_for(h->n * ldw), 256, 0, h->stream>>>(b, dense, h->d_perm, h->n, width, ldw, 0);
+      CU(cudaGetLastError());
+      h->launches += 2;   // the two row permutations
+      CU(cudaMemcpyAsync(out, dense, rows * width * sizeof(float), dev_out ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost,
+                         h->stream));
+      CU(cudaStreamSynchronize(h->stream));
+    } catch (...) {
+      release();
+      throw;
+    }
+    release();
+    if (staged_rows) *staged_rows = staged;
   });
 }
 

@@ -1581,6 +1581,17 @@ __global__ void k_fill_int(int* __restrict__ p, long long count, int value) {
 
 // Row gather / scatter between the caller's dense layout (original order, width C) and the
 // internal one (community order, leading dimension ld).  to_internal != 0: dst[new] = src[perm[new]].
+// dst[r] = src[rows[r]] for padded rows of ld4 float4: the staging copy of the rows a rank does not own
+// (what a receive from their owners would deliver) behind its own rows.
+__global__ void k_gather_rows(const float4* __restrict__ src, const int* __restrict__ rows, float4* __restrict__ dst,
+                              int ld4, long long count) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count * ld4;
+       i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i / ld4;
+    dst[i] = src[(long long)rows[r] * ld4 + (i - r * ld4)];
+  }
+}
+
 __global__ void k_permute_rows(const float* __restrict__ src, float* __restrict__ dst, const int* __restrict__ perm,
                                long long n, int C, int ld, int to_internal) {
   const long long total = n * ld;
