@@ -60,8 +60,9 @@ enum {
  *                  1e-7 of sum |a||b|); products of 16384 rows or more first split the weight operand once
  *                  into the staged layout and fetch it with bulk copies (smaller ones re-split it per row
  *                  tile, which is cheaper than another launch), and with at most 128 output columns they also
- *                  fetch the tiles of the row operand by tensor copies; 2: the same kernels, pre-split at
- *                  every size; 0: fp32 FMA kernels everywhere
+ *                  fetch the tiles of the row operand by tensor copies (products with 129 to 256 output columns
+ *                  and K <= 128 run in that form as two groups of 128 columns); 2: the same kernels, pre-split
+ *                  at every size; 0: fp32 FMA kernels everywhere
  *  use_graph       1: gcn_admm_step records one pass as a CUDA graph on first use and replays it (only when
  *                  the handle's stream is not the default stream and profiling is off); 2: the same, but
  *                  only for problems small enough for launch gaps to show (N x widest layer < 2^27);
