@@ -50,3 +50,30 @@ def test_more_ranks_than_communities_is_refused(case):
     with pytest.raises(Exception):
         g.propagate_sharded(wl.n_comm + 1, x)
     g.propagate_sharded(wl.n_comm, x)          # the handle is still usable
+
+
+def test_rank_sums_of_the_weight_gradient(case):
+    """Section 3.1: the W agent adds up what the community agents send.  P^T R over each rank's row range by the
+    library's transposed product, summed over the ranks (the all-reduce), against fp64 and the unsharded product."""
+    import torch
+    wl, g, _ = case
+    n_ranks = min(4, wl.n_comm)
+    ranges = g.shard_plan(n_ranks, 0)
+    row_begin = ranges[n_ranks + 1:]
+    rng = np.random.default_rng(3)
+    ka, nb = 37, 24
+    p = rng.standard_normal((wl.n, ka)).astype(np.float32)
+    r = rng.standard_normal((wl.n, nb)).astype(np.float32)
+    tp, tr = torch.from_numpy(p).cuda(), torch.from_numpy(r).cuda()
+    whole = torch.empty((ka, nb), device="cuda")
+    g.dense_product_tn(tp.data_ptr(), tr.data_ptr(), whole.data_ptr(), wl.n, ka, nb)
+    total = np.zeros((ka, nb))
+    for k in range(n_ranks):
+        lo, hi = int(row_begin[k]), int(row_begin[k + 1])
+        part = torch.empty((ka, nb), device="cuda")
+        g.dense_product_tn(tp[lo:hi].data_ptr(), tr[lo:hi].data_ptr(), part.data_ptr(), hi - lo, ka, nb)
+        total += part.cpu().numpy().astype(np.float64)
+    want = p.astype(np.float64).T @ r.astype(np.float64)
+    scale = np.abs(p).astype(np.float64).T @ np.abs(r).astype(np.float64)
+    assert np.max(np.abs(total - want) / scale) < 2e-6
+    assert np.max(np.abs(total - whole.cpu().numpy()) / scale) < 2e-6
